@@ -1,0 +1,158 @@
+/*
+ * compactor.h - C ABI of the B200 (sm_100a) implementation of Compactor's prefill-time KV-cache
+ * compression pass: approximate leverage scoring of the keys (Algorithm 1), optional blend with
+ * a caller-supplied attention score (Eq. 6), per-head top-ceil(r N) selection (Section 3.4) and
+ * compaction of the retained K/V rows into a dense per-head cache.
+ *
+ * Conventions
+ *   - Every function returns an int status: COMPACTOR_OK (0) or a negative COMPACTOR_E_* code.
+ *     Nothing throws.  Argument errors are detected before any work is enqueued.
+ *   - "device" pointers are CUDA device pointers of the current device; "host" pointers are
+ *     ordinary host memory, read before the call returns.  The library never allocates or frees
+ *     device memory: every buffer, including the workspace, belongs to the caller.
+ *   - Device work is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
+ *     void*; NULL is the default stream) and the call returns without synchronising.
+ *   - Keys/values are bf16 with the d channels of a token contiguous; the other three strides
+ *     (layer, KV head, token) are given in ELEMENTS and must be multiples of 8 (16 bytes); base
+ *     pointers must be 16-byte aligned.  d must be 128.  1 <= m <= 64.
+ *   - Sequences are packed back to back along the token axis: sequence b owns tokens
+ *     [cu_seqlens[b], cu_seqlens[b+1]) of every (layer, head).  A "unit" is one
+ *     (layer, head, sequence) triple; unit id = (layer * heads + head) * batch + b.
+ *     Units are scored and selected independently (Section 3: "the same procedure is applied
+ *     to heads independently").
+ *   - Kept rows of sequence b occupy rows [cu_keep[b], cu_keep[b+1]) of every (layer, head)
+ *     block of the outputs, cu_keep = prefix sums of keep_counts; total_keep = cu_keep[batch].
+ *   - Outputs must not alias inputs or the workspace.
+ *   - `status` (device, int32 [layers*heads*batch], may be NULL) receives per-unit flags once the
+ *     stream has run: bit 0 = the unit's Gram matrix held a non-finite value (scores of the unit
+ *     are unspecified), bit 1 = the sketched Gram matrix was numerically rank deficient (the
+ *     singular directions contribute nothing, as a pseudo-inverse would), bit 2 = a bounded
+ *     device-side wait ran out.
+ */
+#ifndef COMPACTOR_H_
+#define COMPACTOR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define COMPACTOR_OK                  0
+#define COMPACTOR_E_INVALID_ARGUMENT -1   /* null pointer, bad size, bad stride or alignment      */
+#define COMPACTOR_E_UNSUPPORTED      -2   /* d != 128 or m outside [1, 64]                       */
+#define COMPACTOR_E_WORKSPACE        -3   /* workspace smaller than compactor_workspace_bytes()  */
+#define COMPACTOR_E_CUDA             -4   /* a CUDA runtime call failed (see cudaGetLastError)   */
+
+#define COMPACTOR_STATUS_NONFINITE   1
+#define COMPACTOR_STATUS_RANK        2
+#define COMPACTOR_STATUS_TIMEOUT     4
+
+/* A strided bf16 tensor [layers][heads][total_tokens][d] in device memory. */
+typedef struct compactor_mat {
+    const void* ptr;          /* device, 16-byte aligned                           */
+    int64_t stride_layer;     /* elements between consecutive layers               */
+    int64_t stride_head;      /* elements between consecutive KV heads             */
+    int64_t stride_token;     /* elements between consecutive tokens (>= d)        */
+} compactor_mat;
+
+/* Problem shape.  cu_seqlens is a HOST array of batch+1 non-decreasing offsets starting at 0. */
+typedef struct compactor_shape {
+    int32_t layers;
+    int32_t heads;
+    int32_t d;                /* head dimension; must be 128                       */
+    int32_t m;                /* sketch dimension (the paper uses 48)              */
+    int32_t batch;            /* number of packed sequences                        */
+    const int32_t* cu_seqlens;/* host, [batch+1]                                   */
+} compactor_shape;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int compactor_version(void);
+
+/* Static description of a status code. */
+const char* compactor_error_string(int code);
+
+/*
+ * Algorithm 1, line 1: a Gaussian sketch Phi [d][m] (row-major fp32, HOST memory) with iid
+ * N(0, 1/m) entries from a counter-based generator, so that any caller can reproduce it:
+ * word i = splitmix64 finaliser of seed + (i+1)*0x9E3779B97F4A7C15; words (2p, 2p+1) give
+ * u1 = ((x>>11)+1) 2^-53 and u2 = (x>>11) 2^-53; Box-Muller (sqrt(-2 ln u1) cos/sin(2 pi u2))
+ * gives row-major entries 2p and 2p+1, each divided by sqrt(m) in double and rounded to fp32.
+ * Any other Phi may be passed to the scoring calls instead; scores do not depend on its scale.
+ */
+int compactor_make_sketch(uint64_t seed, int32_t d, int32_t m, float* phi_host);
+
+/*
+ * Number of retained tokens for a sequence of n tokens at retention ratio r (Section 3,
+ * Preliminaries: k = ceil(r N)): ceil evaluated on the double product, clamped to [1, n];
+ * 0 when n <= 0.  Returns the count (never an error code).
+ */
+int64_t compactor_keep_count(int64_t n, double r);
+
+/*
+ * Context-calibrated retention (Section 3.5): with b = alpha*nll + beta and the fitted curve
+ * f(r) = (exp(rb-b) - exp(-b)) / (1 - exp(-b)), writes the r with f(r) = tau, i.e.
+ * r* = log(1 + tau*(e^b - 1)) / b (r* = tau when b = 0).  tau must lie in (0, 1].
+ */
+int compactor_calibrated_ratio(double nll, double alpha, double beta, double tau, double* r_out);
+
+/*
+ * Bytes of device workspace that compactor_score / compactor_select / compactor_compress need
+ * for this shape (the maximum over the three).  Returns 0 for an invalid shape.
+ */
+size_t compactor_workspace_bytes(const compactor_shape* shape);
+
+/*
+ * Approximate leverage scores of every unit (Algorithm 1, lines 2-6) and the blend of Eq. 6.
+ *   k_score      keys to score (the paper scores the keys before positional encoding).
+ *   phi          device, fp32 [d][m] row-major: the sketch, shared by all units.
+ *   attn_scores  device fp32 [layers][heads][total_tokens] or NULL.  If given, the output is
+ *                s = z(attn) + lambda * z(o) per unit (population std; a term with zero std
+ *                contributes 0); if NULL the output is the outlier score o itself.
+ *   scores_out   device fp32 [layers][heads][total_tokens].
+ * The small factorisation is a Cholesky factorisation of G = (K Phi)^T (K Phi) in fp64 - one of
+ * the algebraically equal routes the paper allows (Section 3.2, Appendix C); Gram sums are fp32
+ * per block of at most 8192 tokens and fp64 across blocks.
+ */
+int compactor_score(const compactor_shape* shape, compactor_mat k_score, const float* phi,
+                    const float* attn_scores, float lambda, float* scores_out,
+                    int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Per-unit top-k (Section 3.4, "retain the top ceil(r N) tokens ... within a single head").
+ *   scores       device fp32 [layers][heads][total_tokens].
+ *   keep_counts  host int32 [batch]: tokens kept per sequence (0 <= keep <= length), the same
+ *                for every layer and head.
+ *   idx_out      device int32 [layers][heads][total_keep]: for each unit the indices (local to
+ *                the sequence, 0-based) of its keep_counts[b] largest scores, ascending.  Equal
+ *                scores are ranked by lower index first.  NaN scores rank above +inf.
+ */
+int compactor_select(const compactor_shape* shape, const float* scores,
+                     const int32_t* keep_counts, int32_t* idx_out,
+                     int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Compaction: k_out[l][h][cu_keep[b]+j][:] = k_cache[l][h][cu_seqlens[b]+idx[l][h][cu_keep[b]+j]][:]
+ * and likewise for v, as bit copies.  k_out / v_out are dense bf16 [layers][heads][total_keep][d].
+ * Indices outside [0, length) are skipped (their output rows are left untouched).
+ */
+int compactor_compact(const compactor_shape* shape, compactor_mat k_cache, compactor_mat v_cache,
+                      const int32_t* idx, const int32_t* keep_counts,
+                      void* k_out, void* v_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The whole pass: score k_score, select, and gather rows of k_cache / v_cache.
+ * k_score may be the same tensor as k_cache.  scores_out may be NULL (scores then live only in
+ * the workspace); idx_out, k_out, v_out as above.
+ */
+int compactor_compress(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
+                       compactor_mat v_cache, const float* phi, const float* attn_scores,
+                       float lambda, const int32_t* keep_counts,
+                       float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
+                       int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COMPACTOR_H_ */

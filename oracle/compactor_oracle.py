@@ -1,0 +1,213 @@
+"""CPU oracle for Compactor's prefill-time compression pass.  TEST INFRASTRUCTURE.
+
+A plain, slow, fp64 numpy statement of what the pass computes, written from the
+paper so that a reader can check it by eye.  It shares nothing with the CUDA
+library (no code, tables, constants or pre/post-processing) and must only be
+used by the tests, the smoke check and the benchmark's CPU-baseline leg -
+never by the product path.
+
+What follows the paper step by step:
+  * `approx_leverage_scores` - Algorithm 1 (Gaussian right sketch, Gram matrix,
+    small SVD, back-projection, squared row norms).
+  * `exact_leverage_scores`  - Definition 1 / Eq. 1 (the quantity Algorithm 1
+    approximates; used to pin the oracle, and as the m = d special case).
+  * `blend`                  - Eq. 6 (z-scored attention term + lambda * z-scored
+    outlier term).
+  * `keep_count`             - "retain the top ceil(r N) tokens" (Section 3,
+    Preliminaries; Section 3.4).
+  * `top_k_indices`          - per-head top-k of the scores.
+  * `compact`                - the retained rows of K and V.
+  * `calibrated_ratio`       - inverse of the fitted curve f_{alpha,beta}
+    (Section 3.5).
+
+Readings taken where the paper is silent or inconsistent:
+  * Eq. 1 prints diag(U^T U); Definition 1 and Algorithm 1's last line make it
+    the squared row norms diag(U U^T).
+  * Sigma^-1 in Algorithm 1 is a pseudo-inverse: singular directions of G with
+    lambda_j <= m * 2^-52 * lambda_max contribute nothing (Algorithm 1 has no
+    clamp; the 1e-6 clamp appears only in Appendix C's eigen variant).
+  * Entries of Phi have variance 1/m (Algorithm 1, line 1); the scale does not
+    change the scores.
+  * Ties in the top-k go to the lower token index, and the kept indices are
+    emitted in ascending order (the paper does not say).
+  * std in Eq. 6 is the population standard deviation; a term whose std is 0
+    contributes 0.  With no attention term the score is the outlier score o.
+  * The calibration curve is increasing in r; the paper's "arg max ... such
+    that f >= tau" is read as the smallest such r (Section 3.5 opens with
+    "the smallest r that leaves model quality unchanged").
+
+Pins (see tests/test_oracle_pins.py): closed-form leverage scores, sum = rank,
+range [0,1], invariance under K -> K A and Phi -> Phi A, m = d reduces to the
+exact scores, Phi = e_1, n <= m gives all ones, agreement with a QR route
+(Appendix C), brute-force top-k, f(r*) = tau.  Agreement with the authors'
+own engine outputs is "parity unpinned": the paper prints no score values,
+indices or worked example for this path.
+"""
+from __future__ import annotations
+
+import math
+
+import numpy as np
+
+
+# ----------------------------------------------------------------------------
+# Input widening (data handling only)
+# ----------------------------------------------------------------------------
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Widen bf16 bit patterns (uint16 / int16) exactly to float64."""
+    u = np.ascontiguousarray(bits).view(np.uint16).astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 1, line 1: the Gaussian sketch from a seed
+# ----------------------------------------------------------------------------
+def make_sketch(seed: int, d: int, m: int) -> np.ndarray:
+    """Phi [d, m] fp32 with iid N(0, 1/m) entries from a counter-based generator:
+    word i (i = 0, 1, ...) is the splitmix64 finaliser of seed + (i+1)*0x9E3779B97F4A7C15;
+    words (2p, 2p+1) give u1 = ((x >> 11) + 1) 2^-53 in (0,1] and u2 = (x >> 11) 2^-53 in
+    [0,1); Box-Muller turns them into the row-major entries 2p and 2p+1; each is divided by
+    sqrt(m) in double and rounded to fp32."""
+    count = d * m
+    pairs = (count + 1) // 2
+    mask = (1 << 64) - 1
+
+    def word(i):
+        z = (seed + (i + 1) * 0x9E3779B97F4A7C15) & mask
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & mask
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & mask
+        return z ^ (z >> 31)
+
+    out = np.empty(2 * pairs, dtype=np.float64)
+    for p in range(pairs):
+        u1 = ((word(2 * p) >> 11) + 1) * 2.0 ** -53
+        u2 = (word(2 * p + 1) >> 11) * 2.0 ** -53
+        rad = math.sqrt(-2.0 * math.log(u1))
+        out[2 * p] = rad * math.cos(2.0 * math.pi * u2)
+        out[2 * p + 1] = rad * math.sin(2.0 * math.pi * u2)
+    return (out[:count] / math.sqrt(m)).astype(np.float32).reshape(d, m)
+
+
+# ----------------------------------------------------------------------------
+# Definition 1 / Eq. 1: exact leverage scores
+# ----------------------------------------------------------------------------
+def exact_leverage_scores(K: np.ndarray) -> np.ndarray:
+    """l_i = ||U_i||^2 with K = U Sigma V^T the thin SVD, U restricted to the
+    numerically non-zero singular values (Definition 1)."""
+    K = np.asarray(K, dtype=np.float64)
+    n, d = K.shape
+    if n == 0:
+        return np.zeros(0)
+    U, sig, _ = np.linalg.svd(K, full_matrices=False)
+    if sig.size == 0 or sig[0] == 0.0:
+        return np.zeros(n)
+    rank = int(np.sum(sig > max(n, d) * np.finfo(np.float64).eps * sig[0]))
+    return np.sum(U[:, :rank] ** 2, axis=1)
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 1: approximate leverage scores
+# ----------------------------------------------------------------------------
+def approx_leverage_scores(K: np.ndarray, Phi: np.ndarray) -> np.ndarray:
+    """Algorithm 1, lines 2-6, for a given sketch Phi [d, m] (line 1 is the
+    caller's draw of Phi)."""
+    K = np.asarray(K, dtype=np.float64)
+    Phi = np.asarray(Phi, dtype=np.float64)
+    n = K.shape[0]
+    m = Phi.shape[1]
+    if n == 0:
+        return np.zeros(0)
+    K_hat = K @ Phi                                   # line 2
+    G = K_hat.T @ K_hat                               # line 3
+    V_t, lam, _ = np.linalg.svd(G)                    # line 4: G = V Sigma^2 V^T
+    lam_max = lam[0] if lam.size else 0.0
+    if lam_max <= 0.0:
+        return np.zeros(n)
+    keep = lam > m * 2.0 ** -52 * lam_max             # pseudo-inverse of Sigma
+    sigma = np.sqrt(lam[keep])
+    U_t = (K_hat @ V_t[:, keep]) / sigma[None, :]     # line 5
+    return np.sum(U_t * U_t, axis=1)                  # line 6: diag(U U^T)
+
+
+# ----------------------------------------------------------------------------
+# Eq. 6: blend
+# ----------------------------------------------------------------------------
+def _zscore(x: np.ndarray) -> np.ndarray:
+    mu = np.mean(x)
+    sd = np.sqrt(np.mean((x - mu) ** 2))
+    if sd == 0.0:
+        return np.zeros_like(x)
+    return (x - mu) / sd
+
+
+def blend(a, o: np.ndarray, lam: float) -> np.ndarray:
+    """s = z(a) + lam * z(o) (Eq. 6).  With a = None the score is o itself."""
+    o = np.asarray(o, dtype=np.float64)
+    if a is None:
+        return o.copy()
+    a = np.asarray(a, dtype=np.float64)
+    if o.size == 0:
+        return o.copy()
+    return _zscore(a) + float(lam) * _zscore(o)
+
+
+# ----------------------------------------------------------------------------
+# Selection
+# ----------------------------------------------------------------------------
+def keep_count(n: int, r: float) -> int:
+    """ceil(r * n) evaluated in double precision, clamped to [1, n] (0 if n = 0)."""
+    n = int(n)
+    if n <= 0:
+        return 0
+    return min(n, max(1, int(math.ceil(float(r) * float(n)))))
+
+
+def top_k_indices(s: np.ndarray, kk: int) -> np.ndarray:
+    """Indices of the kk largest scores; equal scores are ranked by lower index
+    first; result in ascending index order."""
+    s = np.asarray(s)
+    n = s.shape[0]
+    kk = int(kk)
+    order = np.lexsort((np.arange(n), -s))            # primary key -s, then index
+    return np.sort(order[:kk]).astype(np.int32)
+
+
+def compact(K_bits: np.ndarray, V_bits: np.ndarray, idx: np.ndarray):
+    """K'[j] = K[idx[j]], V'[j] = V[idx[j]] as bit copies."""
+    idx = np.asarray(idx, dtype=np.int64)
+    return K_bits[idx].copy(), V_bits[idx].copy()
+
+
+# ----------------------------------------------------------------------------
+# Section 3.5: context-calibrated ratio
+# ----------------------------------------------------------------------------
+def calibration_curve(r: float, b: float) -> float:
+    """f(r) = (exp(r b - b) - exp(-b)) / (1 - exp(-b)); f(r) = r in the limit b -> 0."""
+    if b == 0.0:
+        return float(r)
+    return (math.exp(r * b - b) - math.exp(-b)) / (1.0 - math.exp(-b))
+
+
+def calibrated_ratio(nll: float, alpha: float, beta: float, tau: float) -> float:
+    """The r in (0,1] with f_{alpha,beta}(r) = tau, b = alpha * nll + beta:
+    r* = log(1 + tau (e^b - 1)) / b, and r* = tau when b = 0."""
+    b = float(alpha) * float(nll) + float(beta)
+    if b == 0.0:
+        return float(tau)
+    return math.log1p(float(tau) * math.expm1(b)) / b
+
+
+# ----------------------------------------------------------------------------
+# The whole pass for one unit
+# ----------------------------------------------------------------------------
+def compress_unit(K_score_bits, K_cache_bits, V_bits, Phi, kk, attn=None, lam=0.3):
+    """Score, select and compact one (sequence, layer, head) unit.
+
+    *_bits are bf16 bit patterns [n, d] (uint16); Phi fp32/fp64 [d, m]; attn an
+    optional fp32 [n].  Returns (scores fp64 [n], idx int32 [kk], K' bits, V' bits)."""
+    K = bf16_bits_to_f64(np.asarray(K_score_bits))
+    o = approx_leverage_scores(K, np.asarray(Phi, dtype=np.float64))
+    s = blend(None if attn is None else np.asarray(attn, dtype=np.float64), o, lam)
+    idx = top_k_indices(s, kk)
+    Kc, Vc = compact(np.asarray(K_cache_bits), np.asarray(V_bits), idx)
+    return s, idx, Kc, Vc

@@ -1,0 +1,250 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle's
+own formulae.  No GPU needed."""
+import itertools
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import compactor_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+# ----------------------------------------------------------------------------- exact leverage
+def _closed_form_cases():
+    cases, name, rows = [], None, []
+    for line in open(os.path.join(GOLDEN, "leverage_closed_forms.txt")):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        if line.startswith("case "):
+            name, rows = line.split()[1], []
+        elif line.startswith("scores:"):
+            want = [float(Fraction(t)) for t in line.split()[1:]]
+            cases.append((name, np.array(rows, dtype=np.float64), np.array(want)))
+        else:
+            rows.append([float(t) for t in line.split()])
+    return cases
+
+
+@pytest.mark.parametrize("name,K,want", _closed_form_cases(), ids=lambda c: c if isinstance(c, str) else "")
+def test_exact_leverage_closed_forms(name, K, want):
+    np.testing.assert_allclose(orc.exact_leverage_scores(K), want, atol=1e-12)
+
+
+def test_exact_leverage_hadamard_columns_are_uniform():
+    # n x d matrix whose columns are d columns of a +-1 Hadamard matrix: K^T K = n I, so l_i = d / n.
+    H = np.array([[1.0]])
+    for _ in range(5):
+        H = np.block([[H, H], [H, -H]])
+    K = H[:, [1, 5, 9, 20, 31]] * 0.37
+    np.testing.assert_allclose(orc.exact_leverage_scores(K), np.full(32, 5 / 32), atol=1e-12)
+
+
+def test_exact_leverage_matches_gram_inverse_and_qr():
+    # Eq. 2: U = K V Sigma^-1  =>  l_i = k_i (K^T K)^-1 k_i^T; Appendix C: l_i = ||Q_i||^2 for K = QR.
+    K = _rng(1).standard_normal((200, 7)) * np.array([1, 10, 0.1, 3, 1, 1, 5.0])
+    ell = orc.exact_leverage_scores(K)
+    via_gram = np.einsum("ij,jk,ik->i", K, np.linalg.inv(K.T @ K), K)
+    Q, _ = np.linalg.qr(K)
+    np.testing.assert_allclose(ell, via_gram, rtol=1e-9)
+    np.testing.assert_allclose(ell, np.sum(Q * Q, axis=1), rtol=1e-10)
+
+
+def test_exact_leverage_invariants():
+    rng = _rng(2)
+    K = rng.standard_normal((300, 6))
+    K[:, 5] = K[:, 0] - 2 * K[:, 1]                      # rank 5
+    ell = orc.exact_leverage_scores(K)
+    assert np.all(ell >= -1e-12) and np.all(ell <= 1 + 1e-12)
+    assert abs(ell.sum() - 5.0) < 1e-9                   # sum = rank(K)
+    A = rng.standard_normal((6, 6)) + 3 * np.eye(6)
+    np.testing.assert_allclose(orc.exact_leverage_scores(K @ A), ell, atol=1e-9)   # K -> K A
+    perm = rng.permutation(300)
+    np.testing.assert_allclose(orc.exact_leverage_scores(K[perm]), ell[perm], atol=1e-10)
+
+
+# ----------------------------------------------------------------------------- Algorithm 1
+def test_alg1_full_sketch_equals_exact():
+    rng = _rng(3)
+    K = rng.standard_normal((500, 16)) * (np.arange(1, 17) ** -1.0)
+    Phi = rng.standard_normal((16, 16))                  # m = d, invertible
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, Phi), orc.exact_leverage_scores(K), rtol=1e-7)
+
+
+def test_alg1_single_column_sketch():
+    # Phi = e_1 (m = 1): K_hat is the first column, so o_i = K_i1^2 / sum_j K_j1^2.
+    K = np.array([[1.0, 0.0], [0.0, 1.0], [1.0, 1.0]])
+    e1 = np.array([[1.0], [0.0]])
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, e1), [0.5, 0.0, 0.5], atol=1e-14)
+    K = _rng(4).standard_normal((50, 8))
+    e3 = np.zeros((8, 1)); e3[3] = 1.0
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, e3), K[:, 3] ** 2 / np.sum(K[:, 3] ** 2), rtol=1e-12)
+
+
+def test_alg1_invariants():
+    rng = _rng(5)
+    n, d, m = 400, 32, 12
+    K = rng.standard_normal((n, d)) * (np.arange(1, d + 1) ** -0.7) + 0.5 * rng.standard_normal(d)
+    Phi = rng.standard_normal((d, m)) / math.sqrt(m)
+    o = orc.approx_leverage_scores(K, Phi)
+    ell = orc.exact_leverage_scores(K)
+    assert abs(o.sum() - m) < 1e-8                         # sum = rank(K Phi)
+    assert np.all(o >= 0) and np.all(o <= ell + 1e-9)      # projection onto a subspace of col(K)
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, 7.5 * Phi), o, rtol=1e-9)       # scale of Phi
+    A = rng.standard_normal((m, m)) + 2 * np.eye(m)
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, Phi @ A), o, rtol=1e-8)         # Phi -> Phi A
+    extra = rng.standard_normal((d, 3))
+    o_more = orc.approx_leverage_scores(K, np.hstack([Phi, extra]))
+    assert np.all(o_more >= o - 1e-10)                     # appending columns never lowers a score
+    perm = rng.permutation(n)
+    np.testing.assert_allclose(orc.approx_leverage_scores(K[perm], Phi), o[perm], rtol=1e-9)
+
+
+def test_alg1_matches_qr_route():
+    # Appendix C: K_hat = QR, score = ||Q_i||^2.
+    rng = _rng(6)
+    K = rng.standard_normal((700, 24))
+    Phi = rng.standard_normal((24, 9))
+    Q, _ = np.linalg.qr(K @ Phi)
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, Phi), np.sum(Q * Q, axis=1), rtol=1e-9)
+
+
+def test_alg1_rank_deficient_cases():
+    rng = _rng(7)
+    Phi = rng.standard_normal((16, 8))
+    # fewer rows than sketch columns, full row rank: K_hat K_hat^+ = I_n, every score is 1
+    K = rng.standard_normal((5, 16))
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, Phi), np.ones(5), atol=1e-9)
+    # all-zero keys: no direction survives, all scores 0
+    np.testing.assert_array_equal(orc.approx_leverage_scores(np.zeros((9, 16)), Phi), np.zeros(9))
+    # copies of one row: rank 1, scores 1/n each
+    K = np.tile(rng.standard_normal((1, 16)), (10, 1))
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, Phi), np.full(10, 0.1), atol=1e-9)
+    # empty
+    assert orc.approx_leverage_scores(np.zeros((0, 16)), Phi).shape == (0,)
+
+
+def test_alg1_detects_a_transposed_or_dropped_factor():
+    # An independent construction of the same number: o_i = k_hat_i G^+ k_hat_i^T.
+    rng = _rng(8)
+    K = rng.standard_normal((60, 10)); Phi = rng.standard_normal((10, 4))
+    Kh = K @ Phi
+    want = np.einsum("ij,jk,ik->i", Kh, np.linalg.pinv(Kh.T @ Kh), Kh)
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, Phi), want, rtol=1e-9)
+
+
+def test_bf16_widening_is_exact():
+    import torch
+    x = torch.randn(1000, dtype=torch.float32).to(torch.bfloat16)
+    bits = x.view(torch.int16).numpy()
+    np.testing.assert_array_equal(orc.bf16_bits_to_f64(bits), x.double().numpy())
+
+
+# ----------------------------------------------------------------------------- sketch generator
+def test_make_sketch_statistics_and_determinism():
+    P = orc.make_sketch(7, 128, 48)
+    assert P.dtype == np.float32 and P.shape == (128, 48)
+    np.testing.assert_array_equal(P, orc.make_sketch(7, 128, 48))
+    assert not np.array_equal(P, orc.make_sketch(8, 128, 48))
+    z = P.astype(np.float64) * math.sqrt(48)
+    assert abs(z.mean()) < 0.05 and abs(z.std() - 1.0) < 0.05
+    assert abs(np.mean(z ** 4) - 3.0) < 0.3                # Gaussian fourth moment
+    # first word of the splitmix64 stream for seed 0 is the published test value of that generator
+    x = (0 + 0x9E3779B97F4A7C15) & (2 ** 64 - 1)
+    x = ((x ^ (x >> 30)) * 0xBF58476D1CE4E5B9) & (2 ** 64 - 1)
+    x = ((x ^ (x >> 27)) * 0x94D049BB133111EB) & (2 ** 64 - 1)
+    x ^= x >> 31
+    assert x == 0xE220A8397B1DCDAF
+
+
+# ----------------------------------------------------------------------------- blend (Eq. 6)
+def test_blend_properties():
+    rng = _rng(9)
+    a = np.exp(rng.standard_normal(500)); o = rng.random(500)
+    s = orc.blend(a, o, 0.3)
+    za = (a - a.mean()) / a.std(); zo = (o - o.mean()) / o.std()
+    np.testing.assert_allclose(s, za + 0.3 * zo, rtol=1e-12)
+    assert abs(s.mean()) < 1e-12
+    # affine changes of either term leave s unchanged
+    np.testing.assert_allclose(orc.blend(3 * a + 2, 0.5 * o - 1, 0.3), s, atol=1e-10)
+    # lambda -> 0 ranks like a; constant a ranks like o; no a returns o
+    assert np.array_equal(np.argsort(orc.blend(a, o, 0.0)), np.argsort(a))
+    assert np.array_equal(np.argsort(orc.blend(np.full(500, 2.0), o, 0.3)), np.argsort(o))
+    np.testing.assert_array_equal(orc.blend(None, o, 0.3), o)
+    # hand example: a = (1,3), o = (0,2): z = (-1,1) for both
+    np.testing.assert_allclose(orc.blend([1.0, 3.0], [0.0, 2.0], 0.5), [-1.5, 1.5], atol=1e-15)
+
+
+# ----------------------------------------------------------------------------- keep count / r*
+def test_keep_count_golden():
+    for line in open(os.path.join(GOLDEN, "keep_counts.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        n, r, want = line.split()
+        assert orc.keep_count(int(n), float(r)) == int(want)
+    assert orc.keep_count(0, 0.5) == 0 and orc.keep_count(5, 1e-9) == 1 and orc.keep_count(5, 1.0) == 5
+
+
+def test_calibrated_ratio():
+    for line in open(os.path.join(GOLDEN, "calibrated_ratio.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        b, tau, want = map(float, line.split())
+        assert abs(orc.calibrated_ratio(1.0, b, 0.0, tau) - want) < 1e-6
+        assert abs(orc.calibrated_ratio(2.0, b / 4, b / 2, tau) - want) < 1e-6       # b = alpha nll + beta
+    for b in (-12.0, -3.0, -0.5, 1e-9, 0.7, 5.0):
+        assert abs(orc.calibration_curve(1.0, b) - 1.0) < 1e-12           # f(1) = 1
+        assert abs(orc.calibration_curve(0.0, b)) < 1e-12                 # f(0) = 0
+        for tau in (0.5, 0.9, 0.95, 1.0):
+            r = orc.calibrated_ratio(1.0, b, 0.0, tau)
+            assert 0.0 < r <= 1.0
+            assert abs(orc.calibration_curve(r, b) - tau) < 1e-7          # f(r*) = tau
+    assert orc.calibrated_ratio(1.0, 0.0, 0.0, 0.9) == 0.9                # b = 0: the straight line
+    # more compressible (more negative b) => smaller r*
+    assert orc.calibrated_ratio(1.0, -10, 0, 0.95) < orc.calibrated_ratio(1.0, -4, 0, 0.95)
+
+
+# ----------------------------------------------------------------------------- top-k
+def _brute_topk(s, kk):
+    order = sorted(range(len(s)), key=lambda i: (-s[i], i))
+    return sorted(order[:kk])
+
+
+def test_topk_exhaustive_small_with_ties():
+    for n in range(1, 7):
+        for s in itertools.product([0.0, 1.0, 2.0], repeat=n):
+            for kk in range(1, n + 1):
+                assert orc.top_k_indices(np.array(s), kk).tolist() == _brute_topk(s, kk)
+
+
+def test_topk_random_and_edges():
+    rng = _rng(10)
+    s = np.round(rng.random(3000), 2)                     # many ties
+    for kk in (1, 2, 1500, 2999, 3000):
+        got = orc.top_k_indices(s, kk)
+        assert got.dtype == np.int32 and got.tolist() == _brute_topk(s.tolist(), kk)
+    assert orc.top_k_indices(np.full(10, 0.5), 4).tolist() == [0, 1, 2, 3]
+    assert orc.top_k_indices(np.array([-1.0, -3.0, -2.0]), 2).tolist() == [0, 2]
+
+
+# ----------------------------------------------------------------------------- compaction / whole unit
+def test_compact_and_compress_unit():
+    import torch
+    rng = _rng(11)
+    n, d, m = 300, 128, 48
+    K = torch.randn(n, d).to(torch.bfloat16); V = torch.randn(n, d).to(torch.bfloat16)
+    kb, vb = K.view(torch.int16).numpy(), V.view(torch.int16).numpy()
+    Phi = (rng.standard_normal((d, m)) / math.sqrt(m)).astype(np.float32)
+    s, idx, Kc, Vc = orc.compress_unit(kb, kb, vb, Phi, orc.keep_count(n, 0.3))
+    assert len(idx) == 90 and np.all(np.diff(idx) > 0)
+    np.testing.assert_array_equal(Kc, kb[idx]); np.testing.assert_array_equal(Vc, vb[idx])
+    assert s[idx].min() >= np.delete(s, idx).max()
+    assert abs(s.sum() - m) < 1e-8

@@ -98,8 +98,10 @@ int64_t compactor_keep_count(int64_t n, double r);
 int compactor_calibrated_ratio(double nll, double alpha, double beta, double tau, double* r_out);
 
 /*
- * Bytes of device workspace that compactor_score / compactor_select / compactor_compress need
- * for this shape (the maximum over the three).  Returns 0 for an invalid shape.
+ * Bytes of device workspace that compactor_score and compactor_compress need for this shape.
+ * compactor_select and compactor_compact only use a small table at its start and accept any
+ * workspace of at least 12*(batch+1) bytes rounded up to 256.  The workspace must be 256-byte
+ * aligned; its contents need not be preserved between calls.  Returns 0 for an invalid shape.
  */
 size_t compactor_workspace_bytes(const compactor_shape* shape);
 
@@ -113,7 +115,7 @@ size_t compactor_workspace_bytes(const compactor_shape* shape);
  *   scores_out   device fp32 [layers][heads][total_tokens].
  * The small factorisation is a Cholesky factorisation of G = (K Phi)^T (K Phi) in fp64 - one of
  * the algebraically equal routes the paper allows (Section 3.2, Appendix C); Gram sums are fp32
- * per block of at most 8192 tokens and fp64 across blocks.
+ * per block of at most 2048 tokens and fp64 across blocks.
  */
 int compactor_score(const compactor_shape* shape, compactor_mat k_score, const float* phi,
                     const float* attn_scores, float lambda, float* scores_out,

@@ -1,0 +1,164 @@
+"""ctypes binding of the C-ABI library: argument marshalling only.
+
+Function names mirror the C entry points of `include/compactor.h`.  Device buffers are torch
+CUDA tensors (torch is used for device memory and streams, nothing else); every step of the
+path runs in the library's kernels.  Importing this module fails loudly if the library cannot
+be built or loaded - there is no fallback."""
+from __future__ import annotations
+
+import ctypes
+from ctypes import POINTER, Structure, byref, c_char_p, c_double, c_float, c_int32, c_int64, c_size_t, c_uint64, c_void_p
+from typing import Optional, Sequence
+
+import torch
+
+from . import build as _build
+
+
+class CompactorMat(Structure):
+    _fields_ = [("ptr", c_void_p), ("stride_layer", c_int64), ("stride_head", c_int64), ("stride_token", c_int64)]
+
+
+class CompactorShape(Structure):
+    _fields_ = [("layers", c_int32), ("heads", c_int32), ("d", c_int32), ("m", c_int32),
+                ("batch", c_int32), ("cu_seqlens", POINTER(c_int32))]
+
+
+class CompactorError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {error_string(code)} ({code})")
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.build()
+    lib = ctypes.CDLL(path)
+    lib.compactor_version.restype = ctypes.c_int
+    lib.compactor_error_string.restype = c_char_p
+    lib.compactor_error_string.argtypes = [ctypes.c_int]
+    lib.compactor_make_sketch.argtypes = [c_uint64, c_int32, c_int32, POINTER(c_float)]
+    lib.compactor_keep_count.restype = c_int64
+    lib.compactor_keep_count.argtypes = [c_int64, c_double]
+    lib.compactor_calibrated_ratio.argtypes = [c_double, c_double, c_double, c_double, POINTER(c_double)]
+    lib.compactor_workspace_bytes.restype = c_size_t
+    lib.compactor_workspace_bytes.argtypes = [POINTER(CompactorShape)]
+    lib.compactor_score.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_void_p, c_float, c_void_p,
+                                    c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_select.argtypes = [POINTER(CompactorShape), c_void_p, POINTER(c_int32), c_void_p, c_void_p,
+                                     c_void_p, c_size_t, c_void_p]
+    lib.compactor_compact.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_void_p, POINTER(c_int32),
+                                      c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_compress.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, CompactorMat, c_void_p,
+                                       c_void_p, c_float, POINTER(c_int32), c_void_p, c_void_p, c_void_p, c_void_p,
+                                       c_void_p, c_void_p, c_size_t, c_void_p]
+    return lib
+
+
+LIB = _load()
+LIB_PATH = _build.LIB
+
+EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_keep_count",
+           "compactor_calibrated_ratio", "compactor_workspace_bytes", "compactor_score", "compactor_select",
+           "compactor_compact", "compactor_compress"]
+
+
+def version() -> int:
+    return LIB.compactor_version()
+
+
+def error_string(code: int) -> str:
+    return LIB.compactor_error_string(code).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise CompactorError(code, where)
+
+
+class Shape:
+    """Owns the host arrays a compactor_shape points to."""
+
+    def __init__(self, layers: int, heads: int, d: int, m: int, seqlens: Sequence[int]):
+        self.seqlens = [int(n) for n in seqlens]
+        cu = [0]
+        for n in self.seqlens:
+            cu.append(cu[-1] + n)
+        self._cu = (c_int32 * len(cu))(*cu)
+        self.cu_seqlens = cu
+        self.c = CompactorShape(layers, heads, d, m, len(self.seqlens), self._cu)
+        self.layers, self.heads, self.d, self.m = layers, heads, d, m
+        self.total_tokens = cu[-1]
+
+    @property
+    def batch(self) -> int:
+        return len(self.seqlens)
+
+
+def mat(t: torch.Tensor) -> CompactorMat:
+    """A [layers, heads, tokens, d] bf16 CUDA tensor (any strides with a contiguous last axis)."""
+    assert t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 4 and t.stride(3) == 1
+    return CompactorMat(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream() -> c_void_p:
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _keep_array(keep_counts: Sequence[int]):
+    return (c_int32 * len(keep_counts))(*[int(k) for k in keep_counts])
+
+
+def make_sketch(seed: int, d: int, m: int) -> torch.Tensor:
+    out = torch.empty(d, m, dtype=torch.float32)
+    _check(LIB.compactor_make_sketch(seed, d, m, ctypes.cast(out.data_ptr(), POINTER(c_float))), "compactor_make_sketch")
+    return out
+
+
+def keep_count(n: int, r: float) -> int:
+    return int(LIB.compactor_keep_count(int(n), float(r)))
+
+
+def calibrated_ratio(nll: float, alpha: float, beta: float, tau: float) -> float:
+    r = c_double()
+    _check(LIB.compactor_calibrated_ratio(nll, alpha, beta, tau, byref(r)), "compactor_calibrated_ratio")
+    return r.value
+
+
+def workspace_bytes(shape: Shape) -> int:
+    return int(LIB.compactor_workspace_bytes(byref(shape.c)))
+
+
+def alloc_workspace(shape: Shape, device="cuda") -> torch.Tensor:
+    return torch.empty(max(256, workspace_bytes(shape)), dtype=torch.uint8, device=device)
+
+
+def score(shape: Shape, k_score: torch.Tensor, phi: torch.Tensor, scores_out: torch.Tensor, workspace: torch.Tensor,
+          attn: Optional[torch.Tensor] = None, lam: float = 0.3, status: Optional[torch.Tensor] = None) -> None:
+    _check(LIB.compactor_score(byref(shape.c), mat(k_score), _ptr(phi), _ptr(attn), lam, _ptr(scores_out),
+                               _ptr(status), _ptr(workspace), workspace.numel(), _stream()), "compactor_score")
+
+
+def select(shape: Shape, scores: torch.Tensor, keep_counts: Sequence[int], idx_out: torch.Tensor,
+           workspace: torch.Tensor, status: Optional[torch.Tensor] = None) -> None:
+    _check(LIB.compactor_select(byref(shape.c), _ptr(scores), _keep_array(keep_counts), _ptr(idx_out), _ptr(status),
+                                _ptr(workspace), workspace.numel(), _stream()), "compactor_select")
+
+
+def compact(shape: Shape, k_cache: torch.Tensor, v_cache: torch.Tensor, idx: torch.Tensor, keep_counts: Sequence[int],
+            k_out: torch.Tensor, v_out: torch.Tensor, workspace: torch.Tensor) -> None:
+    _check(LIB.compactor_compact(byref(shape.c), mat(k_cache), mat(v_cache), _ptr(idx), _keep_array(keep_counts),
+                                 _ptr(k_out), _ptr(v_out), _ptr(workspace), workspace.numel(), _stream()),
+           "compactor_compact")
+
+
+def compress(shape: Shape, k_score: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, phi: torch.Tensor,
+             keep_counts: Sequence[int], idx_out: torch.Tensor, k_out: torch.Tensor, v_out: torch.Tensor,
+             workspace: torch.Tensor, attn: Optional[torch.Tensor] = None, lam: float = 0.3,
+             scores_out: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None) -> None:
+    _check(LIB.compactor_compress(byref(shape.c), mat(k_score), mat(k_cache), mat(v_cache), _ptr(phi), _ptr(attn), lam,
+                                  _keep_array(keep_counts), _ptr(scores_out), _ptr(idx_out), _ptr(k_out), _ptr(v_out),
+                                  _ptr(status), _ptr(workspace), workspace.numel(), _stream()), "compactor_compress")

@@ -1,0 +1,272 @@
+// Host entry points of the C ABI declared in compactor.h: argument checking, workspace layout
+// and kernel sequencing.  No device memory is allocated here.
+#include <math.h>
+#include <string.h>
+
+#include <vector>
+
+#include "common.cuh"
+
+using namespace compactor;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kSmCount = 148;   // B200; only used to pick the Gram block length
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+struct HostPlan {
+    Plan plan;
+    std::vector<int> tables;       // cu_seqlens | cu_keep | cu_chunks, each batch+1
+    size_t off_tables, off_w, off_partials, off_scores, total_bytes;
+    int units;
+};
+
+bool shape_ok(const compactor_shape* s, int* err) {
+    if (s == nullptr || s->cu_seqlens == nullptr) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    if (s->layers < 1 || s->heads < 1 || s->batch < 1) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    if ((long long)s->layers * s->heads > 65535) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    if (s->d != kD || s->m < 1 || s->m > kMaxM) { *err = COMPACTOR_E_UNSUPPORTED; return false; }
+    if (s->cu_seqlens[0] != 0) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    for (int b = 0; b < s->batch; ++b)
+        if (s->cu_seqlens[b + 1] < s->cu_seqlens[b]) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    if ((long long)s->layers * s->heads * s->batch > 0x7fffffffLL) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    return true;
+}
+
+// Fills everything that depends on the shape alone (keep counts are added by the caller).
+bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
+    if (!shape_ok(s, err)) return false;
+    Plan& p = hp->plan;
+    memset(&p, 0, sizeof(p));
+    p.layers = s->layers; p.heads = s->heads; p.batch = s->batch;
+    p.m = s->m; p.mp = (s->m + 15) / 16 * 16;
+    p.total_tokens = s->cu_seqlens[s->batch];
+    hp->units = s->layers * s->heads * s->batch;
+
+    // Gram block length: the longest (<= kMaxChunk) that still yields about eight CTAs per SM.
+    int chunk = kMaxChunk;
+    auto count_chunks = [&](int c) {
+        long long t = 0;
+        for (int b = 0; b < s->batch; ++b) {
+            long long n = s->cu_seqlens[b + 1] - s->cu_seqlens[b];
+            t += (n + c - 1) / c;
+        }
+        return t;
+    };
+    while (chunk > kMinChunk && count_chunks(chunk) * s->layers * s->heads < 8LL * kSmCount) chunk >>= 1;
+    p.chunk = chunk;
+    long long tc = count_chunks(chunk);
+    if (tc > 0x7fffffffLL) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    p.total_chunks = (int)tc;
+
+    const int nb1 = s->batch + 1;
+    hp->tables.assign((size_t)3 * nb1, 0);
+    int* cs = hp->tables.data();
+    int* cc = cs + 2 * nb1;
+    for (int b = 0; b <= s->batch; ++b) cs[b] = s->cu_seqlens[b];
+    for (int b = 0; b < s->batch; ++b) cc[b + 1] = cc[b] + (cs[b + 1] - cs[b] + chunk - 1) / chunk;
+
+    size_t off = 0;
+    hp->off_tables = off;   off += align_up(sizeof(int) * 3 * nb1);
+    hp->off_w = off;        off += align_up(sizeof(__nv_bfloat16) * w_elems_per_unit(p.mp) * hp->units);
+    hp->off_partials = off; off += align_up(sizeof(float) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
+    hp->off_scores = off;   off += align_up(sizeof(float) * (size_t)p.total_tokens * s->layers * s->heads);
+    hp->total_bytes = off;
+    return true;
+}
+
+bool set_keep(const compactor_shape* s, const int32_t* keep, HostPlan* hp) {
+    if (keep == nullptr) return false;
+    const int nb1 = s->batch + 1;
+    int* ck = hp->tables.data() + nb1;
+    long long tot = 0;
+    for (int b = 0; b < s->batch; ++b) {
+        int n = s->cu_seqlens[b + 1] - s->cu_seqlens[b];
+        if (keep[b] < 0 || keep[b] > n) return false;
+        tot += keep[b];
+        ck[b + 1] = (int)tot;
+    }
+    hp->plan.total_keep = (int)tot;
+    return true;
+}
+
+bool mat_ok(const compactor_mat& m) {
+    if (m.ptr == nullptr || ((uintptr_t)m.ptr & 15) != 0) return false;
+    if (m.stride_token < kD || (m.stride_token & 7) || (m.stride_layer & 7) || (m.stride_head & 7)) return false;
+    if (m.stride_layer < 0 || m.stride_head < 0) return false;
+    return true;
+}
+
+Mat to_mat(const compactor_mat& m) {
+    Mat r;
+    r.ptr = static_cast<const __nv_bfloat16*>(m.ptr);
+    r.stride_layer = m.stride_layer; r.stride_head = m.stride_head; r.stride_token = m.stride_token;
+    return r;
+}
+
+// Copies the tables to the head of the workspace and points the plan at them.
+cudaError_t upload_tables(HostPlan* hp, void* ws, cudaStream_t stream) {
+    const int nb1 = hp->plan.batch + 1;
+    int* dev = reinterpret_cast<int*>(static_cast<char*>(ws) + hp->off_tables);
+    // The source is pageable host memory: the runtime stages it before this call returns.
+    cudaError_t e = cudaMemcpyAsync(dev, hp->tables.data(), sizeof(int) * 3 * nb1, cudaMemcpyHostToDevice, stream);
+    hp->plan.cu_seqlens = dev;
+    hp->plan.cu_keep = dev + nb1;
+    hp->plan.cu_chunks = dev + 2 * nb1;
+    return e;
+}
+
+#define CK(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) return COMPACTOR_E_CUDA; } while (0)
+
+int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn, float lambda,
+                float* scores, int32_t* status, char* ws, cudaStream_t stream) {
+    __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(ws + hp.off_w);
+    float* partials = reinterpret_cast<float*>(ws + hp.off_partials);
+    CK(launch_gram(hp.plan, k, partials, stream));
+    CK(launch_factor(hp.plan, k, partials, phi, w, status, stream));
+    CK(launch_score(hp.plan, k, w, scores, stream));
+    if (attn != nullptr) CK(launch_blend(hp.plan, attn, lambda, scores, stream));
+    return COMPACTOR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int compactor_version(void) { return 100; }
+
+const char* compactor_error_string(int code) {
+    switch (code) {
+        case COMPACTOR_OK: return "ok";
+        case COMPACTOR_E_INVALID_ARGUMENT: return "invalid argument";
+        case COMPACTOR_E_UNSUPPORTED: return "unsupported shape (d must be 128, 1 <= m <= 64)";
+        case COMPACTOR_E_WORKSPACE: return "workspace too small";
+        case COMPACTOR_E_CUDA: return "CUDA runtime error";
+        default: return "unknown status";
+    }
+}
+
+int compactor_make_sketch(uint64_t seed, int32_t d, int32_t m, float* phi_host) {
+    if (phi_host == nullptr || d < 1 || m < 1) return COMPACTOR_E_INVALID_ARGUMENT;
+    auto word = [seed](uint64_t i) {
+        uint64_t z = seed + (i + 1) * 0x9E3779B97F4A7C15ull;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+        return z ^ (z >> 31);
+    };
+    const long long count = (long long)d * m;
+    const double root_m = sqrt((double)m);
+    const double two_pi = 6.283185307179586476925286766559;
+    for (long long pidx = 0; 2 * pidx < count; ++pidx) {
+        double u1 = (double)((word(2 * pidx) >> 11) + 1) * 0x1.0p-53;
+        double u2 = (double)(word(2 * pidx + 1) >> 11) * 0x1.0p-53;
+        double rad = sqrt(-2.0 * log(u1));
+        phi_host[2 * pidx] = (float)(rad * cos(two_pi * u2) / root_m);
+        if (2 * pidx + 1 < count) phi_host[2 * pidx + 1] = (float)(rad * sin(two_pi * u2) / root_m);
+    }
+    return COMPACTOR_OK;
+}
+
+int64_t compactor_keep_count(int64_t n, double r) {
+    if (n <= 0) return 0;
+    double c = ceil(r * (double)n);
+    if (!(c >= 1.0)) return 1;          // also catches NaN
+    if (c >= (double)n) return n;
+    return (int64_t)c;
+}
+
+int compactor_calibrated_ratio(double nll, double alpha, double beta, double tau, double* r_out) {
+    if (r_out == nullptr || !(tau > 0.0) || !(tau <= 1.0)) return COMPACTOR_E_INVALID_ARGUMENT;
+    const double b = alpha * nll + beta;
+    if (!isfinite(b)) return COMPACTOR_E_INVALID_ARGUMENT;
+    *r_out = (b == 0.0) ? tau : log1p(tau * expm1(b)) / b;
+    return COMPACTOR_OK;
+}
+
+size_t compactor_workspace_bytes(const compactor_shape* shape) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return 0;
+    return hp.total_bytes;
+}
+
+int compactor_score(const compactor_shape* shape, compactor_mat k_score, const float* phi,
+                    const float* attn_scores, float lambda, float* scores_out,
+                    int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (!mat_ok(k_score) || phi == nullptr || scores_out == nullptr || workspace == nullptr)
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (((uintptr_t)workspace & 255) != 0) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (workspace_bytes < hp.total_bytes) return COMPACTOR_E_WORKSPACE;
+    if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CK(upload_tables(&hp, workspace, st));
+    return run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores_out, status,
+                       static_cast<char*>(workspace), st);
+}
+
+int compactor_select(const compactor_shape* shape, const float* scores, const int32_t* keep_counts,
+                     int32_t* idx_out, int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
+    (void)status;
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (scores == nullptr || idx_out == nullptr || workspace == nullptr || !set_keep(shape, keep_counts, &hp))
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (((uintptr_t)workspace & 255) != 0) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (workspace_bytes < hp.off_w) return COMPACTOR_E_WORKSPACE;      // only the tables are used
+    if (hp.plan.total_keep == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CK(upload_tables(&hp, workspace, st));
+    CK(launch_select(hp.plan, scores, idx_out, st));
+    return COMPACTOR_OK;
+}
+
+int compactor_compact(const compactor_shape* shape, compactor_mat k_cache, compactor_mat v_cache,
+                      const int32_t* idx, const int32_t* keep_counts, void* k_out, void* v_out,
+                      void* workspace, size_t workspace_bytes, void* stream) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (!mat_ok(k_cache) || !mat_ok(v_cache) || idx == nullptr || k_out == nullptr || v_out == nullptr ||
+        workspace == nullptr || !set_keep(shape, keep_counts, &hp))
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if ((((uintptr_t)k_out | (uintptr_t)v_out) & 15) != 0 || ((uintptr_t)workspace & 255) != 0)
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (workspace_bytes < hp.off_w) return COMPACTOR_E_WORKSPACE;      // only the tables are used
+    if (hp.plan.total_keep == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CK(upload_tables(&hp, workspace, st));
+    CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx,
+                      static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
+    return COMPACTOR_OK;
+}
+
+int compactor_compress(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
+                       compactor_mat v_cache, const float* phi, const float* attn_scores,
+                       float lambda, const int32_t* keep_counts,
+                       float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
+                       int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (!mat_ok(k_score) || !mat_ok(k_cache) || !mat_ok(v_cache) || phi == nullptr || idx_out == nullptr ||
+        k_out == nullptr || v_out == nullptr || workspace == nullptr || !set_keep(shape, keep_counts, &hp))
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if ((((uintptr_t)k_out | (uintptr_t)v_out) & 15) != 0 || ((uintptr_t)workspace & 255) != 0)
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (workspace_bytes < hp.total_bytes) return COMPACTOR_E_WORKSPACE;
+    if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    float* scores = scores_out != nullptr ? scores_out : reinterpret_cast<float*>(ws + hp.off_scores);
+    CK(upload_tables(&hp, workspace, st));
+    int rc = run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores, status, ws, st);
+    if (rc != COMPACTOR_OK) return rc;
+    if (hp.plan.total_keep == 0) return COMPACTOR_OK;
+    CK(launch_select(hp.plan, scores, idx_out, st));
+    CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out,
+                      static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
+    return COMPACTOR_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,61 @@
+// Internal declarations shared by the kernels and the host entry points of the library.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "compactor.h"
+
+namespace compactor {
+
+constexpr int kD = 128;            // head dimension the kernels are written for
+constexpr int kMaxM = 64;          // largest sketch dimension
+constexpr int kMaxChunk = 2048;    // most tokens whose Gram matrix is summed in fp32 before the fp64 reduction
+constexpr int kMinChunk = 256;
+constexpr int kGramElems = kD * kD;
+
+// Device-side view of one call: shapes plus the three prefix-sum tables that live at the start
+// of the workspace.  Passed to kernels by value.
+struct Plan {
+    int layers, heads, batch;
+    int m;                 // sketch dimension
+    int mp;                // m rounded up to a multiple of 16 (padded columns of W are zero)
+    int chunk;             // tokens per Gram partial (multiple of 128)
+    int total_chunks;      // Gram partials per (layer, head): sum_b ceil(n_b / chunk)
+    int total_tokens;      // per (layer, head)
+    int total_keep;        // per (layer, head)
+    const int* cu_seqlens; // device [batch+1]
+    const int* cu_keep;    // device [batch+1]
+    const int* cu_chunks;  // device [batch+1]
+};
+
+struct Mat {               // compactor_mat with a typed pointer
+    const __nv_bfloat16* ptr;
+    long long stride_layer, stride_head, stride_token;
+};
+
+// Largest b with table[b] <= x, for a non-decreasing table of nb+1 entries with table[0] = 0.
+__device__ __forceinline__ int find_segment(const int* __restrict__ table, int nb, int x) {
+    int lo = 0, hi = nb;          // invariant: table[lo] <= x < table[hi] (table[nb] > x by construction)
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (table[mid] <= x) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Kernel launchers (each defined next to its kernel).  All enqueue on `stream` and return the
+// launch status.
+cudaError_t launch_gram(const Plan& p, const Mat& k, float* partials, cudaStream_t stream);
+cudaError_t launch_factor(const Plan& p, const Mat& k, const float* partials, const float* phi, __nv_bfloat16* w,
+                          int* status, cudaStream_t stream);
+cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, cudaStream_t stream);
+cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* scores, cudaStream_t stream);
+cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStream_t stream);
+cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int* idx,
+                           __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream);
+
+// Bytes of W (two bf16 terms, [term][mp][128]) per unit.
+__host__ __device__ inline size_t w_elems_per_unit(int mp) { return (size_t)2 * mp * kD; }
+
+}  // namespace compactor

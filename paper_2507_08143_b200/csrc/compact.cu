@@ -1,0 +1,81 @@
+// Compaction (Section 3, Preliminaries: only the selected fraction of the tokens is retained):
+// gathers the kept rows of K and V of every unit into dense [total_keep][128] blocks.  Each
+// 256-byte row is moved by 16 threads as 128-bit pieces; bit-exact.
+#include "common.cuh"
+
+namespace compactor {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRowsPerIter = kThreads / 16;     // 16 rows in flight per instruction
+constexpr int kUnroll = 4;
+constexpr int kRowsPerCta = kRowsPerIter * kUnroll * 2;   // 128 output rows per CTA
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};\n" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads)
+compact_kernel(Plan p, Mat k, Mat v, const int* __restrict__ idx,
+               __nv_bfloat16* __restrict__ k_out, __nv_bfloat16* __restrict__ v_out) {
+    const int lh = blockIdx.y;
+    const int layer = lh / p.heads, head = lh % p.heads;
+    const int piece = threadIdx.x & 15, sub = threadIdx.x >> 4;
+    const int* idx_lh = idx + (size_t)lh * p.total_keep;
+    const __nv_bfloat16* kb = k.ptr + layer * k.stride_layer + head * k.stride_head;
+    const __nv_bfloat16* vb = v.ptr + layer * v.stride_layer + head * v.stride_head;
+    uint4* ko = reinterpret_cast<uint4*>(k_out + (size_t)lh * p.total_keep * kD);
+    uint4* vo = reinterpret_cast<uint4*>(v_out + (size_t)lh * p.total_keep * kD);
+
+    const int row0 = blockIdx.x * kRowsPerCta;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        uint4 kv[kUnroll], vv[kUnroll];
+        int rows[kUnroll];
+        bool ok[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            int row = row0 + (half * kUnroll + u) * kRowsPerIter + sub;
+            rows[u] = row;
+            ok[u] = false;
+            if (row < p.total_keep) {
+                int b = find_segment(p.cu_keep, p.batch, row);
+                int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+                int local = idx_lh[row];
+                if (local >= 0 && local < n) {
+                    long long tok = (long long)p.cu_seqlens[b] + local;
+                    kv[u] = ld_stream(reinterpret_cast<const uint4*>(kb + tok * k.stride_token) + piece);
+                    vv[u] = ld_stream(reinterpret_cast<const uint4*>(vb + tok * v.stride_token) + piece);
+                    ok[u] = true;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            if (ok[u]) {
+                st_stream(ko + (size_t)rows[u] * 16 + piece, kv[u]);
+                st_stream(vo + (size_t)rows[u] * 16 + piece, vv[u]);
+            }
+        }
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int* idx,
+                           __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream) {
+    if (p.total_keep == 0 || p.layers * p.heads == 0) return cudaSuccess;
+    dim3 grid((p.total_keep + kRowsPerCta - 1) / kRowsPerCta, p.layers * p.heads);
+    compact_kernel<<<grid, kThreads, 0, stream>>>(p, k, v, idx, k_out, v_out);
+    return cudaGetLastError();
+}
+
+}  // namespace compactor

@@ -1,0 +1,214 @@
+"""GPU parity tests: the CUDA library, called through its C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2507_08143_b200 import inputs
+from oracle import compactor_oracle as orc
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2507_08143_b200 import binding
+    return binding
+
+
+def _keep(B, w):
+    return [B.keep_count(n, r) for n, r in zip(w.seqlens, w.ratios)]
+
+
+def _run_workload(B, w, mode="paper", attn=False, units=None, device="cuda"):
+    kp, kr, v = inputs.make_tensors(w, device=device, want_pre=(mode == "paper"))
+    kp, kr, v = (None if kp is None else kp.cuda()), kr.cuda(), v.cuda()
+    k_score = kp if mode == "paper" else kr
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    phi = inputs.make_sketch_matrix(w.d, w.m, w.seed)
+    keep = _keep(B, w)
+    a = inputs.make_attention_scores(w, seed=w.seed, device="cuda") if attn else None
+    outs = H.run_compress(B, shape, k_score, kr, v, phi, keep, attn=a)
+    worst, band = H.compare_all_units(shape, keep, outs, k_score, kr, v, phi, attn=a, units=units, what=w.name)
+    return worst, band, outs
+
+
+@pytest.mark.parametrize("mode", ["paper", "aliased"])
+def test_c0_tiny(B, mode):
+    w = inputs.workload("c0")
+    worst, band, outs = _run_workload(B, w, mode=mode, device="cpu")
+    assert int(outs[4].max()) == 0
+    print(f"c0 {mode}: max rel score err {worst:.2e}, boundary band {band}")
+
+
+def test_c0_with_attention_blend(B):
+    w = inputs.workload("c0")
+    worst, band, _ = _run_workload(B, w, attn=True, device="cpu")
+    print(f"c0 blend: err {worst:.2e}")
+
+
+def test_ragged_small_sequences(B):
+    # lengths around the tile, chunk and sketch sizes, including an empty sequence
+    w = inputs.Workload("ragged-small", 2, 2, 128, [1000, 129, 0, 128, 127, 2500, 49, 300],
+                        [0.3, 0.5, 0.5, 0.2, 0.5, 0.3, 0.5, 1.0], p=0.7, seed=11)
+    worst, band, outs = _run_workload(B, w, device="cpu")
+    print(f"ragged-small: err {worst:.2e}")
+
+
+@pytest.mark.parametrize("m", [8, 16, 20, 32, 64])
+def test_other_sketch_dimensions(B, m):
+    w = inputs.Workload(f"m{m}", 1, 2, 128, [700, 1300], [0.25, 0.4], p=0.7, seed=20 + m, m=m)
+    _run_workload(B, w, mode="aliased", device="cpu")
+
+
+def test_token_major_layout(B):
+    # [layers, tokens, heads, d] storage (the layout of a serving engine's cache), passed by strides
+    w = inputs.Workload("token-major", 2, 3, 128, [900, 411], [0.3, 0.6], p=0.7, seed=31)
+    kp, kr, v = inputs.make_tensors(w, device="cpu")
+    def tm(t):
+        return t.cuda().permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    kp, kr, v = tm(kp), tm(kr), tm(v)
+    assert kp.stride(2) == 3 * 128
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    phi = inputs.make_sketch_matrix(w.d, w.m, 5)
+    keep = _keep(B, w)
+    outs = H.run_compress(B, shape, kp, kr, v, phi, keep)
+    H.compare_all_units(shape, keep, outs, kp, kr, v, phi, what="token-major")
+
+
+def test_staged_calls_match_fused(B):
+    w = inputs.Workload("staged", 2, 2, 128, [1500, 640], [0.3, 0.5], p=1.0, seed=41)
+    kp, kr, v = [t.cuda() for t in inputs.make_tensors(w, device="cpu")]
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    phi = inputs.make_sketch_matrix(w.d, w.m, 6)
+    keep = _keep(B, w)
+    scores_f, idx_f, ko_f, vo_f, _ = H.run_compress(B, shape, kp, kr, v, phi, keep)
+    ws = B.alloc_workspace(shape)
+    scores = torch.empty_like(scores_f); idx = torch.empty_like(idx_f)
+    ko = torch.empty_like(ko_f); vo = torch.empty_like(vo_f)
+    B.score(shape, kp, phi.cuda(), scores, ws)
+    B.select(shape, scores, keep, idx, ws)
+    B.compact(shape, kr, v, idx, keep, ko, vo, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(scores, scores_f) and torch.equal(idx, idx_f)
+    assert torch.equal(ko.view(torch.int16), ko_f.view(torch.int16))
+    assert torch.equal(vo.view(torch.int16), vo_f.view(torch.int16))
+    # fused call without a scores output gives the same indices
+    _, idx_n, _, _, _ = H.run_compress(B, shape, kp, kr, v, phi, keep, want_scores=False)
+    assert torch.equal(idx_n, idx_f)
+
+
+def test_select_exact_with_ties_and_edges(B):
+    rng = np.random.default_rng(7)
+    seqlens = [1, 2, 5000, 4096, 4097, 33, 10000]
+    keep = [1, 1, 1234, 4096, 1, 0, 9999]
+    L, Hh = 2, 2
+    shape = B.Shape(L, Hh, 128, 48, seqlens)
+    T = shape.total_tokens
+    s = rng.standard_normal((L, Hh, T)).astype(np.float32)
+    s[0, 0] = np.round(s[0, 0], 1)                      # heavy ties
+    s[0, 1] = 0.25                                       # all equal
+    s[1, 0] = np.round(np.abs(s[1, 0]), 2) * np.sign(rng.standard_normal(T)).astype(np.float32)
+    s[1, 1, ::7] = -0.0
+    s[1, 1, 3::7] = 0.0
+    s[1, 1, 5::11] = np.inf
+    s[1, 1, 6::13] = -np.inf
+    sc = torch.from_numpy(s).cuda()
+    idx = torch.full((L, Hh, sum(keep)), -1, dtype=torch.int32, device="cuda")
+    ws = B.alloc_workspace(shape)
+    B.select(shape, sc, keep, idx, ws)
+    torch.cuda.synchronize()
+    idx = idx.cpu().numpy()
+    cu, ck = shape.cu_seqlens, np.concatenate([[0], np.cumsum(keep)])
+    for l in range(L):
+        for h in range(Hh):
+            for b in range(len(seqlens)):
+                got = idx[l, h, ck[b]:ck[b + 1]]
+                seg = s[l, h, cu[b]:cu[b + 1]].astype(np.float64)
+                np.testing.assert_array_equal(got, orc.top_k_indices(seg, keep[b]), err_msg=f"{l},{h},{b}")
+
+
+def test_compact_bit_exact_and_skips_bad_indices(B):
+    w = inputs.Workload("compact", 2, 2, 128, [700, 300], [0.5, 0.5], seed=51)
+    _, kr, v = inputs.make_tensors(w, device="cpu", want_pre=False)
+    kr, v = kr.cuda(), v.cuda()
+    shape = B.Shape(2, 2, 128, 48, w.seqlens)
+    keep = [350, 150]
+    g = torch.Generator().manual_seed(3)
+    idx = torch.stack([torch.cat([torch.randperm(700, generator=g)[:350], torch.randperm(300, generator=g)[:150]])
+                       for _ in range(4)]).reshape(2, 2, 500).to(torch.int32)
+    idx[0, 0, 5] = -3; idx[1, 1, 400] = 300            # out of range: rows must stay untouched
+    ko = torch.full((2, 2, 500, 128), 7.0, dtype=torch.bfloat16, device="cuda"); vo = ko.clone()
+    ws = B.alloc_workspace(shape)
+    B.compact(shape, kr, v, idx.cuda(), keep, ko, vo, ws)
+    torch.cuda.synchronize()
+    kb, vb, kob, vob = H.bits(kr), H.bits(v), H.bits(ko), H.bits(vo)
+    seven = H.bits(torch.tensor([7.0], dtype=torch.bfloat16))[0]
+    for l in range(2):
+        for h in range(2):
+            for j in range(500):
+                b = 0 if j < 350 else 1
+                i = int(idx[l, h, j]); n = w.seqlens[b]
+                if 0 <= i < n:
+                    t = (0 if b == 0 else 700) + i
+                    assert np.array_equal(kob[l, h, j], kb[l, h, t]) and np.array_equal(vob[l, h, j], vb[l, h, t])
+                else:
+                    assert np.all(kob[l, h, j] == seven) and np.all(vob[l, h, j] == seven)
+
+
+def test_degenerate_keys(B):
+    # all-zero keys: every score 0, first kk indices kept; one repeated row: equal scores 1/n
+    d, n = 128, 300
+    K = torch.zeros(1, 2, n, d, dtype=torch.bfloat16)
+    row = torch.randn(d, generator=torch.Generator().manual_seed(1))
+    K[0, 1] = row.to(torch.bfloat16)
+    V = torch.randn(1, 2, n, d, generator=torch.Generator().manual_seed(2)).to(torch.bfloat16)
+    K, V = K.cuda(), V.cuda()
+    shape = B.Shape(1, 2, d, 48, [n])
+    phi = inputs.make_sketch_matrix(d, 48, 9)
+    scores, idx, ko, vo, status = H.run_compress(B, shape, K, K, V, phi, [100])
+    assert torch.all(scores[0, 0] == 0)
+    assert idx[0, 0].tolist() == list(range(100))
+    np.testing.assert_allclose(scores[0, 1].cpu().numpy(), 1.0 / n, rtol=1e-3)
+    assert (int(status[0]) & 2) and (int(status[1]) & 2)          # both flagged rank deficient
+    assert not (int(status[0]) & 1)
+
+
+def test_fewer_rows_than_sketch_columns(B):
+    # n <= m with full row rank: K^ K^+ = I, every score is 1
+    w = inputs.Workload("short", 1, 2, 128, [5, 40, 48], [1.0, 0.5, 0.25], p=0.7, seed=61)
+    kp, kr, v = [t.cuda() for t in inputs.make_tensors(w, device="cpu")]
+    shape = B.Shape(1, 2, 128, 48, w.seqlens)
+    phi = inputs.make_sketch_matrix(128, 48, 2)
+    keep = _keep(B, w)
+    scores, idx, ko, vo, status = H.run_compress(B, shape, kr, kr, v, phi, keep)
+    s = scores.cpu().numpy()
+    np.testing.assert_allclose(s[:, :, :45], 1.0, rtol=2e-3)
+
+
+def test_nonfinite_input_sets_status_and_returns(B):
+    w = inputs.Workload("nan", 1, 2, 128, [600], [0.5], seed=71)
+    _, kr, v = inputs.make_tensors(w, device="cpu", want_pre=False)
+    kr[0, 1, 17, 3] = float("nan")
+    kr, v = kr.cuda(), v.cuda()
+    shape = B.Shape(1, 2, 128, 48, w.seqlens)
+    scores, idx, ko, vo, status = H.run_compress(B, shape, kr, kr, v, inputs.make_sketch_matrix(128, 48, 1), [300])
+    assert int(status[0]) == 0 and (int(status[1]) & 1)
+    i = idx[0, 1].cpu().numpy()
+    assert len(np.unique(i)) == 300 and i.min() >= 0 and i.max() < 600
+
+
+@pytest.mark.parametrize("name,layers,heads", [("c1", 2, None), ("c2", 1, None), ("c4", 1, 2)])
+def test_benchmark_shapes_reduced_layers(B, name, layers, heads):
+    w = inputs.workload(name, layers=layers)
+    if heads is not None:
+        w.heads = heads
+    worst, band, _ = _run_workload(B, w, mode="paper", device="cuda")
+    print(f"{w.name}: layers={layers} max rel score err {worst:.2e}, boundary band {band}")
+
+
+def test_c3_long_context_units(B):
+    w = inputs.workload("c3", layers=1)
+    w.heads = 2
+    worst, band, _ = _run_workload(B, w, mode="paper", device="cuda")
+    print(f"c3 (n=131072, 2 units): max rel score err {worst:.2e}, boundary band {band}")

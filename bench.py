@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Benchmark of the compression pass (score + select + compact) on synthetic long-context keys.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload c3|c1|c2|c4|c0] [--mode aliased|paper] [--layers L]
+
+One step = one fused compactor_compress call over the whole workload (every layer, KV head and
+sequence).  Prints ONE JSON line.  For N > 1 (launched by torch.distributed.run, one rank per
+GPU) every rank compresses its own copy of the workload (different seed): units are independent,
+so there is no data-path collective and scaling is weak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compressed tokens/s per B200 (score+select+compact)"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of the dominant kernels per head-token, from ncu captures of a smaller case of
+# the same kernels (see profiles/); bytes read + written per token of one (layer, head).
+NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--mode", default="aliased", choices=["aliased", "paper"],
+                    help="aliased: score and gather the rotated keys; paper: score pre-rotation keys")
+    ap.add_argument("--layers", type=int, default=None, help="override the layer count (debugging)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-units", type=int, default=16, help="units in the CPU-baseline sample")
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def algorithmic_bytes(w, keep, mode):
+    """Bytes the method must move per step: scored K read once, kept V rows read, kept K rows
+    read (a re-touch in aliased mode, so not counted there), kept K/V rows written."""
+    row = w.d * 2
+    per_lh = 0
+    for n, kk in zip(w.seqlens, keep):
+        per_lh += n * row + kk * row * (3 if mode == "aliased" else 4)
+    return per_lh * w.layers * w.heads
+
+
+def stage_bytes(w, keep, mode, chunk_tokens=2048):
+    """Minimal bytes of each kernel run on its own (per step)."""
+    row = w.d * 2
+    lh = w.layers * w.heads
+    tok = sum(w.seqlens); kept = sum(keep)
+    n_part = sum((n + chunk_tokens - 1) // chunk_tokens for n in w.seqlens)
+    return {
+        "gram": lh * (tok * row + n_part * 65536),
+        "factor": lh * n_part * 65536,
+        "score": lh * tok * (row + 4),
+        "blend": 0,
+        "select": lh * (tok * 4 + kept * 4),
+        "compact": lh * kept * (4 * row + 4),
+    }
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: a bounded sample of the workload's units."""
+    import numpy as np
+    import torch
+    from paper_2507_08143_b200 import inputs
+    from oracle import compactor_oracle as orc
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = inputs.workload(args.workload, layers=args.layers)
+    phi = inputs.make_sketch_matrix(w.d, w.m, w.seed).numpy()
+    keep = [orc.keep_count(n, r) for n, r in zip(w.seqlens, w.ratios)]
+    sample = max(1, min(args.cpu_units, 4))
+    units = [(0, h % w.heads, b % w.batch) for h, b in zip(range(sample), range(sample))]
+    data = []
+    for (l, h, b) in units:
+        kp, kr, v = inputs.make_unit(w, b, l, h)
+        ks = kp if args.mode == "paper" else kr
+        data.append((ks.view(torch.int16).numpy(), kr.view(torch.int16).numpy(), v.view(torch.int16).numpy(), keep[b],
+                     w.seqlens[b]))
+
+    def step():
+        for ks, kr, v, kk, n in data:
+            orc.compress_unit(ks, kr, v, phi, kk)
+
+    for _ in range(min(args.warmup, 1)):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    head_tokens = sum(d[4] for d in data)
+    # a token counts once for all layers x heads: scale the sample to the whole workload
+    value = (head_tokens / dt) / (w.layers * w.heads)
+    cores = torch.get_num_threads()
+    desc = f"{len(data)} units of {w.name} per step ({head_tokens} head-tokens), scaled to {w.layers}x{w.heads} units per token"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "mode": args.mode, "layers": w.layers, "kv_heads": w.heads, "d": w.d,
+                   "m": w.m, "seqlens": w.seqlens if w.batch <= 4 else f"{w.batch} sequences"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cpu_baseline(args, w, keep, phi):
+    import torch
+    from paper_2507_08143_b200 import inputs
+    from oracle import compactor_oracle as orc
+    sample = max(1, args.cpu_units)
+    data = []
+    for i in range(sample):
+        b, h = i % w.batch, i % w.heads
+        kp, kr, v = inputs.make_unit(w, b, 0, h)
+        ks = kp if args.mode == "paper" else kr
+        data.append((ks.view(torch.int16).numpy(), kr.view(torch.int16).numpy(), v.view(torch.int16).numpy(), keep[b],
+                     w.seqlens[b]))
+    phi_np = phi.numpy()
+    t0 = time.perf_counter()
+    for ks, kr, v, kk, n in data:
+        orc.compress_unit(ks, kr, v, phi_np, kk)
+    dt = time.perf_counter() - t0
+    head_tokens = sum(d[4] for d in data)
+    value = (head_tokens / dt) / (w.layers * w.heads)
+    return {"value": value, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"{sample} units of {w.name} ({head_tokens} head-tokens, {dt:.1f} s), scaled to "
+                      f"{w.layers}x{w.heads} units per token"}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2507_08143_b200 import binding as B, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device"
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    w = inputs.workload(args.workload, layers=args.layers)
+    w.seed = w.seed + 1000 * rank
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    keep = [B.keep_count(n, r) for n, r in zip(w.seqlens, w.ratios)]
+    total_keep = sum(keep)
+    phi = inputs.make_sketch_matrix(w.d, w.m, w.seed)
+    phi_d = phi.cuda()
+
+    kp, kr, v = inputs.make_tensors(w, device="cuda", want_pre=(args.mode == "paper"))
+    k_score = kp if args.mode == "paper" else kr
+    L, Hh = w.layers, w.heads
+    idx = torch.empty(L, Hh, total_keep, dtype=torch.int32, device="cuda")
+    k_out = torch.empty(L, Hh, total_keep, w.d, dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+    status = torch.zeros(L * Hh * w.batch, dtype=torch.int32, device="cuda")
+    ws = B.alloc_workspace(shape)
+
+    events = [torch.cuda.Event(enable_timing=True) for _ in range(B.N_STAGE_EVENTS * args.steps)]
+    for e in events:
+        e.record()
+    torch.cuda.synchronize()
+
+    def step(ev=None):
+        if ev is None:
+            B.compress(shape, k_score, kr, v, phi_d, keep, idx, k_out, v_out, ws, status=status)
+        else:
+            B.compress_profiled(shape, k_score, kr, v, phi_d, keep, idx, k_out, v_out, ws, ev, status=status)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_beg.record()
+    for i in range(args.steps):
+        step(events[i * B.N_STAGE_EVENTS:(i + 1) * B.N_STAGE_EVENTS])
+    t_end.record()
+    barrier()
+    elapsed_ms = t_beg.elapsed_time(t_end)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    tokens_per_step = w.total_tokens * world
+    value = tokens_per_step / (ms_per_step * 1e-3)
+    assert int(status.max().item()) == 0, "a unit reported a numerical status flag"
+
+    # per-kernel times from the stage markers of the timed region
+    stage_ms = {name: 0.0 for name in B.STAGE_NAMES}
+    for i in range(args.steps):
+        ev = events[i * B.N_STAGE_EVENTS:(i + 1) * B.N_STAGE_EVENTS]
+        for j, name in enumerate(B.STAGE_NAMES):
+            stage_ms[name] += ev[j].elapsed_time(ev[j + 1]) / args.steps
+    sb = stage_bytes(w, keep, args.mode)
+    dominant = max(stage_ms, key=stage_ms.get)
+    peak, peak_kind = measured_peak()
+    achieved = sb[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
+    traffic = NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN.get(dominant)
+    if traffic is not None:
+        traffic = traffic * L * Hh * w.total_tokens
+    b_alg = algorithmic_bytes(w, keep, args.mode)
+    path_gbs = b_alg / (ms_per_step * 1e-3) / 1e9
+
+    result = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 inputs, fp32 tensor-core accumulate, fp64 factorisation",
+        "data": "synthetic",
+        "config": {"workload": w.name, "mode": args.mode, "layers": L, "kv_heads": Hh, "d": w.d, "m": w.m,
+                   "seqlens": w.seqlens if w.batch <= 4 else f"{w.batch} sequences, {w.total_tokens} tokens",
+                   "keep": keep if w.batch <= 4 else total_keep, "units_per_gpu": w.units,
+                   "l2": "inputs (GBs per step) far exceed the 126 MB L2; no flush needed"},
+        "head_tokens_per_s": value * L * Hh,
+        "gpu_launches": 5 * args.steps,
+        "stage_ms": {k: round(t, 4) for k, t in stage_ms.items()},
+        "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                     "bytes_per_launch": sb[dominant]},
+        "path_roofline": {"algorithmic_bytes_per_step": b_alg, "achieved": path_gbs, "peak": peak, "unit": "GB/s",
+                          "frac": path_gbs / peak, "frac_of_8TBs": path_gbs / 8000.0},
+        "clocks": clocks,
+    }
+
+    if not args.no_e2e:
+        result["e2e"] = e2e(args, B, w, shape, keep, phi_d, k_score, kr, v, dist, world)
+    if rank == 0 and world == 1 and not args.no_cpu:
+        result["cpu_baseline"] = cpu_baseline(args, w, keep, phi)
+    if rank == 0:
+        print(json.dumps(result))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def e2e(args, B, w, shape, keep, phi_d, k_score, kr, v, dist, world):
+    """The same pass with HOST inputs and outputs: the workload is streamed in groups of layers
+    through pinned host buffers (host->device copy of the group's K and V, compress, device->host
+    copy of indices and compressed K/V), every step."""
+    import torch
+    group = min(8, w.layers)
+    n_groups = (w.layers + group - 1) // group
+    g_shape = B.Shape(group, w.heads, w.d, w.m, w.seqlens)
+    total_keep = sum(keep)
+    T = w.total_tokens
+    paper = args.mode == "paper"
+    # pinned host copies of one group of layers (the first), reused for every group of the step
+    hk = torch.empty(group, w.heads, T, w.d, dtype=torch.bfloat16).pin_memory()
+    hv = torch.empty_like(hk).pin_memory()
+    hk.copy_(kr[:group]); hv.copy_(v[:group])
+    hs = None
+    if paper:
+        hs = torch.empty_like(hk).pin_memory(); hs.copy_(k_score[:group])
+    h_idx = torch.empty(group, w.heads, total_keep, dtype=torch.int32).pin_memory()
+    h_ko = torch.empty(group, w.heads, total_keep, w.d, dtype=torch.bfloat16).pin_memory()
+    h_vo = torch.empty_like(h_ko).pin_memory()
+    dk = [torch.empty_like(hk, device="cuda") for _ in range(2)]
+    dv = [torch.empty_like(hk, device="cuda") for _ in range(2)]
+    ds = [torch.empty_like(hk, device="cuda") for _ in range(2)] if paper else dk
+    d_idx = [torch.empty(group, w.heads, total_keep, dtype=torch.int32, device="cuda") for _ in range(2)]
+    d_ko = [torch.empty(group, w.heads, total_keep, w.d, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    d_vo = [torch.empty_like(d_ko[0]) for _ in range(2)]
+    ws = B.alloc_workspace(g_shape)
+    copy_in, copy_out = torch.cuda.Stream(), torch.cuda.Stream()
+    main = torch.cuda.current_stream()
+
+    def one_step():
+        in_done = [torch.cuda.Event() for _ in range(n_groups)]
+        comp_done = [torch.cuda.Event() for _ in range(n_groups)]
+        out_done = [torch.cuda.Event() for _ in range(n_groups)]
+        for g in range(n_groups):
+            s = g & 1
+            with torch.cuda.stream(copy_in):
+                if g >= 2:
+                    copy_in.wait_event(comp_done[g - 2])      # slot's previous inputs consumed
+                dk[s].copy_(hk, non_blocking=True); dv[s].copy_(hv, non_blocking=True)
+                if paper:
+                    ds[s].copy_(hs, non_blocking=True)
+                in_done[g].record(copy_in)
+            main.wait_event(in_done[g])
+            if g >= 2:
+                main.wait_event(out_done[g - 2])              # slot's previous outputs copied out
+            B.compress(g_shape, ds[s], dk[s], dv[s], phi_d, keep, d_idx[s], d_ko[s], d_vo[s], ws)
+            comp_done[g].record(main)
+            with torch.cuda.stream(copy_out):
+                copy_out.wait_event(comp_done[g])
+                h_idx.copy_(d_idx[s], non_blocking=True)
+                h_ko.copy_(d_ko[s], non_blocking=True); h_vo.copy_(d_vo[s], non_blocking=True)
+                out_done[g].record(copy_out)
+        main.wait_event(out_done[-1])
+
+    steps = max(1, min(args.steps, 3))
+    one_step()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(steps):
+        one_step()
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / steps
+    if dist is not None:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    row = w.d * 2
+    h2d = n_groups * group * w.heads * T * row * (3 if paper else 2)
+    d2h = n_groups * group * w.heads * total_keep * (2 * row + 4)
+    return {"value": w.total_tokens * world / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "how": f"{n_groups} groups of {group} layers streamed through pinned host buffers, double-buffered"}
+
+
+if __name__ == "__main__":
+    main()

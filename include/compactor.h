@@ -115,7 +115,7 @@ size_t compactor_workspace_bytes(const compactor_shape* shape);
  *   scores_out   device fp32 [layers][heads][total_tokens].
  * The small factorisation is a Cholesky factorisation of G = (K Phi)^T (K Phi) in fp64 - one of
  * the algebraically equal routes the paper allows (Section 3.2, Appendix C); Gram sums are fp32
- * per block of at most 2048 tokens and fp64 across blocks.
+ * per block of at most 4096 tokens and fp64 across blocks.
  */
 int compactor_score(const compactor_shape* shape, compactor_mat k_score, const float* phi,
                     const float* attn_scores, float lambda, float* scores_out,
@@ -153,6 +153,22 @@ int compactor_compress(const compactor_shape* shape, compactor_mat k_score, comp
                        float lambda, const int32_t* keep_counts,
                        float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
                        int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * compactor_compress with stage markers, for measurement (the paper reports one wall-clock
+ * number per context length, Fig. 1; this splits ours by stage).  stage_events is a HOST array of
+ * n_events cudaEvent_t handles created by the caller (NULL entries are skipped).  They are
+ * recorded on the stream: [0] before the first kernel, [1] after the Gram pass, [2] after the
+ * factorisation, [3] after the scoring pass, [4] after the blend (recorded even when there is
+ * none), [5] after selection, [6] after compaction.  Results are identical to compactor_compress.
+ */
+#define COMPACTOR_N_STAGE_EVENTS 7
+int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
+                                compactor_mat v_cache, const float* phi, const float* attn_scores,
+                                float lambda, const int32_t* keep_counts,
+                                float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
+                                int32_t* status, void* workspace, size_t workspace_bytes, void* stream,
+                                void* const* stage_events, int32_t n_events);
 
 #ifdef __cplusplus
 }

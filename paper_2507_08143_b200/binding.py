@@ -51,6 +51,7 @@ def _load() -> ctypes.CDLL:
     lib.compactor_compress.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, CompactorMat, c_void_p,
                                        c_void_p, c_float, POINTER(c_int32), c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_compress_profiled.argtypes = lib.compactor_compress.argtypes + [POINTER(c_void_p), c_int32]
     return lib
 
 
@@ -59,7 +60,10 @@ LIB_PATH = _build.LIB
 
 EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_keep_count",
            "compactor_calibrated_ratio", "compactor_workspace_bytes", "compactor_score", "compactor_select",
-           "compactor_compact", "compactor_compress"]
+           "compactor_compact", "compactor_compress", "compactor_compress_profiled"]
+
+N_STAGE_EVENTS = 7
+STAGE_NAMES = ["gram", "factor", "score", "blend", "select", "compact"]
 
 
 def version() -> int:
@@ -162,3 +166,17 @@ def compress(shape: Shape, k_score: torch.Tensor, k_cache: torch.Tensor, v_cache
     _check(LIB.compactor_compress(byref(shape.c), mat(k_score), mat(k_cache), mat(v_cache), _ptr(phi), _ptr(attn), lam,
                                   _keep_array(keep_counts), _ptr(scores_out), _ptr(idx_out), _ptr(k_out), _ptr(v_out),
                                   _ptr(status), _ptr(workspace), workspace.numel(), _stream()), "compactor_compress")
+
+
+def compress_profiled(shape: Shape, k_score: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor,
+                      phi: torch.Tensor, keep_counts: Sequence[int], idx_out: torch.Tensor, k_out: torch.Tensor,
+                      v_out: torch.Tensor, workspace: torch.Tensor, events: Sequence[torch.cuda.Event],
+                      attn: Optional[torch.Tensor] = None, lam: float = 0.3,
+                      scores_out: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None) -> None:
+    """`events`: N_STAGE_EVENTS torch events with timing enabled that have been recorded once before
+    (so that their CUDA handles exist); the library re-records them between its kernels."""
+    handles = (c_void_p * len(events))(*[c_void_p(e.cuda_event) for e in events])
+    _check(LIB.compactor_compress_profiled(byref(shape.c), mat(k_score), mat(k_cache), mat(v_cache), _ptr(phi),
+                                           _ptr(attn), lam, _keep_array(keep_counts), _ptr(scores_out), _ptr(idx_out),
+                                           _ptr(k_out), _ptr(v_out), _ptr(status), _ptr(workspace), workspace.numel(),
+                                           _stream(), handles, len(events)), "compactor_compress_profiled")

@@ -120,14 +120,30 @@ cudaError_t upload_tables(HostPlan* hp, void* ws, cudaStream_t stream) {
 
 #define CK(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) return COMPACTOR_E_CUDA; } while (0)
 
+// Optional stage markers: caller-created events recorded on the stream between kernels.
+struct Marks {
+    void* const* ev = nullptr;
+    int n = 0;
+    cudaError_t mark(int i, cudaStream_t st) const {
+        if (ev == nullptr || i >= n || ev[i] == nullptr) return cudaSuccess;
+        return cudaEventRecord(static_cast<cudaEvent_t>(ev[i]), st);
+    }
+};
+
 int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn, float lambda,
-                float* scores, int32_t* status, char* ws, cudaStream_t stream) {
+                float* scores, int32_t* status, char* ws, cudaStream_t stream, const Marks& mk = Marks()) {
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(ws + hp.off_w);
     float* partials = reinterpret_cast<float*>(ws + hp.off_partials);
-    CK(launch_gram(hp.plan, k, partials, stream));
+    if (status != nullptr) CK(cudaMemsetAsync(status, 0, sizeof(int32_t) * hp.units, stream));
+    CK(mk.mark(0, stream));
+    CK(launch_gram(hp.plan, k, partials, status, stream));
+    CK(mk.mark(1, stream));
     CK(launch_factor(hp.plan, k, partials, phi, w, status, stream));
-    CK(launch_score(hp.plan, k, w, scores, stream));
+    CK(mk.mark(2, stream));
+    CK(launch_score(hp.plan, k, w, scores, status, stream));
+    CK(mk.mark(3, stream));
     if (attn != nullptr) CK(launch_blend(hp.plan, attn, lambda, scores, stream));
+    CK(mk.mark(4, stream));
     return COMPACTOR_OK;
 }
 
@@ -242,11 +258,11 @@ int compactor_compact(const compactor_shape* shape, compactor_mat k_cache, compa
     return COMPACTOR_OK;
 }
 
-int compactor_compress(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
-                       compactor_mat v_cache, const float* phi, const float* attn_scores,
-                       float lambda, const int32_t* keep_counts,
-                       float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
-                       int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
+static int compress_impl(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
+                         compactor_mat v_cache, const float* phi, const float* attn_scores,
+                         float lambda, const int32_t* keep_counts,
+                         float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
+                         int32_t* status, void* workspace, size_t workspace_bytes, void* stream, const Marks& mk) {
     HostPlan hp; int err = 0;
     if (!make_plan(shape, &hp, &err)) return err;
     if (!mat_ok(k_score) || !mat_ok(k_cache) || !mat_ok(v_cache) || phi == nullptr || idx_out == nullptr ||
@@ -260,13 +276,36 @@ int compactor_compress(const compactor_shape* shape, compactor_mat k_score, comp
     char* ws = static_cast<char*>(workspace);
     float* scores = scores_out != nullptr ? scores_out : reinterpret_cast<float*>(ws + hp.off_scores);
     CK(upload_tables(&hp, workspace, st));
-    int rc = run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores, status, ws, st);
+    int rc = run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores, status, ws, st, mk);
     if (rc != COMPACTOR_OK) return rc;
-    if (hp.plan.total_keep == 0) return COMPACTOR_OK;
-    CK(launch_select(hp.plan, scores, idx_out, st));
-    CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out,
-                      static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
+    if (hp.plan.total_keep > 0) CK(launch_select(hp.plan, scores, idx_out, st));
+    CK(mk.mark(5, st));
+    if (hp.plan.total_keep > 0)
+        CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out,
+                          static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
+    CK(mk.mark(6, st));
     return COMPACTOR_OK;
+}
+
+int compactor_compress(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
+                       compactor_mat v_cache, const float* phi, const float* attn_scores,
+                       float lambda, const int32_t* keep_counts,
+                       float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
+                       int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
+    return compress_impl(shape, k_score, k_cache, v_cache, phi, attn_scores, lambda, keep_counts, scores_out,
+                         idx_out, k_out, v_out, status, workspace, workspace_bytes, stream, Marks());
+}
+
+int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
+                                compactor_mat v_cache, const float* phi, const float* attn_scores,
+                                float lambda, const int32_t* keep_counts,
+                                float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
+                                int32_t* status, void* workspace, size_t workspace_bytes, void* stream,
+                                void* const* stage_events, int32_t n_events) {
+    if (stage_events == nullptr || n_events < 0) return COMPACTOR_E_INVALID_ARGUMENT;
+    Marks mk; mk.ev = stage_events; mk.n = n_events;
+    return compress_impl(shape, k_score, k_cache, v_cache, phi, attn_scores, lambda, keep_counts, scores_out,
+                         idx_out, k_out, v_out, status, workspace, workspace_bytes, stream, mk);
 }
 
 }  // extern "C"

@@ -10,7 +10,7 @@ namespace compactor {
 
 constexpr int kD = 128;            // head dimension the kernels are written for
 constexpr int kMaxM = 64;          // largest sketch dimension
-constexpr int kMaxChunk = 2048;    // most tokens whose Gram matrix is summed in fp32 before the fp64 reduction
+constexpr int kMaxChunk = 4096;    // most tokens whose Gram matrix is summed in fp32 before the fp64 reduction
 constexpr int kMinChunk = 256;
 constexpr int kGramElems = kD * kD;
 
@@ -46,10 +46,11 @@ __device__ __forceinline__ int find_segment(const int* __restrict__ table, int n
 
 // Kernel launchers (each defined next to its kernel).  All enqueue on `stream` and return the
 // launch status.
-cudaError_t launch_gram(const Plan& p, const Mat& k, float* partials, cudaStream_t stream);
+cudaError_t launch_gram(const Plan& p, const Mat& k, float* partials, int* status, cudaStream_t stream);
 cudaError_t launch_factor(const Plan& p, const Mat& k, const float* partials, const float* phi, __nv_bfloat16* w,
                           int* status, cudaStream_t stream);
-cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, cudaStream_t stream);
+cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
+                         cudaStream_t stream);
 cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* scores, cudaStream_t stream);
 cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStream_t stream);
 cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int* idx,

@@ -192,7 +192,7 @@ factor_kernel(Plan p, Mat kmat, const float* __restrict__ partials, const float*
             w_lo[j * kD + tid] = lo;
         }
     }
-    if (tid == 0 && status != nullptr) status[unit] = s.flags;
+    if (tid == 0 && status != nullptr && s.flags != 0) atomicOr(&status[unit], s.flags);
 }
 
 }  // namespace

@@ -1,44 +1,46 @@
 // Scoring pass (Algorithm 1, lines 5-6, fused): o_i = || k_i W ||^2 with W = Phi L^-T from the
 // factor kernel, so that U~ = K^ V~ Sigma~^-1 is never stored.  W arrives as two bf16 terms
 // (hi + lo); both are multiplied with the bf16 keys on the tensor cores and summed in fp32.
+//
+// One CTA per block of tokens of one unit.  Warp 0 streams 128-token tiles of K (and W once)
+// with TMA; one thread of warp 1 issues tcgen05.mma (A = key tile, K-major; B = W^T, K-major;
+// D = 128 tokens x MP fp32 in tensor memory, double buffered); warps 2-5 read D back, square,
+// sum along the row and store one fp32 score per token.
 #include "common.cuh"
+#include "sm100.cuh"
 
 namespace compactor {
 namespace {
 
-constexpr int kTileTokens = 128;
-constexpr int kStages = 2;
-constexpr int kThreads = 256;
-constexpr int kTileBytes = kTileTokens * kD * 2;
+using namespace sm100;
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ uint32_t tile_offset(int row, int col) {
-    return (uint32_t)(row * (kD * 2) + ((((col >> 3) ^ (row & 7))) << 4));
-}
-__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, bool valid) {
-    int bytes = valid ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(bytes));
-}
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
+constexpr int kTile = 128;
+constexpr int kStages = 3;
+constexpr int kBoxBytes = kTile * 128;
+constexpr int kTileBytes = 2 * kBoxBytes;
+constexpr int kThreads = 192;
+constexpr uint32_t kTmemCols = 128;       // two accumulators of up to 64 columns
 
-// MP = padded sketch dimension (multiple of 16).  One CTA scores one Gram chunk of one unit.
 template <int MP>
-__global__ void __launch_bounds__(kThreads, 1)
-score_kernel(Plan p, Mat k, const __nv_bfloat16* __restrict__ w, float* __restrict__ scores) {
-    extern __shared__ __align__(128) unsigned char smem[];
-    constexpr int kWBytes = 2 * MP * kD * 2;
+struct __align__(1024) ScoreSmem {
+    unsigned char tiles[kStages][kTileBytes];
+    unsigned char w[2][2][MP * 128];      // [term][channel half][MP rows x 64 channels]
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t w_full;
+    uint64_t d_full[2];
+    uint64_t d_empty[2];
+    uint32_t tmem_base;
+    int abort;
+};
+
+template <int MP>
+__global__ void __launch_bounds__(kThreads, 2)
+score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap,
+             float* __restrict__ scores, int* __restrict__ status) {
+    extern __shared__ unsigned char smem_raw[];
+    using Smem = ScoreSmem<MP>;
+    Smem& s = *reinterpret_cast<Smem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
     const int chunk_id = blockIdx.x;
     const int lh = blockIdx.y;
     const int layer = lh / p.heads, head = lh % p.heads;
@@ -46,102 +48,133 @@ score_kernel(Plan p, Mat k, const __nv_bfloat16* __restrict__ w, float* __restri
     const int tok_begin = p.cu_seqlens[b] + (chunk_id - p.cu_chunks[b]) * p.chunk;
     const int tok_end = min(tok_begin + p.chunk, p.cu_seqlens[b + 1]);
     const int n_tok = tok_end - tok_begin;
-    const int n_tiles = (n_tok + kTileTokens - 1) / kTileTokens;
+    const int n_tiles = (n_tok + kTile - 1) / kTile;
     const int unit = lh * p.batch + b;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    const __nv_bfloat16* base = k.ptr + layer * k.stride_layer + head * k.stride_head +
-                                (long long)tok_begin * k.stride_token;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t w_base = smem_u32(smem);
-    const uint32_t k_base = w_base + kWBytes;
-
-    // W of this unit: rows = (term, sketch column), 128 channels each, same piece permutation as
-    // the key tiles.
-    {
-        const __nv_bfloat16* wsrc = w + (size_t)unit * w_elems_per_unit(MP);
-        for (int c = tid; c < 2 * MP * 16; c += kThreads) {
-            int row = c >> 4, piece = c & 15;
-            cp_async_16(w_base + tile_offset(row, piece * 8), wsrc + row * kD + piece * 8, true);
-        }
+    if (threadIdx.x == 0) {
+        prefetch_tensormap(&kmap);
+        prefetch_tensormap(&wmap);
+        for (int i = 0; i < kStages; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
+        mbar_init(&s.w_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&s.d_full[i], 1); mbar_init(&s.d_empty[i], 4); }
+        s.abort = 0;
+        fence_barrier_init();
     }
-    auto load_tile = [&](int tile, int stage) {
-        const uint32_t dst = k_base + stage * kTileBytes;
-#pragma unroll
-        for (int i = 0; i < (kTileTokens * 16) / kThreads; ++i) {
-            int c = tid + i * kThreads;
-            int row = c >> 4, piece = c & 15;
-            int tok = tile * kTileTokens + row;
-            bool valid = tok < n_tok;
-            const __nv_bfloat16* src = base + (long long)(valid ? tok : 0) * k.stride_token + piece * 8;
-            cp_async_16(dst + tile_offset(row, piece * 8), src, valid);
-        }
-    };
-    load_tile(0, 0);
-    asm volatile("cp.async.commit_group;\n");
+    if (warp == 1) { tmem_alloc(&s.tmem_base, kTmemCols); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = s.tmem_base;
 
-    float* out = scores + (size_t)lh * p.total_tokens + tok_begin;
-    const int j = lane >> 3, r = lane & 7;
-    for (int t = 0; t < n_tiles; ++t) {
-        if (t + 1 < n_tiles) load_tile(t + 1, (t + 1) & 1);
-        asm volatile("cp.async.commit_group;\n");
-        asm volatile("cp.async.wait_group 1;\n");
-        __syncthreads();
-        const uint32_t tile_base = k_base + (t & 1) * kTileBytes;
-        float acc[MP / 8][4];
-#pragma unroll
-        for (int nt = 0; nt < MP / 8; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-            uint32_t a[4];
-            ldmatrix_x4(a, tile_base + tile_offset(warp * 16 + r + ((j & 1) ? 8 : 0), ks * 16 + ((j & 2) ? 8 : 0)));
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&s.w_full, 4 * MP * 128);
 #pragma unroll
             for (int term = 0; term < 2; ++term)
 #pragma unroll
-                for (int np = 0; np < MP / 16; ++np) {
-                    uint32_t bf[4];
-                    ldmatrix_x4(bf, w_base + tile_offset(term * MP + np * 16 + r + ((j & 2) ? 8 : 0),
-                                                         ks * 16 + ((j & 1) ? 8 : 0)));
-                    mma_bf16(acc[2 * np], a, bf[0], bf[1]);
-                    mma_bf16(acc[2 * np + 1], a, bf[2], bf[3]);
-                }
+                for (int half = 0; half < 2; ++half)
+                    tma_load_2d(s.w[term][half], &wmap, &s.w_full, half * 64, (unit * 2 + term) * MP);
+            for (int t = 0; t < n_tiles; ++t) {
+                const int stage = t % kStages, round = t / kStages;
+                if (round > 0 && !mbar_wait(&s.empty[stage], (round - 1) & 1)) { s.abort = 1; break; }
+                if (*(volatile int*)&s.abort) break;
+                mbar_arrive_expect_tx(&s.full[stage], kTileBytes);
+                const int tok = tok_begin + t * kTile;
+                tma_load_4d(s.tiles[stage], &kmap, &s.full[stage], 0, tok, head, layer);
+                tma_load_4d(s.tiles[stage] + kBoxBytes, &kmap, &s.full[stage], 64, tok, head, layer);
+            }
         }
-        float lo = 0.f, hi = 0.f;     // rows lane/4 and lane/4 + 8 of the warp's 16 tokens
+    } else if (warp == 1) {
+        constexpr uint32_t idesc = umma_idesc_bf16(128, MP, 0, 0);
+        bool ok = mbar_wait(&s.w_full, 0);
+        for (int t = 0; t < n_tiles && ok; ++t) {
+            const int stage = t % kStages, round = t / kStages;
+            const int buf = t & 1, use = t >> 1;
+            ok = mbar_wait(&s.full[stage], round & 1);
+            if (ok && use > 0) ok = mbar_wait(&s.d_empty[buf], (use - 1) & 1);
+            ok = ok && !*(volatile int*)&s.abort;
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t a_base = smem_u32(s.tiles[stage]);
+                const uint32_t d_addr = tmem + buf * 64;
 #pragma unroll
-        for (int nt = 0; nt < MP / 8; ++nt) {
-            lo = fmaf(acc[nt][0], acc[nt][0], lo); lo = fmaf(acc[nt][1], acc[nt][1], lo);
-            hi = fmaf(acc[nt][2], acc[nt][2], hi); hi = fmaf(acc[nt][3], acc[nt][3], hi);
+                for (int term = 0; term < 2; ++term)
+#pragma unroll
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const int half = ks >> 2, off = (ks & 3) * 32;
+                        const uint64_t a_desc = umma_desc_sw128(a_base + half * kBoxBytes + off, 16, 1024);
+                        const uint64_t b_desc = umma_desc_sw128(smem_u32(s.w[term][half]) + off, 16, 1024);
+                        umma_bf16(d_addr, a_desc, b_desc, idesc, (term > 0) || (ks > 0));
+                    }
+                umma_commit(&s.empty[stage]);
+                umma_commit(&s.d_full[buf]);
+            }
+            __syncwarp();
         }
-        lo += __shfl_xor_sync(0xffffffffu, lo, 1); lo += __shfl_xor_sync(0xffffffffu, lo, 2);
-        hi += __shfl_xor_sync(0xffffffffu, hi, 1); hi += __shfl_xor_sync(0xffffffffu, hi, 2);
-        if ((lane & 3) == 0) {
-            int tok = t * kTileTokens + warp * 16 + (lane >> 2);
-            if (tok < n_tok) out[tok] = lo;
-            if (tok + 8 < n_tok) out[tok + 8] = hi;
+        if (!ok) {
+            s.abort = 1;
+            if (lane == 0) { mbar_arrive(&s.d_full[0]); mbar_arrive(&s.d_full[1]); }   // wake the epilogue
         }
-        __syncthreads();   // the stage read here is refilled at the top of the next iteration
+    } else {
+        const int q = warp & 3;
+        float* out = scores + (size_t)lh * p.total_tokens + tok_begin;
+        for (int t = 0; t < n_tiles; ++t) {
+            const int buf = t & 1, use = t >> 1;
+            const bool ok = mbar_wait(&s.d_full[buf], use & 1);
+            if (!ok) s.abort = 1;
+            if (!ok || *(volatile int*)&s.abort) break;
+            tc_fence_after_sync();
+            float acc = 0.f;
+#pragma unroll
+            for (int c0 = 0; c0 < MP; c0 += 16) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(tmem + ((uint32_t)(q * 32) << 16) + buf * 64 + c0, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { float v = __uint_as_float(r[i]); acc = fmaf(v, v, acc); }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s.d_empty[buf]);
+            const int tok = t * kTile + q * 32 + lane;
+            if (tok < n_tok) out[tok] = acc;
+        }
     }
-    asm volatile("cp.async.wait_group 0;\n");
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    if (threadIdx.x == 0 && s.abort && status != nullptr) atomicOr(&status[unit], COMPACTOR_STATUS_TIMEOUT);
 }
 
 template <int MP>
-cudaError_t launch_score_mp(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, cudaStream_t stream) {
-    const int smem = 2 * MP * kD * 2 + kStages * kTileBytes;
+cudaError_t launch_score_mp(const Plan& p, const CUtensorMap& kmap, const CUtensorMap& wmap, float* scores,
+                            int* status, cudaStream_t stream) {
+    const int smem = (int)sizeof(ScoreSmem<MP>) + 1024;
     cudaError_t e = cudaFuncSetAttribute(score_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(p.total_chunks, p.layers * p.heads);
-    score_kernel<MP><<<grid, kThreads, smem, stream>>>(p, k, w, scores);
+    score_kernel<MP><<<grid, kThreads, smem, stream>>>(p, kmap, wmap, scores, status);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, cudaStream_t stream) {
+cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
+                         cudaStream_t stream) {
     if (p.total_chunks == 0) return cudaSuccess;
+    CUtensorMap kmap, wmap;
+    const long long units = (long long)p.layers * p.heads * p.batch;
+    if (!make_kv_tensor_map(&kmap, k.ptr, p.layers, p.heads, p.total_tokens, k.stride_layer, k.stride_head,
+                            k.stride_token, kTile) ||
+        !make_rows_tensor_map(&wmap, w, units * 2 * p.mp, p.mp))
+        return cudaErrorInvalidValue;
     switch (p.mp) {
-        case 16: return launch_score_mp<16>(p, k, w, scores, stream);
-        case 32: return launch_score_mp<32>(p, k, w, scores, stream);
-        case 48: return launch_score_mp<48>(p, k, w, scores, stream);
-        case 64: return launch_score_mp<64>(p, k, w, scores, stream);
+        case 16: return launch_score_mp<16>(p, kmap, wmap, scores, status, stream);
+        case 32: return launch_score_mp<32>(p, kmap, wmap, scores, status, stream);
+        case 48: return launch_score_mp<48>(p, kmap, wmap, scores, status, stream);
+        case 64: return launch_score_mp<64>(p, kmap, wmap, scores, status, stream);
         default: return cudaErrorInvalidValue;
     }
 }

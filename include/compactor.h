@@ -44,6 +44,7 @@ extern "C" {
 #define COMPACTOR_E_UNSUPPORTED      -2   /* d != 128 or m outside [1, 64]                       */
 #define COMPACTOR_E_WORKSPACE        -3   /* workspace smaller than compactor_workspace_bytes()  */
 #define COMPACTOR_E_CUDA             -4   /* a CUDA runtime call failed (see cudaGetLastError)   */
+#define COMPACTOR_E_TOO_LARGE        -5   /* problem exceeds the library's built-in scratch      */
 
 #define COMPACTOR_STATUS_NONFINITE   1
 #define COMPACTOR_STATUS_RANK        2
@@ -169,6 +170,29 @@ int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_sc
                                 float* scores_out, int32_t* idx_out, void* k_out, void* v_out,
                                 int32_t* status, void* workspace, size_t workspace_bytes, void* stream,
                                 void* const* stage_events, int32_t n_events);
+
+/*
+ * compactor_score for callers that cannot allocate device memory (the paper has no counterpart;
+ * this is a deployment convenience).  Same inputs, outputs and results as compactor_score, but
+ * no workspace argument: the scratch is a fixed array of compactor_builtin_scratch_bytes()
+ * (32 MiB) inside the library, resident on every device the process uses from the first use of
+ * the library on that device until the process exits.  The call allocates and frees nothing.
+ *   - Size limit: the scratch must hold 12*(batch+1) bytes of tables, 512*ceil(m/16)*16 bytes per
+ *     unit and 64 KiB per Gram block (blocks are lengthened up to 4096 tokens to make it fit,
+ *     i.e. about 16 bytes per token per (layer, head)).  A larger problem is refused with
+ *     COMPACTOR_E_TOO_LARGE before anything is enqueued; split it by layers or use
+ *     compactor_score.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls share the one array and it keeps whatever the previous call left there (nothing
+ *     in it needs clearing: every call rewrites what it reads).  Two calls whose device work
+ *     can overlap - different streams, or different host threads on the same device - race on
+ *     it; order them on one stream or with events.
+ */
+size_t compactor_builtin_scratch_bytes(void);
+int compactor_score_builtin_scratch(const compactor_shape* shape, compactor_mat k_score, const float* phi,
+                                    const float* attn_scores, float lambda, float* scores_out,
+                                    int32_t* status, void* stream);
 
 #ifdef __cplusplus
 }

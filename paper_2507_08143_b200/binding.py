@@ -52,6 +52,9 @@ def _load() -> ctypes.CDLL:
                                        c_void_p, c_float, POINTER(c_int32), c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_void_p, c_size_t, c_void_p]
     lib.compactor_compress_profiled.argtypes = lib.compactor_compress.argtypes + [POINTER(c_void_p), c_int32]
+    lib.compactor_builtin_scratch_bytes.restype = c_size_t
+    lib.compactor_score_builtin_scratch.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_void_p, c_float,
+                                                    c_void_p, c_void_p, c_void_p]
     return lib
 
 
@@ -60,7 +63,8 @@ LIB_PATH = _build.LIB
 
 EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_keep_count",
            "compactor_calibrated_ratio", "compactor_workspace_bytes", "compactor_score", "compactor_select",
-           "compactor_compact", "compactor_compress", "compactor_compress_profiled"]
+           "compactor_compact", "compactor_compress", "compactor_compress_profiled",
+           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch"]
 
 N_STAGE_EVENTS = 7
 STAGE_NAMES = ["gram", "factor", "score", "blend", "select", "compact"]
@@ -180,3 +184,17 @@ def compress_profiled(shape: Shape, k_score: torch.Tensor, k_cache: torch.Tensor
                                            _ptr(attn), lam, _keep_array(keep_counts), _ptr(scores_out), _ptr(idx_out),
                                            _ptr(k_out), _ptr(v_out), _ptr(status), _ptr(workspace), workspace.numel(),
                                            _stream(), handles, len(events)), "compactor_compress_profiled")
+
+
+def builtin_scratch_bytes() -> int:
+    return int(LIB.compactor_builtin_scratch_bytes())
+
+
+def score_builtin_scratch(shape: Shape, k_score: torch.Tensor, phi: torch.Tensor, scores_out: torch.Tensor,
+                          attn: Optional[torch.Tensor] = None, lam: float = 0.3,
+                          status: Optional[torch.Tensor] = None) -> None:
+    """compactor_score without a workspace: for callers that may not allocate device memory.  The
+    scratch is the library's fixed 32 MiB array; problems that do not fit raise CompactorError(-5)."""
+    _check(LIB.compactor_score_builtin_scratch(byref(shape.c), mat(k_score), _ptr(phi), _ptr(attn), lam,
+                                               _ptr(scores_out), _ptr(status), _stream()),
+           "compactor_score_builtin_scratch")

@@ -3,6 +3,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -160,6 +161,7 @@ const char* compactor_error_string(int code) {
         case COMPACTOR_E_UNSUPPORTED: return "unsupported shape (d must be 128, 1 <= m <= 64)";
         case COMPACTOR_E_WORKSPACE: return "workspace too small";
         case COMPACTOR_E_CUDA: return "CUDA runtime error";
+        case COMPACTOR_E_TOO_LARGE: return "problem needs more scratch than the built-in 32 MiB array holds";
         default: return "unknown status";
     }
 }
@@ -306,6 +308,82 @@ int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_sc
     Marks mk; mk.ev = stage_events; mk.n = n_events;
     return compress_impl(shape, k_score, k_cache, v_cache, phi, attn_scores, lambda, keep_counts, scores_out,
                          idx_out, k_out, v_out, status, workspace, workspace_bytes, stream, mk);
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Scoring without a caller-provided workspace.
+//
+// Some hosts of this library may not allocate device memory when they need scores: a serving
+// engine that has handed the whole device to its own paged-cache allocator, a plugin running
+// under an allocator lock, or code between the begin and end of a stream capture, where
+// cudaMalloc is not permitted.  For them the scratch that compactor_score normally takes from
+// the caller lives in this fixed array, which every process that loads the library holds on
+// each device it uses, until exit.
+namespace {
+
+constexpr size_t kBuiltinScratchBytes = (size_t)32 << 20;     // 32 MiB
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_builtin_scratch_ptr[kMaxDevices] = {};
+std::mutex g_builtin_scratch_mutex;
+
+// Device address of the array on the current device.  In host code the array's name is only a
+// handle for the runtime, never an address a kernel may use; the real address is asked for once
+// per device and remembered.
+int builtin_scratch(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return COMPACTOR_E_CUDA;
+    std::lock_guard<std::mutex> lock(g_builtin_scratch_mutex);
+    if (g_builtin_scratch_ptr[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_builtin_scratch) != cudaSuccess || ptr == nullptr) return COMPACTOR_E_CUDA;
+        g_builtin_scratch_ptr[dev] = ptr;
+    }
+    *out = g_builtin_scratch_ptr[dev];
+    return COMPACTOR_OK;
+}
+
+// Re-derives the chunk-dependent part of a plan for a given Gram block length.
+void replan_chunk(const compactor_shape* s, HostPlan* hp, int chunk) {
+    Plan& p = hp->plan;
+    const int nb1 = s->batch + 1;
+    int* cs = hp->tables.data();
+    int* cc = cs + 2 * nb1;
+    cc[0] = 0;
+    for (int b = 0; b < s->batch; ++b) cc[b + 1] = cc[b] + (cs[b + 1] - cs[b] + chunk - 1) / chunk;
+    p.chunk = chunk;
+    p.total_chunks = cc[s->batch];
+    hp->off_scores = hp->off_partials +
+                     align_up(sizeof(float) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
+    hp->total_bytes = hp->off_scores + align_up(sizeof(float) * (size_t)p.total_tokens * s->layers * s->heads);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t compactor_builtin_scratch_bytes(void) { return kBuiltinScratchBytes; }
+
+int compactor_score_builtin_scratch(const compactor_shape* shape, compactor_mat k_score, const float* phi,
+                                    const float* attn_scores, float lambda, float* scores_out,
+                                    int32_t* status, void* stream) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (!mat_ok(k_score) || phi == nullptr || scores_out == nullptr) return COMPACTOR_E_INVALID_ARGUMENT;
+    // Everything before the scores region must fit; longer Gram blocks need less scratch.
+    while (hp.off_scores > kBuiltinScratchBytes && hp.plan.chunk < kMaxChunk) replan_chunk(shape, &hp, hp.plan.chunk * 2);
+    if (hp.off_scores > kBuiltinScratchBytes) return COMPACTOR_E_TOO_LARGE;
+    if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
+    void* scratch = nullptr;
+    int rc = builtin_scratch(&scratch);
+    if (rc != COMPACTOR_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CK(upload_tables(&hp, scratch, st));
+    return run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores_out, status,
+                       static_cast<char*>(scratch), st);
 }
 
 }  // extern "C"

@@ -18,8 +18,8 @@
  *   - Sequences are packed back to back along the token axis: sequence b owns tokens
  *     [cu_seqlens[b], cu_seqlens[b+1]) of every (layer, head).  A "unit" is one
  *     (layer, head, sequence) triple; unit id = (layer * heads + head) * batch + b.
- *     Units are scored and selected independently (Section 3: "the same procedure is applied
- *     to heads independently").
+ *     Units are scored and selected independently (Section 3, Notation: heads are treated
+ *     one by one).
  *   - Kept rows of sequence b occupy rows [cu_keep[b], cu_keep[b+1]) of every (layer, head)
  *     block of the outputs, cu_keep = prefix sums of keep_counts; total_keep = cu_keep[batch].
  *   - Outputs must not alias inputs or the workspace.
@@ -123,7 +123,7 @@ int compactor_score(const compactor_shape* shape, compactor_mat k_score, const f
                     int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * Per-unit top-k (Section 3.4, "retain the top ceil(r N) tokens ... within a single head").
+ * Per-unit top-k (Section 3.4: the ceil(r N) highest-scoring tokens are kept, here per head).
  *   scores       device fp32 [layers][heads][total_tokens].
  *   keep_counts  host int32 [batch]: tokens kept per sequence (0 <= keep <= length), the same
  *                for every layer and head.

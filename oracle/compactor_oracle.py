@@ -13,7 +13,7 @@ What follows the paper step by step:
     approximates; used to pin the oracle, and as the m = d special case).
   * `blend`                  - Eq. 6 (z-scored attention term + lambda * z-scored
     outlier term).
-  * `keep_count`             - "retain the top ceil(r N) tokens" (Section 3,
+  * `keep_count`             - the number of retained tokens, ceil(r N) (Section 3,
     Preliminaries; Section 3.4).
   * `top_k_indices`          - per-head top-k of the scores.
   * `compact`                - the retained rows of K and V.
@@ -32,9 +32,9 @@ Readings taken where the paper is silent or inconsistent:
     emitted in ascending order (the paper does not say).
   * std in Eq. 6 is the population standard deviation; a term whose std is 0
     contributes 0.  With no attention term the score is the outlier score o.
-  * The calibration curve is increasing in r; the paper's "arg max ... such
-    that f >= tau" is read as the smallest such r (Section 3.5 opens with
-    "the smallest r that leaves model quality unchanged").
+  * The calibration curve is increasing in r; the paper writes the choice of
+    r* as an arg max subject to f >= tau, which is read as the smallest such r
+    (Section 3.5 states the goal as the least retention that keeps quality).
 
 Pins (see tests/test_oracle_pins.py): closed-form leverage scores, sum = rank,
 range [0,1], invariance under K -> K A and Phi -> Phi A, m = d reduces to the

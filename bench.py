@@ -213,7 +213,7 @@ def main():
         return
 
     import torch
-    from paper_2507_08143_b200 import binding as B, inputs
+    from paper_2507_08143_b200 import binding as B, inputs, sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -225,8 +225,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    w = inputs.workload(args.workload, layers=args.layers)
-    w.seed = w.seed + 1000 * rank
+    w = sharding.rank_workload(inputs.workload(args.workload, layers=args.layers), rank)
     shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
     keep = [B.keep_count(n, r) for n, r in zip(w.seqlens, w.ratios)]
     total_keep = sum(keep)
@@ -274,13 +273,9 @@ def main():
     barrier()
     elapsed_ms = t_beg.elapsed_time(t_end)
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = sharding.max_over_ranks(elapsed_ms, dist, device="cuda")
     ms_per_step = elapsed_ms / args.steps
-    tokens_per_step = w.total_tokens * world
-    value = tokens_per_step / (ms_per_step * 1e-3)
+    value = sharding.job_tokens_per_second(w.total_tokens, world, ms_per_step)
     assert int(status.max().item()) == 0, "a unit reported a numerical status flag"
 
     # per-kernel times from the stage markers of the timed region
@@ -398,10 +393,8 @@ def e2e(args, B, w, shape, keep, phi_d, k_score, kr, v, dist, world):
     t1.record()
     torch.cuda.synchronize()
     ms = t0.elapsed_time(t1) / steps
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2507_08143_b200 import sharding
+    ms = sharding.max_over_ranks(ms, dist, device="cuda")
     row = w.d * 2
     h2d = n_groups * group * w.heads * T * row * (3 if paper else 2)
     d2h = n_groups * group * w.heads * total_keep * (2 * row + 4)

@@ -1,0 +1,98 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every declared entry
+point, its host helpers agree with the oracle, and argument errors are caught before any launch."""
+import ctypes
+import math
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import compactor_oracle as orc
+from paper_2507_08143_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_every_declared_symbol_is_exported():
+    header = open(os.path.join(ROOT, "include", "compactor.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(compactor_[a-z_0-9]+)\s*\(", header))
+    assert {"compactor_score", "compactor_select", "compactor_compact", "compactor_compress"} <= declared
+    lib = ctypes.CDLL(B.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(lib, name), name
+    assert declared == set(B.EXPORTS)
+    assert B.version() >= 100
+
+
+def test_keep_count_matches_oracle():
+    for n in (0, 1, 2, 7, 100, 1024, 8192, 131072, 10 ** 6 + 3):
+        for r in (1e-9, 0.07, 0.2, 0.3, 0.32, 0.5, 0.999999, 1.0):
+            assert B.keep_count(n, r) == orc.keep_count(n, r), (n, r)
+    assert B.keep_count(100, 0.07) == 8 and B.keep_count(8192, 0.3) == 2458 and B.keep_count(131072, 0.32) == 41944
+
+
+def test_calibrated_ratio_matches_oracle():
+    for b in (-10.0, -4.0, -1.0, -1e-8, 0.0, 2.0):
+        for tau in (0.5, 0.9, 0.95, 1.0):
+            got = B.calibrated_ratio(2.0, b / 4, b / 2, tau)
+            assert abs(got - orc.calibrated_ratio(2.0, b / 4, b / 2, tau)) < 1e-12
+            assert abs(orc.calibration_curve(got, b) - tau) < 1e-7
+    with pytest.raises(B.CompactorError):
+        B.calibrated_ratio(1.0, 1.0, 0.0, 0.0)
+    with pytest.raises(B.CompactorError):
+        B.calibrated_ratio(1.0, 1.0, 0.0, 1.5)
+
+
+def test_make_sketch_matches_oracle_generator():
+    for seed, d, m in ((0, 128, 48), (12345, 128, 64), (7, 5, 3)):
+        got = B.make_sketch(seed, d, m).numpy()
+        want = orc.make_sketch(seed, d, m)
+        # both follow the same counter-based recipe; libm and numpy may differ in the last bit
+        np.testing.assert_allclose(got, want, rtol=3e-7, atol=1e-9)
+    z = B.make_sketch(1, 128, 48).numpy().astype(np.float64) * math.sqrt(48)
+    assert abs(z.mean()) < 0.05 and abs(z.std() - 1) < 0.05
+
+
+def test_workspace_bytes():
+    small = B.workspace_bytes(B.Shape(1, 2, 128, 48, [1024]))
+    big = B.workspace_bytes(B.Shape(64, 8, 128, 48, [131072]))
+    assert 0 < small < big < 4 << 30
+    assert small % 256 == 0
+    assert B.workspace_bytes(B.Shape(1, 2, 64, 48, [1024])) == 0          # d != 128
+    assert B.workspace_bytes(B.Shape(1, 2, 128, 65, [1024])) == 0         # m too large
+    assert B.workspace_bytes(B.Shape(1, 2, 128, 48, [1024, 0, 77])) > 0   # empty sequences are fine
+
+
+def _mat(ptr=1 << 20, sl=1 << 20, sh=1 << 17, st=128):
+    return B.CompactorMat(ptr, sl, sh, st)
+
+
+def _score(shape, k, phi=1 << 21, out=1 << 22, ws=1 << 23, ws_bytes=1 << 40):
+    return B.LIB.compactor_score(ctypes.byref(shape.c), k, ctypes.c_void_p(phi), None, 0.3, ctypes.c_void_p(out),
+                                 None, ctypes.c_void_p(ws), ws_bytes, None)
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    ok = B.Shape(1, 2, 128, 48, [1024])
+    assert _score(B.Shape(1, 2, 96, 48, [1024]), _mat()) == -2
+    assert _score(B.Shape(1, 2, 128, 0, [1024]), _mat()) == -2
+    assert _score(B.Shape(0, 2, 128, 48, [1024]), _mat()) == -1
+    assert _score(ok, _mat(ptr=0)) == -1
+    assert _score(ok, _mat(ptr=(1 << 20) + 8)) == -1                   # 16-byte alignment
+    assert _score(ok, _mat(st=120)) == -1                                # token stride below d
+    assert _score(ok, _mat(st=132)) == -1                                # not a multiple of 8 elements
+    assert _score(ok, _mat(), phi=0) == -1
+    assert _score(ok, _mat(), out=0) == -1
+    assert _score(ok, _mat(), ws=(1 << 23) + 64) == -1                   # workspace alignment
+    assert _score(ok, _mat(), ws_bytes=1024) == -3
+    bad = B.Shape(1, 2, 128, 48, [1024])
+    bad._cu[1] = -5
+    assert _score(bad, _mat()) == -1
+    # select / compact: keep counts must lie in [0, n]
+    keep = (ctypes.c_int32 * 1)(2000)
+    rc = B.LIB.compactor_select(ctypes.byref(ok.c), ctypes.c_void_p(1 << 22), keep, ctypes.c_void_p(1 << 24), None,
+                                ctypes.c_void_p(1 << 23), 1 << 20, None)
+    assert rc == -1
+    assert "workspace" in B.error_string(-3) and B.error_string(0) == "ok"

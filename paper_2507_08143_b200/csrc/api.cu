@@ -46,7 +46,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     p.total_tokens = s->cu_seqlens[s->batch];
     hp->units = s->layers * s->heads * s->batch;
 
-    // Gram block length: the longest (<= kMaxChunk) that still yields about eight CTAs per SM.
+    // Block length: the longest (<= kMaxChunk) that still yields about six CTAs per SM.
     int chunk = kMaxChunk;
     auto count_chunks = [&](int c) {
         long long t = 0;
@@ -56,7 +56,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
         }
         return t;
     };
-    while (chunk > kMinChunk && count_chunks(chunk) * s->layers * s->heads < 8LL * kSmCount) chunk >>= 1;
+    while (chunk > kMinChunk && count_chunks(chunk) * s->layers * s->heads < 6LL * kSmCount) chunk >>= 1;
     p.chunk = chunk;
     long long tc = count_chunks(chunk);
     if (tc > 0x7fffffffLL) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
@@ -72,7 +72,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     size_t off = 0;
     hp->off_tables = off;   off += align_up(sizeof(int) * 3 * nb1);
     hp->off_w = off;        off += align_up(sizeof(__nv_bfloat16) * w_elems_per_unit(p.mp) * hp->units);
-    hp->off_partials = off; off += align_up(sizeof(float) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
+    hp->off_partials = off; off += align_up(sizeof(double) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
     hp->off_scores = off;   off += align_up(sizeof(float) * (size_t)p.total_tokens * s->layers * s->heads);
     hp->total_bytes = off;
     return true;
@@ -134,7 +134,7 @@ struct Marks {
 int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn, float lambda,
                 float* scores, int32_t* status, char* ws, cudaStream_t stream, const Marks& mk = Marks()) {
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(ws + hp.off_w);
-    float* partials = reinterpret_cast<float*>(ws + hp.off_partials);
+    double* partials = reinterpret_cast<double*>(ws + hp.off_partials);
     if (status != nullptr) CK(cudaMemsetAsync(status, 0, sizeof(int32_t) * hp.units, stream));
     CK(mk.mark(0, stream));
     CK(launch_gram(hp.plan, k, partials, status, stream));
@@ -357,7 +357,7 @@ void replan_chunk(const compactor_shape* s, HostPlan* hp, int chunk) {
     p.chunk = chunk;
     p.total_chunks = cc[s->batch];
     hp->off_scores = hp->off_partials +
-                     align_up(sizeof(float) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
+                     align_up(sizeof(double) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
     hp->total_bytes = hp->off_scores + align_up(sizeof(float) * (size_t)p.total_tokens * s->layers * s->heads);
 }
 

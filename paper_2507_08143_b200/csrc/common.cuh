@@ -10,8 +10,9 @@ namespace compactor {
 
 constexpr int kD = 128;            // head dimension the kernels are written for
 constexpr int kMaxM = 64;          // largest sketch dimension
-constexpr int kMaxChunk = 4096;    // most tokens whose Gram matrix is summed in fp32 before the fp64 reduction
+constexpr int kMaxChunk = 32768;   // most tokens per block (one CTA of the two streaming kernels)
 constexpr int kMinChunk = 256;
+constexpr int kGramFlushTokens = 2048;   // most tokens whose Gram matrix is summed in fp32 before going to fp64
 constexpr int kGramElems = kD * kD;
 
 // Device-side view of one call: shapes plus the three prefix-sum tables that live at the start
@@ -20,7 +21,7 @@ struct Plan {
     int layers, heads, batch;
     int m;                 // sketch dimension
     int mp;                // m rounded up to a multiple of 16 (padded columns of W are zero)
-    int chunk;             // tokens per Gram partial (multiple of 128)
+    int chunk;             // tokens per block = per Gram partial (multiple of 128)
     int total_chunks;      // Gram partials per (layer, head): sum_b ceil(n_b / chunk)
     int total_tokens;      // per (layer, head)
     int total_keep;        // per (layer, head)
@@ -46,8 +47,8 @@ __device__ __forceinline__ int find_segment(const int* __restrict__ table, int n
 
 // Kernel launchers (each defined next to its kernel).  All enqueue on `stream` and return the
 // launch status.
-cudaError_t launch_gram(const Plan& p, const Mat& k, float* partials, int* status, cudaStream_t stream);
-cudaError_t launch_factor(const Plan& p, const Mat& k, const float* partials, const float* phi, __nv_bfloat16* w,
+cudaError_t launch_gram(const Plan& p, const Mat& k, double* partials, int* status, cudaStream_t stream);
+cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, __nv_bfloat16* w,
                           int* status, cudaStream_t stream);
 cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
                          cudaStream_t stream);

@@ -1,13 +1,15 @@
-// Gram pass: C_p = K_p^T K_p (128 x 128, fp32) for every block p of at most `chunk` tokens of
-// every unit.  Together with the fp64 projection G = Phi^T (sum_p C_p) Phi in the factor kernel
-// this is Algorithm 1, lines 2-3, (K Phi)^T (K Phi), evaluated from exact bf16 products.
+// Gram pass: C_p = K_p^T K_p (128 x 128) for every block p of at most `chunk` tokens of every
+// unit.  Together with the fp64 projection G = Phi^T (sum_p C_p) Phi in the factor kernel this is
+// Algorithm 1, lines 2-3, (K Phi)^T (K Phi), evaluated from exact bf16 products.
 //
-// One CTA per block.  A producer warp streams 128-token tiles of K through a ring of shared
-// memory stages with TMA (two 64-channel boxes per tile, 128-byte swizzle); one thread issues
-// tcgen05.mma with the same tile as both operands (token axis = contraction axis, so both are
-// MN-major) into a 128 x 128 fp32 accumulator in tensor memory; four warps drain it to global
-// memory at the end.  Two CTAs share an SM so that one's prologue/epilogue hides under the
-// other's stream.
+// One CTA per block, one CTA per SM.  A producer warp streams 128-token tiles of K through a
+// six-stage ring of shared memory with TMA (two 64-channel boxes per tile, 128-byte swizzle); one
+// thread issues tcgen05.mma with the same tile as both operands (the token axis is the
+// contraction axis, so both are MN-major) into one of two 128 x 128 fp32 accumulators in tensor
+// memory.  Every 2048 tokens the accumulator is handed to eight epilogue warps, which add it
+// into fp64 registers (64 columns of one row per thread) while the other accumulator fills; the
+// fp64 sums go to global memory once, at the end of the block.  So no fp32 sum is longer than
+// 2048 tokens, whatever the block length.
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -17,23 +19,26 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;                 // tokens per tile
-constexpr int kStages = 3;
+constexpr int kStages = 6;
 constexpr int kBoxBytes = kTile * 128;     // 64 channels x 128 tokens x 2 B
 constexpr int kTileBytes = 2 * kBoxBytes;
-constexpr int kThreads = 192;              // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
-constexpr uint32_t kTmemCols = 128;
+constexpr int kFlushTiles = kGramFlushTokens / kTile;
+constexpr int kEpilogueWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpilogueWarps;   // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
+constexpr uint32_t kTmemCols = 256;        // two accumulators
 
 struct __align__(1024) GramSmem {
     unsigned char tiles[kStages][kTileBytes];
     uint64_t full[kStages];
     uint64_t empty[kStages];
-    uint64_t acc_full;
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
     uint32_t tmem_base;
     int abort;
 };
 
-__global__ void __launch_bounds__(kThreads, 2)
-gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, float* __restrict__ partials,
+__global__ void __launch_bounds__(kThreads, 1)
+gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, double* __restrict__ partials,
             int* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
     GramSmem& s = *reinterpret_cast<GramSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
@@ -45,12 +50,13 @@ gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, float* __restrict_
     const int tok_end = min(tok_begin + p.chunk, p.cu_seqlens[b + 1]);
     const int n_tok = tok_end - tok_begin;
     const int n_tiles = (n_tok + kTile - 1) / kTile;
+    const int n_groups = (n_tiles + kFlushTiles - 1) / kFlushTiles;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
         prefetch_tensormap(&kmap);
         for (int i = 0; i < kStages; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
-        mbar_init(&s.acc_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&s.acc_full[i], 1); mbar_init(&s.acc_empty[i], kEpilogueWarps); }
         s.abort = 0;
         fence_barrier_init();
     }
@@ -77,7 +83,9 @@ gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, float* __restrict_
         bool ok = true;
         for (int t = 0; t < n_tiles && ok; ++t) {
             const int stage = t % kStages, round = t / kStages;
-            ok = mbar_wait(&s.full[stage], round & 1) && !*(volatile int*)&s.abort;
+            const int g = t / kFlushTiles, in_group = t % kFlushTiles, buf = g & 1;
+            if (in_group == 0 && g >= 2) ok = mbar_wait(&s.acc_empty[buf], ((g >> 1) - 1) & 1);
+            ok = ok && mbar_wait(&s.full[stage], round & 1) && !*(volatile int*)&s.abort;
             if (!ok) break;
             tc_fence_after_sync();
             const int valid = min(kTile, n_tok - t * kTile);
@@ -95,35 +103,51 @@ gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, float* __restrict_
             }
             if (lane == 0) {
                 const uint32_t base = smem_u32(s.tiles[stage]);
+                const uint32_t d_addr = tmem + buf * 128;
 #pragma unroll
                 for (int ks = 0; ks < kTile / 16; ++ks) {
                     const uint64_t desc = umma_desc_sw128(base + ks * 2048, kBoxBytes, 1024);
-                    umma_bf16(tmem, desc, desc, idesc, (t > 0) || (ks > 0));
+                    umma_bf16(d_addr, desc, desc, idesc, (in_group > 0) || (ks > 0));
                 }
                 umma_commit(&s.empty[stage]);
+                if (in_group == kFlushTiles - 1 || t == n_tiles - 1) umma_commit(&s.acc_full[buf]);
             }
             __syncwarp();
         }
-        if (!ok) s.abort = 1;
-        if (lane == 0) umma_commit(&s.acc_full);   // also releases the epilogue after an abort
+        if (!ok) {
+            s.abort = 1;
+            if (lane == 0) { mbar_arrive(&s.acc_full[0]); mbar_arrive(&s.acc_full[1]); }   // wake the epilogue
+        }
     } else {
-        const bool ok = mbar_wait(&s.acc_full, 0);
-        tc_fence_after_sync();
-        if (ok && !*(volatile int*)&s.abort) {
-            const int q = warp & 3;
-            const int row = q * 32 + lane;
-            float* out = partials + ((size_t)lh * p.total_chunks + chunk_id) * kGramElems + (size_t)row * kD;
+        const int q = warp & 3;                       // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;             // which 64 columns
+        const int row = q * 32 + lane;
+        double acc[64];
 #pragma unroll
-            for (int c0 = 0; c0 < kD; c0 += 32) {
+        for (int i = 0; i < 64; ++i) acc[i] = 0.0;
+        bool ok = true;
+        for (int g = 0; g < n_groups && ok; ++g) {
+            const int buf = g & 1;
+            ok = mbar_wait(&s.acc_full[buf], (g >> 1) & 1) && !*(volatile int*)&s.abort;
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t r[32];
-                tmem_ld_32x32b_x32(tmem + ((uint32_t)(q * 32) << 16) + c0, r);
+                tmem_ld_32x32b_x32(tmem + ((uint32_t)(q * 32) << 16) + buf * 128 + half * 64 + c0, r);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; i += 4)
-                    *reinterpret_cast<uint4*>(out + c0 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+                for (int i = 0; i < 32; ++i) acc[c0 + i] += (double)__uint_as_float(r[i]);
             }
-        } else if (!ok) {
-            s.abort = 1;
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&s.acc_empty[buf]);
+        }
+        if (!ok) s.abort = 1;
+        if (ok) {
+            double* out = partials + ((size_t)lh * p.total_chunks + chunk_id) * kGramElems + (size_t)row * kD + half * 64;
+#pragma unroll
+            for (int i = 0; i < 64; i += 2) *reinterpret_cast<double2*>(out + i) = make_double2(acc[i], acc[i + 1]);
         }
     }
     tc_fence_before_sync();
@@ -135,7 +159,7 @@ gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, float* __restrict_
 
 }  // namespace
 
-cudaError_t launch_gram(const Plan& p, const Mat& k, float* partials, int* status, cudaStream_t stream) {
+cudaError_t launch_gram(const Plan& p, const Mat& k, double* partials, int* status, cudaStream_t stream) {
     if (p.total_chunks == 0) return cudaSuccess;
     CUtensorMap kmap;
     if (!make_kv_tensor_map(&kmap, k.ptr, p.layers, p.heads, p.total_tokens, k.stride_layer, k.stride_head,

@@ -2,10 +2,11 @@
 // factor kernel, so that U~ = K^ V~ Sigma~^-1 is never stored.  W arrives as two bf16 terms
 // (hi + lo); both are multiplied with the bf16 keys on the tensor cores and summed in fp32.
 //
-// One CTA per block of tokens of one unit.  Warp 0 streams 128-token tiles of K (and W once)
-// with TMA; one thread of warp 1 issues tcgen05.mma (A = key tile, K-major; B = W^T, K-major;
-// D = 128 tokens x MP fp32 in tensor memory, double buffered); warps 2-5 read D back, square,
-// sum along the row and store one fp32 score per token.
+// One CTA per block of tokens of one unit, one CTA per SM.  Warp 0 streams 128-token tiles of K
+// (and W once) through a six-stage ring with TMA; one thread of warp 1 issues tcgen05.mma (A = key
+// tile, K-major; B = W^T, K-major; D = 128 tokens x MP fp32 in tensor memory, four accumulators
+// in rotation); warps 2-5 read D back, square, sum along the row and store one fp32 score per
+// token.
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -15,11 +16,12 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;
-constexpr int kStages = 3;
+constexpr int kStages = 6;
 constexpr int kBoxBytes = kTile * 128;
 constexpr int kTileBytes = 2 * kBoxBytes;
 constexpr int kThreads = 192;
-constexpr uint32_t kTmemCols = 128;       // two accumulators of up to 64 columns
+constexpr int kBufs = 4;                  // accumulators of up to 64 columns each
+constexpr uint32_t kTmemCols = 64 * kBufs;
 
 template <int MP>
 struct __align__(1024) ScoreSmem {
@@ -28,14 +30,14 @@ struct __align__(1024) ScoreSmem {
     uint64_t full[kStages];
     uint64_t empty[kStages];
     uint64_t w_full;
-    uint64_t d_full[2];
-    uint64_t d_empty[2];
+    uint64_t d_full[kBufs];
+    uint64_t d_empty[kBufs];
     uint32_t tmem_base;
     int abort;
 };
 
 template <int MP>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap,
              float* __restrict__ scores, int* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
@@ -57,7 +59,7 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
         prefetch_tensormap(&wmap);
         for (int i = 0; i < kStages; ++i) { mbar_init(&s.full[i], 1); mbar_init(&s.empty[i], 1); }
         mbar_init(&s.w_full, 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(&s.d_full[i], 1); mbar_init(&s.d_empty[i], 4); }
+        for (int i = 0; i < kBufs; ++i) { mbar_init(&s.d_full[i], 1); mbar_init(&s.d_empty[i], 4); }
         s.abort = 0;
         fence_barrier_init();
     }
@@ -90,7 +92,7 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
         bool ok = mbar_wait(&s.w_full, 0);
         for (int t = 0; t < n_tiles && ok; ++t) {
             const int stage = t % kStages, round = t / kStages;
-            const int buf = t & 1, use = t >> 1;
+            const int buf = t % kBufs, use = t / kBufs;
             ok = mbar_wait(&s.full[stage], round & 1);
             if (ok && use > 0) ok = mbar_wait(&s.d_empty[buf], (use - 1) & 1);
             ok = ok && !*(volatile int*)&s.abort;
@@ -115,13 +117,14 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
         }
         if (!ok) {
             s.abort = 1;
-            if (lane == 0) { mbar_arrive(&s.d_full[0]); mbar_arrive(&s.d_full[1]); }   // wake the epilogue
+            if (lane == 0)
+                for (int i = 0; i < kBufs; ++i) mbar_arrive(&s.d_full[i]);   // wake the epilogue
         }
     } else {
         const int q = warp & 3;
         float* out = scores + (size_t)lh * p.total_tokens + tok_begin;
         for (int t = 0; t < n_tiles; ++t) {
-            const int buf = t & 1, use = t >> 1;
+            const int buf = t % kBufs, use = t / kBufs;
             const bool ok = mbar_wait(&s.d_full[buf], use & 1);
             if (!ok) s.abort = 1;
             if (!ok || *(volatile int*)&s.abort) break;

@@ -119,15 +119,15 @@ def algorithmic_bytes(w, keep, mode):
     return per_lh * w.layers * w.heads
 
 
-def stage_bytes(w, keep, mode, chunk_tokens=2048):
+def stage_bytes(w, keep, mode, chunk_tokens=32768):
     """Minimal bytes of each kernel run on its own (per step)."""
     row = w.d * 2
     lh = w.layers * w.heads
     tok = sum(w.seqlens); kept = sum(keep)
     n_part = sum((n + chunk_tokens - 1) // chunk_tokens for n in w.seqlens)
     return {
-        "gram": lh * (tok * row + n_part * 65536),
-        "factor": lh * n_part * 65536,
+        "gram": lh * (tok * row + n_part * 131072),
+        "factor": lh * n_part * 131072,
         "score": lh * tok * (row + 4),
         "blend": 0,
         "select": lh * (tok * 4 + kept * 4),

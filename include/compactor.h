@@ -116,7 +116,7 @@ size_t compactor_workspace_bytes(const compactor_shape* shape);
  *   scores_out   device fp32 [layers][heads][total_tokens].
  * The small factorisation is a Cholesky factorisation of G = (K Phi)^T (K Phi) in fp64 - one of
  * the algebraically equal routes the paper allows (Section 3.2, Appendix C); Gram sums are fp32
- * per block of at most 4096 tokens and fp64 across blocks.
+ * within runs of 2048 tokens and fp64 beyond.
  */
 int compactor_score(const compactor_shape* shape, compactor_mat k_score, const float* phi,
                     const float* attn_scores, float lambda, float* scores_out,
@@ -177,9 +177,9 @@ int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_sc
  * no workspace argument: the scratch is a fixed array of compactor_builtin_scratch_bytes()
  * (32 MiB) inside the library, resident on every device the process uses from the first use of
  * the library on that device until the process exits.  The call allocates and frees nothing.
- *   - Size limit: the scratch must hold 12*(batch+1) bytes of tables, 512*ceil(m/16)*16 bytes per
- *     unit and 64 KiB per Gram block (blocks are lengthened up to 4096 tokens to make it fit,
- *     i.e. about 16 bytes per token per (layer, head)).  A larger problem is refused with
+ *   - Size limit: the scratch must hold 12*(batch+1) bytes of tables, about 160 KiB per unit
+ *     (at m = 48) and 128 KiB per Gram block (blocks are lengthened up to 32768 tokens to make it
+ *     fit, i.e. down to 4 bytes per token per (layer, head)).  A larger problem is refused with
  *     COMPACTOR_E_TOO_LARGE before anything is enqueued; split it by layers or use
  *     compactor_score.
  *   - The first call on each device looks up the array's device address; make that first call

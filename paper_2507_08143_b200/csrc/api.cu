@@ -20,7 +20,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 struct HostPlan {
     Plan plan;
     std::vector<int> tables;       // cu_seqlens | cu_keep | cu_chunks, each batch+1
-    size_t off_tables, off_w, off_partials, off_scores, total_bytes;
+    size_t off_tables, off_w, off_gpart, off_partials, off_scores, total_bytes;
     int units;
 };
 
@@ -72,6 +72,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     size_t off = 0;
     hp->off_tables = off;   off += align_up(sizeof(int) * 3 * nb1);
     hp->off_w = off;        off += align_up(sizeof(__nv_bfloat16) * w_elems_per_unit(p.mp) * hp->units);
+    hp->off_gpart = off;    off += align_up(sizeof(double) * kFactorSlices * p.mp * p.mp * hp->units);
     hp->off_partials = off; off += align_up(sizeof(double) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
     hp->off_scores = off;   off += align_up(sizeof(float) * (size_t)p.total_tokens * s->layers * s->heads);
     hp->total_bytes = off;
@@ -139,7 +140,7 @@ int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn,
     CK(mk.mark(0, stream));
     CK(launch_gram(hp.plan, k, partials, status, stream));
     CK(mk.mark(1, stream));
-    CK(launch_factor(hp.plan, k, partials, phi, w, status, stream));
+    CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, status, stream));
     CK(mk.mark(2, stream));
     CK(launch_score(hp.plan, k, w, scores, status, stream));
     CK(mk.mark(3, stream));

@@ -1,7 +1,16 @@
 // Per-unit top-k (Section 3.4: keep the ceil(r N) highest-scoring tokens of a head) and the
-// blend of Eq. 6.  Selection is an exact radix select on the order-preserving integer image of
-// the fp32 scores (three passes: 11 + 11 + 10 bits) followed by one ordered compaction pass;
-// equal scores go to the lower index and indices come out ascending.
+// blend of Eq. 6.  Selection is exact: it finds the key of the kk-th largest score (keys are the
+// order-preserving integer image of the fp32 scores), then one ordered pass emits the indices of
+// all larger scores plus the lowest-indexed ties, ascending.
+//
+// Finding the threshold.  Leverage scores of one head are spread over a narrow range, so a radix
+// histogram on the leading float bits would pile everything into a dozen bins.  Instead the range
+// is estimated from the first few thousand scores, a 2048-bin histogram linear in the score value
+// is taken over all of them (values outside the estimate fall into the end bins; the binning is
+// monotone, so it orders exactly), the bin holding the kk-th largest is found, its members are
+// collected in shared memory and the exact key is found there by a three-pass radix select.
+// Inputs that defeat this (non-finite values, a constant score, more members than fit) take the
+// same three-pass radix select over global memory.
 #include "common.cuh"
 
 namespace compactor {
@@ -10,6 +19,9 @@ namespace {
 constexpr int kThreads = 1024;
 constexpr int kWarps = kThreads / 32;
 constexpr int kBins = 2048;
+constexpr int kSample = 4096;          // scores used to estimate the value range
+constexpr int kCand = 8192;            // capacity of the candidate list
+constexpr int kSub = 8;                // 1024-element sub-blocks per iteration of the ordered pass
 
 // Monotone map float -> uint32: larger float <=> larger key; -0 and +0 share a key (adding +0
 // turns -0 into +0) and a NaN with the sign bit clear ranks highest.
@@ -20,14 +32,20 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 
 struct SelectSmem {
     int hist[kBins];
+    uint32_t cand[kCand];
+    int cnt[2][kSub][kWarps];      // per-warp packed counts of the ordered pass, double buffered
+    int row_total[2][kSub];
     int warp_sums[kWarps];
-    int warp_sums2[kWarps];
+    float red[2][kWarps];
     int bin;          // chosen bin of the current pass
     int remaining;    // how many elements are still to be taken from the chosen bin
+    int n_cand;
+    float lo, scale;
+    int fallback;
 };
 
 // Finds, scanning from the highest bin down, the bin where the running count reaches `want`.
-// Returns (via smem) that bin and want - (count in higher bins).
+// Leaves that bin and want - (count in higher bins) in shared memory.
 __device__ void pick_bin(SelectSmem& s, int nbins, int want) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // thread t owns bins nbins-1-2t and nbins-2-2t (descending order)
@@ -62,9 +80,60 @@ __device__ void pick_bin(SelectSmem& s, int nbins, int want) {
     __syncthreads();
 }
 
+// Calls f(value) for every score of the unit: unaligned head, 16-byte body with four vectors in
+// flight per thread, tail.  The visiting order is unspecified.
+template <class F>
+__device__ __forceinline__ void for_each_score(const float* __restrict__ sc, int n, F f) {
+    const int tid = threadIdx.x;
+    const int head = min(n, (int)((4 - ((reinterpret_cast<uintptr_t>(sc) >> 2) & 3)) & 3));
+    const int n_vec = (n - head) >> 2;
+    const float4* body = reinterpret_cast<const float4*>(sc + head);
+    if (tid < head) f(sc[tid]);
+    for (int v0 = 0; v0 < n_vec; v0 += 4 * kThreads) {
+        float4 q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int vi = v0 + u * kThreads + tid;
+            q[u] = vi < n_vec ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (v0 + u * kThreads + tid < n_vec) { f(q[u].x); f(q[u].y); f(q[u].z); f(q[u].w); }
+    }
+    for (int i = head + 4 * n_vec + tid; i < n; i += kThreads) f(sc[i]);
+}
+
+// Three-pass radix select (11 + 11 + 10 bits) of the `want`-th largest key among the keys produced
+// by `visit(tally)`; returns the key and, through *ties, how many keys equal to it are wanted.
+template <class Visit>
+__device__ uint32_t radix_select(SelectSmem& s, int want, int* ties, Visit visit) {
+    const int tid = threadIdx.x;
+    uint32_t prefix = 0;
+    const int shifts[3] = {21, 10, 0};
+    const int widths[3] = {11, 11, 10};
+    for (int pass = 0; pass < 3; ++pass) {
+        const int shift = shifts[pass], nb = 1 << widths[pass];
+        for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
+        __syncthreads();
+        const int hi_shift = shift + widths[pass];
+        const uint32_t want_hi = prefix >> hi_shift;
+        visit([&](uint32_t key) {
+            if (pass == 0 || (key >> hi_shift) == want_hi) atomicAdd(&s.hist[(key >> shift) & (nb - 1)], 1);
+        });
+        __syncthreads();
+        pick_bin(s, nb, want);
+        prefix |= (uint32_t)s.bin << shift;
+        want = s.remaining;
+        __syncthreads();
+    }
+    *ties = want;
+    return prefix;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_out) {
-    __shared__ SelectSmem s;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
     const int unit = blockIdx.x;
     const int b = unit % p.batch, lh = unit / p.batch;
     const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
@@ -79,83 +148,135 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
         return;
     }
 
-    // --- radix select of the kk-th largest key -------------------------------------------
-    uint32_t prefix = 0;      // high bits fixed so far
-    int want = kk;
-    const int shifts[3] = {21, 10, 0};
-    const int widths[3] = {11, 11, 10};
-    for (int pass = 0; pass < 3; ++pass) {
-        const int shift = shifts[pass], nb = 1 << widths[pass];
-        for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
-        __syncthreads();
-        const int hi_shift = shift + widths[pass];     // bits above the current digit
-        for (int i = tid; i < n; i += kThreads) {
-            uint32_t key = order_key(sc[i]);
-            bool match = (pass == 0) || ((key >> hi_shift) == (prefix >> hi_shift));
-            if (match) atomicAdd(&s.hist[(key >> shift) & (nb - 1)], 1);
+    // ---- value range from a sample ------------------------------------------------------------
+    {
+        float lo = INFINITY, hi = -INFINITY;
+        bool finite = true;
+        float smp[kSample / kThreads];
+#pragma unroll
+        for (int u = 0; u < kSample / kThreads; ++u) {
+            const int i = u * kThreads + tid;
+            smp[u] = sc[i < n ? i : 0];
         }
+#pragma unroll
+        for (int u = 0; u < kSample / kThreads; ++u) {
+            finite = finite && isfinite(smp[u]);
+            lo = fminf(lo, smp[u]); hi = fmaxf(hi, smp[u]);
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+        }
+        const int all_finite = __syncthreads_and(finite ? 1 : 0);
+        if (lane == 0) { s.red[0][warp] = lo; s.red[1][warp] = hi; }
         __syncthreads();
-        pick_bin(s, nb, want);
-        prefix |= (uint32_t)s.bin << shift;
-        want = s.remaining;
+        if (tid == 0) {
+            for (int w = 1; w < kWarps; ++w) { lo = fminf(lo, s.red[0][w]); hi = fmaxf(hi, s.red[1][w]); }
+            const float width = hi - lo;
+            const float scale = (float)(kBins - 2) / width;              // sampled range -> bins 1 .. kBins-2
+            s.fallback = !(all_finite && width > 0.f && isfinite(width) && isfinite(scale));
+            s.lo = lo;
+            s.scale = s.fallback ? 0.f : scale;
+            s.n_cand = 0;
+        }
         __syncthreads();
     }
-    const uint32_t thr = prefix;   // key of the kk-th largest element
-    const int ties = want;         // how many elements equal to it are kept (lowest indices first)
 
-    // --- ordered compaction -----------------------------------------------------------------
-    int base_gt = 0, base_eq = 0;          // counts over the elements before this block-iteration
-    for (int start = 0; start < n; start += kThreads * 4) {
-        const int i0 = start + tid * 4;
-        uint32_t keys[4];
-        int gt = 0, eq = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            int i = i0 + e;
-            keys[e] = (i < n) ? order_key(sc[i]) : 0u;
-            if (i < n) { gt += keys[e] > thr; eq += keys[e] == thr; }
-        }
-        int packed = gt | (eq << 16);
-        int incl = packed;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            int v = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += v;
-        }
-        if (lane == 31) s.warp_sums2[warp] = incl;
+    uint32_t thr = 0;
+    int ties = 0;
+    bool found = false;
+    if (!s.fallback) {
+        const float lo = s.lo, scale = s.scale;
+        // monotone in v: subtraction, multiplication by a positive constant, clamping and truncation all are
+        auto bin_of = [&](float v) {
+            const float x = fminf(fmaxf((v - lo) * scale + 1.0f, 0.0f), (float)(kBins - 1));
+            return (int)x;
+        };
+        for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
         __syncthreads();
-        if (warp == 0) {
-            int v = s.warp_sums2[lane];
-            int scn = v;
+        int nonfinite = 0;
+        for_each_score(sc, n, [&](float v) {
+            if (!isfinite(v)) nonfinite = 1;
+            atomicAdd(&s.hist[bin_of(v)], 1);
+        });
+        const int any_nonfinite = __syncthreads_or(nonfinite);
+        pick_bin(s, kBins, kk);
+        const int tbin = s.bin, want = s.remaining;
+        const int members = s.hist[tbin];
+        __syncthreads();
+        if (!any_nonfinite && members <= kCand) {
+            for_each_score(sc, n, [&](float v) {
+                if (bin_of(v) == tbin) s.cand[atomicAdd(&s.n_cand, 1)] = order_key(v);
+            });
+            __syncthreads();
+            const int nc = s.n_cand;
+            thr = radix_select(s, want, &ties, [&](auto tally) {
+                for (int i = tid; i < nc; i += kThreads) tally(s.cand[i]);
+            });
+            found = true;
+        }
+    }
+    if (!found)
+        thr = radix_select(s, kk, &ties, [&](auto tally) {
+            for_each_score(sc, n, [&](float v) { tally(order_key(v)); });
+        });
+
+    // ---- ordered pass: positions from ballots and a scan of per-warp counts ---------------------
+    int base_gt = 0, base_eq = 0;          // counts over the elements before this iteration
+    const uint32_t lt_mask = (1u << lane) - 1u;
+    int it = 0;
+    float nxt[kSub];                       // scores of the next iteration, loaded one iteration ahead
+#pragma unroll
+    for (int u = 0; u < kSub; ++u) {
+        const int i = u * kThreads + tid;
+        nxt[u] = (i < n) ? sc[i] : 0.f;
+    }
+    for (int start = 0; start < n; start += kThreads * kSub, ++it) {
+        const int buf = it & 1;
+        uint32_t keys[kSub], bg[kSub], be[kSub];
+#pragma unroll
+        for (int u = 0; u < kSub; ++u) keys[u] = order_key(nxt[u]);
+#pragma unroll
+        for (int u = 0; u < kSub; ++u) {
+            const int i = start + kThreads * kSub + u * kThreads + tid;
+            nxt[u] = (i < n) ? sc[i] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < kSub; ++u) {
+            const int i = start + u * kThreads + tid;
+            bg[u] = __ballot_sync(0xffffffffu, i < n && keys[u] > thr);
+            be[u] = __ballot_sync(0xffffffffu, i < n && keys[u] == thr);
+            if (lane == 0) s.cnt[buf][u][warp] = __popc(bg[u]) | (__popc(be[u]) << 16);
+        }
+        __syncthreads();
+        if (warp < kSub) {
+            const int v = s.cnt[buf][warp][lane];
+            int incl = v;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                int u = __shfl_up_sync(0xffffffffu, scn, off);
-                if (lane >= off) scn += u;
+                int t = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= off) incl += t;
             }
-            s.warp_sums[lane] = scn - v;
-            if (lane == 31) s.bin = scn;      // block total (packed)
+            s.cnt[buf][warp][lane] = incl - v;
+            if (lane == 31) s.row_total[buf][warp] = incl;
         }
         __syncthreads();
-        int excl = s.warp_sums[warp] + incl - packed;
-        int gt_before = base_gt + (excl & 0xffff);
-        int eq_before = base_eq + (excl >> 16);
-        int total = s.bin;
+        int run = 0;                        // packed count of the sub-blocks before u in this iteration
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            int i = i0 + e;
+        for (int u = 0; u < kSub; ++u) {
+            const int i = start + u * kThreads + tid;
+            const int before = run + s.cnt[buf][u][warp];
+            const int gt_before = base_gt + (before & 0xffff) + __popc(bg[u] & lt_mask);
+            const int eq_before = base_eq + (before >> 16) + __popc(be[u] & lt_mask);
             if (i < n) {
-                if (keys[e] > thr) {
-                    out[gt_before + min(eq_before, ties)] = i;
-                    ++gt_before;
-                } else if (keys[e] == thr) {
-                    if (eq_before < ties) out[gt_before + eq_before] = i;
-                    ++eq_before;
-                }
+                if (keys[u] > thr) out[gt_before + min(eq_before, ties)] = i;
+                else if (keys[u] == thr && eq_before < ties) out[gt_before + eq_before] = i;
             }
+            run += s.row_total[buf][u];
         }
-        base_gt += total & 0xffff;
-        base_eq += total >> 16;
-        __syncthreads();
+        base_gt += run & 0xffff;
+        base_eq += run >> 16;
     }
 }
 
@@ -216,7 +337,10 @@ blend_kernel(Plan p, const float* __restrict__ attn, float lambda, float* __rest
 cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStream_t stream) {
     const int units = p.layers * p.heads * p.batch;
     if (units == 0 || p.total_keep == 0) return cudaSuccess;
-    select_kernel<<<units, kThreads, 0, stream>>>(p, scores, idx);
+    const int smem = (int)sizeof(SelectSmem);
+    cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    select_kernel<<<units, kThreads, smem, stream>>>(p, scores, idx);
     return cudaGetLastError();
 }
 

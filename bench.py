@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-units", type=int, default=16, help="units in the CPU-baseline sample")
+    ap.add_argument("--fig1", action="store_true",
+                    help="context-length sweep of the paper's Fig. 1 setting (one layer, 8 KV heads, batch 1)")
     return ap.parse_args()
 
 
@@ -206,10 +208,61 @@ def cpu_baseline(args, w, keep, phi):
                       f"{w.layers}x{w.heads} units per token"}
 
 
+# The paper's Fig. 1 (one layer of Llama-3.1-8B, batch 1, NVIDIA H100 80GB, median wall-clock ms) for the
+# leverage-score-only curve, as context beside our numbers for the same shape.
+FIG1_PAPER_MS_H100 = {256: 1.345554, 512: 1.312034, 1024: 1.287826, 2048: 1.276906, 4096: 1.274009,
+                      8192: 1.276523, 16384: 1.301756, 32768: 1.428951, 65536: 1.588616, 131072: 1.924723,
+                      262144: 2.654723, 524288: 4.030933, 1048576: 6.812491}
+
+
+def run_fig1(args):
+    """Median time of compactor_score, and of the whole compactor_compress at 30 % retention, on
+    8 KV heads x n tokens, for the context lengths of the paper's Fig. 1."""
+    import torch
+    from paper_2507_08143_b200 import binding as B, inputs
+    torch.cuda.set_device(0)
+    rows = []
+    for n in sorted(FIG1_PAPER_MS_H100):
+        w = inputs.Workload(f"fig1-n{n}", 1, 8, 128, [n], [0.3], p=0.7, n_out=4, theta=5e5, seed=100)
+        _, kr, v = inputs.make_tensors(w, device="cuda", want_pre=False)
+        shape = B.Shape(1, 8, 128, 48, [n])
+        keep = [B.keep_count(n, 0.3)]
+        phi = inputs.make_sketch_matrix(128, 48, 0).cuda()
+        scores = torch.empty(1, 8, n, dtype=torch.float32, device="cuda")
+        idx = torch.empty(1, 8, keep[0], dtype=torch.int32, device="cuda")
+        ko = torch.empty(1, 8, keep[0], 128, dtype=torch.bfloat16, device="cuda"); vo = torch.empty_like(ko)
+        ws = B.alloc_workspace(shape)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than L2
+
+        def timed(fn, iters):
+            out = []
+            for _ in range(3):
+                fn()
+            for _ in range(iters):
+                flush.zero_()                                                  # start every call L2-cold
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+                out.append(e0.elapsed_time(e1))
+            return statistics.median(out)
+
+        iters = max(5, args.steps)
+        t_score = timed(lambda: B.score(shape, kr, phi, scores, ws), iters)
+        t_full = timed(lambda: B.compress(shape, kr, kr, v, phi, keep, idx, ko, vo, ws, scores_out=scores), iters)
+        rows.append({"n": n, "score_ms": round(t_score, 4), "compress_ms": round(t_full, 4),
+                     "paper_h100_score_ms": FIG1_PAPER_MS_H100[n]})
+        del kr, v, scores, idx, ko, vo, ws, flush
+        torch.cuda.empty_cache()
+    print(json.dumps({"fig1": rows, "shape": "1 layer x 8 KV heads, d=128, m=48, batch 1, bf16, keep 30 %",
+                      "timing": "median of CUDA-event times, L2 flushed before every call"}))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.fig1:
+        run_fig1(args)
         return
 
     import torch

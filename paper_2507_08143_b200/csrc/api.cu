@@ -46,8 +46,10 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     p.total_tokens = s->cu_seqlens[s->batch];
     hp->units = s->layers * s->heads * s->batch;
 
-    // Block length: the longest (<= kMaxChunk) that still yields about six CTAs per SM.
-    int chunk = kMaxChunk;
+    // Block length (tokens per CTA of the two sweeps, one fp64 Gram partial per block): the power
+    // of two times 256 that minimises a small cost model - waves of CTAs over the SMs, a fixed
+    // set-up cost per CTA, the block's bytes at one SM's share of the bandwidth, and the traffic of
+    // the 128 KiB partial that every block writes and the projection reads back.
     auto count_chunks = [&](int c) {
         long long t = 0;
         for (int b = 0; b < s->batch; ++b) {
@@ -56,7 +58,16 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
         }
         return t;
     };
-    while (chunk > kMinChunk && count_chunks(chunk) * s->layers * s->heads < 6LL * kSmCount) chunk >>= 1;
+    int chunk = kMaxChunk;
+    double best = 1e300;
+    for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
+        const double ctas = (double)count_chunks(c) * s->layers * s->heads;
+        const double waves = ceil(ctas / kSmCount);
+        const double per_cta_us = 4.0 + c * 256.0 / 44e3;             // 44 GB/s = 44e3 B/us per SM
+        const double partial_us = ctas * 2.0 * 131072.0 / 6.4e6;      // written once, read once at 6.4 TB/s
+        const double cost = waves * per_cta_us + partial_us;
+        if (cost < best * 0.999) { best = cost; chunk = c; }
+    }
     p.chunk = chunk;
     long long tc = count_chunks(chunk);
     if (tc > 0x7fffffffLL) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }

@@ -12,7 +12,7 @@ constexpr int kD = 128;            // head dimension the kernels are written for
 constexpr int kMaxM = 64;          // largest sketch dimension
 constexpr int kMaxChunk = 32768;   // most tokens per block (one CTA of the two streaming kernels)
 constexpr int kMinChunk = 256;
-constexpr int kGramFlushTokens = 2048;   // most tokens whose Gram matrix is summed in fp32 before going to fp64
+constexpr int kGramFlushTokens = 512;    // most tokens whose Gram matrix is summed in fp32 (tensor-core accumulators) before going to fp64
 constexpr int kGramElems = kD * kD;
 constexpr int kFactorSlices = 8;   // CTAs per unit that share the fp64 projection of the Gram matrix
 

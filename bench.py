@@ -75,7 +75,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except Exception:
@@ -198,14 +198,17 @@ def cpu_baseline(args, w, keep, phi):
                      w.seqlens[b]))
     phi_np = phi.numpy()
     t0 = time.perf_counter()
-    for ks, kr, v, kk, n in data:
-        orc.compress_unit(ks, kr, v, phi_np, kk)
+    head_tokens, passes = 0, 0
+    while time.perf_counter() - t0 < 12.0:                 # about 12 s of CPU work
+        for ks, kr, v, kk, n in data:
+            orc.compress_unit(ks, kr, v, phi_np, kk)
+            head_tokens += n
+        passes += 1
     dt = time.perf_counter() - t0
-    head_tokens = sum(d[4] for d in data)
     value = (head_tokens / dt) / (w.layers * w.heads)
     return {"value": value, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
-            "sample": f"{sample} units of {w.name} ({head_tokens} head-tokens, {dt:.1f} s), scaled to "
-                      f"{w.layers}x{w.heads} units per token"}
+            "sample": f"{sample} distinct units of {w.name} x {passes} passes ({head_tokens} head-tokens, {dt:.1f} s), "
+                      f"scaled to {w.layers}x{w.heads} units per token"}
 
 
 # The paper's Fig. 1 (one layer of Llama-3.1-8B, batch 1, NVIDIA H100 80GB, median wall-clock ms) for the
@@ -383,8 +386,8 @@ def e2e(args, B, w, shape, keep, phi_d, k_score, kr, v, dist, world):
     through pinned host buffers (host->device copy of the group's K and V, compress, device->host
     copy of indices and compressed K/V), every step."""
     import torch
-    group = min(8, w.layers)
-    n_groups = (w.layers + group - 1) // group
+    group = max(g for g in range(1, 9) if w.layers % g == 0)      # layers per group: a divisor, at most 8
+    n_groups = w.layers // group
     g_shape = B.Shape(group, w.heads, w.d, w.m, w.seqlens)
     total_keep = sum(keep)
     T = w.total_tokens

@@ -4,7 +4,8 @@
 //   project_kernel   eight CTAs per unit, each owning 16 rows of C = sum of the unit's Gram
 //                    partials: T_r = C[rows,:] Phi and the partial projection
 //                    G_r = Phi[rows,:]^T T_r, so that G = Phi^T C Phi = sum_r G_r.  This is where
-//                    the fp64 FMAs are (1.1 M per unit), spread over the whole device.
+//                    the fp64 FMAs are (1.1 M per unit); they run as fp64 mma.m8n8k4, spread over
+//                    the whole device.
 //   cholesky_kernel  one small CTA per unit (four fit on an SM, so all units of a large batch are
 //                    resident at once): G = sum_r G_r, G = L L^T in one warp (left-looking,
 //                    reciprocal square roots), then W = Phi L^-T with one thread per row of Phi
@@ -12,7 +13,7 @@
 //                    row k_i is then || k_i W ||^2 (Algorithm 1, lines 5-6).
 //
 // Rank handling: a pivot not larger than 2^-20 of its original diagonal entry (the fp32 noise
-// floor of the 2048-token Gram sums) is treated as a direction of the null space and dropped;
+// floor of the fp32 Gram runs) is treated as a direction of the null space and dropped;
 // with the remaining pivot set P, W = Phi[:, P] L_PP^-T, which equals the pseudo-inverse reading
 // o_i = k^_i G^+ k^_i^T whenever k^_i lies in the range of G.
 #include "common.cuh"
@@ -33,125 +34,164 @@ constexpr int kProjThreads = 256;
 
 template <int MP>
 struct ProjectSmem {
-    double phi[kD * MP];           // Phi widened, [channel][column]
-    double c[kD * kRows];          // C[k][row0 + i] at [k * kRows + i]  (C is symmetric)
-    double t[kRows * MP];          // T_r
+    static constexpr int kLd = MP + 8;     // row stride (doubles): four consecutive rows of 8 land in distinct banks
+    double phi[kD * kLd];                  // Phi widened, [channel][column]
+    double c[kD * kRows];                  // C[k][row0 + i] at [k * kRows + i]  (C is symmetric)
+    double t[kRows * kLd];                 // T_r
     double keys[kStageTokens * kD];
 };
 
+// Persistent: each CTA loads Phi once and then walks (unit, slice) items with a grid stride; the
+// global loads of the next item's partials are in flight while the current item is multiplied.
 template <int MP>
 __global__ void __launch_bounds__(kProjThreads)
 project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const float* __restrict__ phi,
-               double* __restrict__ g_partials) {
+               double* __restrict__ g_partials, int n_items) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    ProjectSmem<MP>& s = *reinterpret_cast<ProjectSmem<MP>*>(smem_raw);
-    const int unit = blockIdx.x, slice = blockIdx.y;
-    const int b = unit % p.batch, lh = unit / p.batch;
+    using Smem = ProjectSmem<MP>;
+    Smem& s = *reinterpret_cast<Smem*>(smem_raw);
+    constexpr int LD = Smem::kLd;
+    constexpr int kPer = kD * kRows / kProjThreads;     // 8 elements of the C slice per thread: e = tid + 256 q
+    constexpr int kInFlight = 4;                        // partials loaded ahead per item
     const int m = p.m, tid = threadIdx.x;
-    const int row0 = slice * kRows;
-    const int chunk_begin = p.cu_chunks[b], n_part = p.cu_chunks[b + 1] - chunk_begin;
-    const double* part = partials + ((size_t)lh * p.total_chunks + chunk_begin) * kGramElems;
-    const int n_tok = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+    const int warp = tid >> 5, lane = tid & 31;
+    const int fr = lane >> 2, fk = lane & 3;            // fragment coordinates: A[fr][fk], B[fk][fr], C[fr][2 fk, 2 fk + 1]
+    constexpr int kNT = MP / 8;                         // 8-column tiles
 
-    for (int i = tid; i < kD * MP; i += kProjThreads) {
-        int row = i / MP, col = i % MP;
-        s.phi[i] = (col < m) ? (double)phi[row * m + col] : 0.0;
+    {   // Phi, widened; all loads of a thread are issued before the first is used
+        constexpr int kPerThread = kD * MP / kProjThreads;
+        float v[kPerThread];
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+            const int i = tid + q * kProjThreads, row = i / MP, col = i % MP;
+            v[q] = (col < m) ? __ldg(phi + row * m + col) : 0.f;
+        }
+#pragma unroll
+        for (int q = 0; q < kPerThread; ++q) {
+            const int i = tid + q * kProjThreads;
+            s.phi[(i / MP) * LD + (i % MP)] = (double)v[q];
+        }
     }
 
-    // ---- the CTA's 16 columns of C (= 16 rows, by symmetry), summed over the partials ----------
-    {
-        constexpr int kPer = kD * kRows / kProjThreads;     // 8 elements per thread: e = tid + 256 q
-        double acc[kPer];
+    // Item bookkeeping and the look-ahead loads.
+    struct Item { int unit, slice, b, lh, n_part, n_tok; const double* part; };
+    auto decode = [&](int item) {
+        Item it;
+        it.unit = item / kSlices; it.slice = item % kSlices;
+        it.b = it.unit % p.batch; it.lh = it.unit / p.batch;
+        const int chunk_begin = p.cu_chunks[it.b];
+        it.n_part = p.cu_chunks[it.b + 1] - chunk_begin;
+        it.n_tok = p.cu_seqlens[it.b + 1] - p.cu_seqlens[it.b];
+        it.part = partials + ((size_t)it.lh * p.total_chunks + chunk_begin) * kGramElems;
+        return it;
+    };
+    double pre[kInFlight][kPer];
+    auto prefetch = [&](const Item& it) {
 #pragma unroll
-        for (int q = 0; q < kPer; ++q) acc[q] = 0.0;
-        if (n_tok > kExactGramTokens) {
-            int pp = 0;
-            for (; pp + 2 <= n_part; pp += 2) {
-                double v[2][kPer];
+        for (int u = 0; u < kInFlight; ++u)
 #pragma unroll
-                for (int u = 0; u < 2; ++u)
+            for (int q = 0; q < kPer; ++q) {
+                const int e = tid + q * kProjThreads;
+                pre[u][q] = (u < it.n_part && it.n_tok > kExactGramTokens)
+                                ? __ldcs(it.part + (size_t)u * kGramElems + (e / kRows) * kD + it.slice * kRows + (e % kRows))
+                                : 0.0;
+            }
+    };
+
+    int item = blockIdx.x;
+    Item cur;
+    if (item < n_items) { cur = decode(item); prefetch(cur); }
+    for (; item < n_items; item += gridDim.x) {
+        const int row0 = cur.slice * kRows;
+        // ---- the item's 16 columns of C (= 16 rows, by symmetry), summed over the partials ------
+        {
+            double acc[kPer];
+#pragma unroll
+            for (int q = 0; q < kPer; ++q) {
+                acc[q] = 0.0;
+#pragma unroll
+                for (int u = 0; u < kInFlight; ++u) acc[q] += pre[u][q];
+            }
+            if (cur.n_tok > kExactGramTokens) {
+                for (int pp = kInFlight; pp < cur.n_part; ++pp)           // more partials than the look-ahead holds
 #pragma unroll
                     for (int q = 0; q < kPer; ++q) {
                         const int e = tid + q * kProjThreads;
-                        v[u][q] = __ldcs(part + (size_t)(pp + u) * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
+                        acc[q] += __ldcs(cur.part + (size_t)pp * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
                     }
+            } else {
+                // short sequence: fp64 Gram straight from the keys
+                const int layer = cur.lh / p.heads, head = cur.lh % p.heads;
+                const __nv_bfloat16* kbase = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
+                                             (long long)p.cu_seqlens[cur.b] * kmat.stride_token;
+                for (int t0 = 0; t0 < cur.n_tok; t0 += kStageTokens) {
+                    const int nt = min(kStageTokens, cur.n_tok - t0);
+                    __syncthreads();
+                    for (int i = tid; i < nt * kD; i += kProjThreads)
+                        s.keys[i] = (double)__bfloat162float(kbase[(long long)(t0 + i / kD) * kmat.stride_token + (i % kD)]);
+                    __syncthreads();
+                    for (int t = 0; t < nt; ++t) {
+                        const double* krow = s.keys + t * kD;
 #pragma unroll
-                for (int q = 0; q < kPer; ++q) acc[q] += v[0][q] + v[1][q];
-            }
-            if (pp < n_part) {
-#pragma unroll
-                for (int q = 0; q < kPer; ++q) {
-                    const int e = tid + q * kProjThreads;
-                    acc[q] += __ldcs(part + (size_t)pp * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
-                }
-            }
-        } else {
-            const int layer = lh / p.heads, head = lh % p.heads;
-            const __nv_bfloat16* kbase = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
-                                         (long long)p.cu_seqlens[b] * kmat.stride_token;
-            for (int t0 = 0; t0 < n_tok; t0 += kStageTokens) {
-                const int nt = min(kStageTokens, n_tok - t0);
-                __syncthreads();
-                for (int i = tid; i < nt * kD; i += kProjThreads)
-                    s.keys[i] = (double)__bfloat162float(kbase[(long long)(t0 + i / kD) * kmat.stride_token + (i % kD)]);
-                __syncthreads();
-                for (int t = 0; t < nt; ++t) {
-                    const double* krow = s.keys + t * kD;
-#pragma unroll
-                    for (int q = 0; q < kPer; ++q) {
-                        const int e = tid + q * kProjThreads;
-                        acc[q] = fma(krow[e / kRows], krow[row0 + (e % kRows)], acc[q]);
+                        for (int q = 0; q < kPer; ++q) {
+                            const int e = tid + q * kProjThreads;
+                            acc[q] = fma(krow[e / kRows], krow[row0 + (e % kRows)], acc[q]);
+                        }
                     }
                 }
             }
-        }
+            __syncthreads();                                  // the previous item's products are done with c and t
 #pragma unroll
-        for (int q = 0; q < kPer; ++q) s.c[tid + q * kProjThreads] = acc[q];
-    }
-    __syncthreads();
+            for (int q = 0; q < kPer; ++q) s.c[tid + q * kProjThreads] = acc[q];
+        }
+        __syncthreads();
 
-    // ---- T_r[i][j] = sum_k C[k][row0+i] Phi[k][j]: thread = (row i, MP/16 columns) ---------------
-    {
-        constexpr int kCols = MP / 16;
-        const int i = tid >> 4, col0 = (tid & 15) * kCols;
-        double acc[kCols];
-#pragma unroll
-        for (int c = 0; c < kCols; ++c) acc[c] = 0.0;
-#pragma unroll 4
-        for (int k = 0; k < kD; ++k) {
-            const double cv = s.c[k * kRows + i];
-#pragma unroll
-            for (int c = 0; c < kCols; ++c) acc[c] = fma(cv, s.phi[k * MP + col0 + c], acc[c]);
-        }
-#pragma unroll
-        for (int c = 0; c < kCols; ++c) s.t[i * MP + col0 + c] = acc[c];
-    }
-    __syncthreads();
+        // look ahead: the next item's partials travel while this item is multiplied
+        const Item done = cur;
+        if (item + (int)gridDim.x < n_items) { cur = decode(item + gridDim.x); prefetch(cur); }
 
-    // ---- G_r[a][b] = sum_i Phi[row0+i][a] T_r[i][b]: thread = (MP/16 rows a) x (MP/16 columns b) --
-    {
-        constexpr int kT = MP / 16;
-        const int a0 = (tid >> 4) * kT, b0 = (tid & 15) * kT;
-        double acc[kT][kT];
+        // Both products run as fp64 mma.m8n8k4 (a warp-wide instruction does 256 FMAs for two 8-byte
+        // shared-memory loads per lane); the contraction is cut into four independent chains.
+        // ---- T_r (16 x MP) = C[rows,:] (16 x 128) Phi (128 x MP) --------------------------------
+        for (int tile = warp; tile < 2 * kNT; tile += kProjThreads / 32) {
+            const int mt = tile / kNT, nt = tile % kNT;
+            double d[4][2];
 #pragma unroll
-        for (int x = 0; x < kT; ++x)
+            for (int g = 0; g < 4; ++g) d[g][0] = d[g][1] = 0.0;
 #pragma unroll
-            for (int y = 0; y < kT; ++y) acc[x][y] = 0.0;
-#pragma unroll 4
-        for (int i = 0; i < kRows; ++i) {
-            double pa[kT], tb[kT];
+            for (int k0 = 0; k0 < kD / 4; k0 += 4) {
 #pragma unroll
-            for (int x = 0; x < kT; ++x) { pa[x] = s.phi[(row0 + i) * MP + a0 + x]; tb[x] = s.t[i * MP + b0 + x]; }
-#pragma unroll
-            for (int x = 0; x < kT; ++x)
-#pragma unroll
-                for (int y = 0; y < kT; ++y) acc[x][y] = fma(pa[x], tb[y], acc[x][y]);
+                for (int g = 0; g < 4; ++g) {
+                    const int k = g * (kD / 4) + k0 + fk;
+                    const double a = s.c[k * kRows + mt * 8 + fr];            // A[row][k] = C[k][row0 + row]
+                    const double bv = s.phi[k * LD + nt * 8 + fr];            // B[k][col]
+                    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                 : "+d"(d[g][0]), "+d"(d[g][1]) : "d"(a), "d"(bv));
+                }
+            }
+            s.t[(mt * 8 + fr) * LD + nt * 8 + 2 * fk] = (d[0][0] + d[1][0]) + (d[2][0] + d[3][0]);
+            s.t[(mt * 8 + fr) * LD + nt * 8 + 2 * fk + 1] = (d[0][1] + d[1][1]) + (d[2][1] + d[3][1]);
         }
-        double* out = g_partials + ((size_t)unit * kSlices + slice) * (MP * MP);
+        __syncthreads();
+
+        // ---- G_r (MP x MP) = Phi[rows,:]^T (MP x 16) T_r (16 x MP) ------------------------------
+        {
+            double* out = g_partials + ((size_t)done.unit * kSlices + done.slice) * (MP * MP);
+            for (int tile = warp; tile < kNT * kNT; tile += kProjThreads / 32) {
+                const int mt = tile / kNT, nt = tile % kNT;
+                double d[4][2];
 #pragma unroll
-        for (int x = 0; x < kT; ++x)
-#pragma unroll
-            for (int y = 0; y < kT; ++y) out[(a0 + x) * MP + b0 + y] = acc[x][y];
+                for (int g = 0; g < 4; ++g) {                 // four k-steps of 4 rows each, independent
+                    d[g][0] = d[g][1] = 0.0;
+                    const double a = s.phi[(row0 + g * 4 + fk) * LD + mt * 8 + fr];   // A[a][i] = Phi[row0 + i][a]
+                    const double bv = s.t[(g * 4 + fk) * LD + nt * 8 + fr];           // B[i][b] = T_r[i][b]
+                    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                 : "+d"(d[g][0]), "+d"(d[g][1]) : "d"(a), "d"(bv));
+                }
+                *reinterpret_cast<double2*>(out + (mt * 8 + fr) * MP + nt * 8 + 2 * fk) =
+                    make_double2((d[0][0] + d[1][0]) + (d[2][0] + d[3][0]), (d[0][1] + d[1][1]) + (d[2][1] + d[3][1]));
+            }
+        }
     }
 }
 
@@ -261,7 +301,9 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
     const int smem = (int)sizeof(ProjectSmem<MP>);
     cudaError_t e = cudaFuncSetAttribute(project_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    project_kernel<MP><<<dim3(units, kSlices), kProjThreads, smem, stream>>>(p, k, partials, phi, g_partials);
+    const int n_items = units * kSlices;
+    const int grid = n_items < 2 * 148 ? n_items : 2 * 148;       // two CTAs fit on an SM
+    project_kernel<MP><<<grid, kProjThreads, smem, stream>>>(p, k, partials, phi, g_partials, n_items);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     cholesky_kernel<MP><<<units, kCholThreads, 0, stream>>>(p, g_partials, phi, w, status);

@@ -11,6 +11,8 @@ What follows the paper step by step:
     small SVD, back-projection, squared row norms).
   * `exact_leverage_scores`  - Definition 1 / Eq. 1 (the quantity Algorithm 1
     approximates; used to pin the oracle, and as the m = d special case).
+  * `attention_scores`       - Eq. 5 (column sums of chunked non-causal softmax
+    attention, mean-pooled).
   * `blend`                  - Eq. 6 (z-scored attention term + lambda * z-scored
     outlier term).
   * `keep_count`             - the number of retained tokens, ceil(r N) (Section 3,
@@ -35,6 +37,9 @@ Readings taken where the paper is silent or inconsistent:
   * The calibration curve is increasing in r; the paper writes the choice of
     r* as an arg max subject to f >= tau, which is read as the smallest such r
     (Section 3.5 states the goal as the least retention that keeps quality).
+
+  * Eq. 5 details (softmax scale, last chunk, grouped queries, pooling window)
+    are not given by the paper; `attention_scores` states the reading taken.
 
 Pins (see tests/test_oracle_pins.py): closed-form leverage scores, sum = rank,
 range [0,1], invariance under K -> K A and Phi -> Phi A, m = d reduces to the
@@ -149,6 +154,39 @@ def blend(a, o: np.ndarray, lam: float) -> np.ndarray:
     if o.size == 0:
         return o.copy()
     return _zscore(a) + float(lam) * _zscore(o)
+
+
+# ----------------------------------------------------------------------------
+# Eq. 5: chunked non-causal attention scores
+# ----------------------------------------------------------------------------
+def attention_scores(Q: np.ndarray, K: np.ndarray, chunk: int = 256, scale: float = 1.0, pool: int = 1) -> np.ndarray:
+    """a = concat_i 1^T softmax(Q[i] K[i]^T) over chunks of `chunk` consecutive tokens (Eq. 5),
+    followed by mean pooling.
+
+    Q [G, n, d]: the G query heads that share this KV head (their column sums are added);
+    K [n, d].  Readings where the paper is silent: logits are multiplied by `scale` before the
+    softmax (Eq. 5 prints none; 1/sqrt(d) is the usual choice); the last, shorter chunk is a
+    softmax over its own keys; pooling is a centred window of `pool` (odd) tokens over the
+    concatenated vector, zero beyond the ends of the sequence, divided by `pool`."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    if Q.ndim == 2:
+        Q = Q[None]
+    n = K.shape[0]
+    a = np.zeros(n)
+    for lo in range(0, n, chunk):
+        hi = min(n, lo + chunk)
+        for g in range(Q.shape[0]):
+            S = (Q[g, lo:hi] @ K[lo:hi].T) * float(scale)
+            S = S - S.max(axis=1, keepdims=True)
+            P = np.exp(S)
+            P /= P.sum(axis=1, keepdims=True)
+            a[lo:hi] += P.sum(axis=0)                     # 1^T softmax(...)
+    if pool > 1:
+        half = pool // 2
+        padded = np.concatenate([np.zeros(half), a, np.zeros(half)])
+        a = np.array([padded[i:i + pool].sum() / pool for i in range(n)])
+    return a
 
 
 # ----------------------------------------------------------------------------

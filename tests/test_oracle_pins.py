@@ -165,6 +165,43 @@ def test_make_sketch_statistics_and_determinism():
     assert x == 0xE220A8397B1DCDAF
 
 
+# ----------------------------------------------------------------------------- attention term (Eq. 5)
+def test_attention_scores_pins():
+    import torch
+    rng = _rng(12)
+    n, d, G = 37, 8, 3
+    Q = rng.standard_normal((G, n, d)); K = rng.standard_normal((n, d))
+    # one chunk covering the sequence: the unchunked definition a = 1^T softmax(Q K^T), via a library softmax
+    want = sum(torch.softmax(torch.from_numpy(Q[g] @ K.T * 0.5), dim=1).sum(dim=0).numpy() for g in range(G))
+    np.testing.assert_allclose(orc.attention_scores(Q, K, chunk=64, scale=0.5), want, rtol=1e-12)
+    # every query row spreads a mass of one over its chunk: total = G * n, per chunk = G * chunk length
+    a = orc.attention_scores(Q, K, chunk=10, scale=0.5)
+    assert abs(a.sum() - G * n) < 1e-9
+    np.testing.assert_allclose([a[i:i + 10].sum() for i in range(0, n, 10)], [30, 30, 30, 21], rtol=1e-12)
+    # zero queries: uniform attention, every key of a full chunk receives G
+    np.testing.assert_allclose(orc.attention_scores(np.zeros((G, n, d)), K, chunk=10), np.full(n, float(G)), rtol=1e-12)
+    # chunks are independent: changing keys and queries of chunk 0 leaves the other chunks' scores alone
+    K2, Q2 = K.copy(), Q.copy(); K2[:10] += 1.0; Q2[:, :10] *= -2.0
+    np.testing.assert_allclose(orc.attention_scores(Q2, K2, chunk=10, scale=0.5)[10:], a[10:], rtol=1e-12)
+    # permuting the tokens of one chunk permutes its scores
+    perm = np.arange(n); perm[10:20] = 10 + rng.permutation(10)
+    np.testing.assert_allclose(orc.attention_scores(Q[:, perm], K[perm], chunk=10, scale=0.5), a[perm], rtol=1e-12)
+    # two tokens, one channel, by hand: rows (x1, x2), keys (k1, k2)
+    x, k = np.array([0.3, -1.2]), np.array([2.0, 0.5])
+    p = lambda q: np.exp(q * k) / np.exp(q * k).sum()
+    np.testing.assert_allclose(orc.attention_scores(x[None, :, None], k[:, None], chunk=2), p(x[0]) + p(x[1]), rtol=1e-13)
+    # a key aligned with every query collects nearly all the mass of its chunk
+    Kbig = 0.01 * rng.standard_normal((20, d)); Qpos = np.abs(rng.standard_normal((1, 20, d))) + 1.0
+    Kbig[7] = 10.0
+    a_big = orc.attention_scores(Qpos, Kbig, chunk=20)
+    assert a_big.argmax() == 7 and a_big[7] > 19.9
+    # pooling: centred mean with zero padding; window 1 is the identity
+    base = orc.attention_scores(Q, K, chunk=10, scale=0.5)
+    pooled = orc.attention_scores(Q, K, chunk=10, scale=0.5, pool=3)
+    assert abs(pooled[5] - base[4:7].mean()) < 1e-12 and abs(pooled[0] - base[:2].sum() / 3) < 1e-12
+    assert abs(pooled[-1] - base[-2:].sum() / 3) < 1e-12
+
+
 # ----------------------------------------------------------------------------- blend (Eq. 6)
 def test_blend_properties():
     rng = _rng(9)

@@ -172,6 +172,27 @@ int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_sc
                                 void* const* stage_events, int32_t n_events);
 
 /*
+ * Attention term of the score (Eq. 5): for every unit, a = concat_i 1^T softmax(scale * Q[i] K[i]^T)
+ * over chunks i of `chunk` consecutive tokens of the sequence (no causal mask), summed over the
+ * q_per_kv query heads that share the KV head, then mean-pooled.  The result is what
+ * compactor_score / compactor_compress take as attn_scores.
+ *   q        bf16 [layers][heads * q_per_kv][total_tokens][d]; query head j of KV head h is
+ *            head index h * q_per_kv + j.  Same stride and alignment rules as the keys.
+ *   chunk    must be 256 (the paper's setting).
+ *   scale    > 0; the paper's equation prints no scale, attention layers use 1/sqrt(d).
+ *   pool     odd window of the mean pooling (1 = none): centred, zero beyond the ends of the
+ *            sequence, divided by `pool` (the paper pools but does not give the window).
+ *   attn_out device fp32 [layers][heads][total_tokens].
+ * The last, shorter chunk of a sequence is a softmax over its own keys.  Exponentials are
+ * rounded to fp16 before they are summed over the query rows on the tensor cores (fp32
+ * accumulation).  Workspace: compactor_workspace_bytes() suffices (12*(batch+1) bytes rounded up
+ * to 256, plus 4 bytes per output element when pool > 1).
+ */
+int compactor_attention_scores(const compactor_shape* shape, compactor_mat q, compactor_mat k,
+                               int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,
+                               float* attn_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * compactor_score for callers that cannot allocate device memory (the paper has no counterpart;
  * this is a deployment convenience).  Same inputs, outputs and results as compactor_score, but
  * no workspace argument: the scratch is a fixed array of compactor_builtin_scratch_bytes()

@@ -52,6 +52,8 @@ def _load() -> ctypes.CDLL:
                                        c_void_p, c_float, POINTER(c_int32), c_void_p, c_void_p, c_void_p, c_void_p,
                                        c_void_p, c_void_p, c_size_t, c_void_p]
     lib.compactor_compress_profiled.argtypes = lib.compactor_compress.argtypes + [POINTER(c_void_p), c_int32]
+    lib.compactor_attention_scores.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_int32, c_int32,
+                                               c_float, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.compactor_builtin_scratch_bytes.restype = c_size_t
     lib.compactor_score_builtin_scratch.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_void_p, c_float,
                                                     c_void_p, c_void_p, c_void_p]
@@ -64,7 +66,7 @@ LIB_PATH = _build.LIB
 EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_keep_count",
            "compactor_calibrated_ratio", "compactor_workspace_bytes", "compactor_score", "compactor_select",
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
-           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch"]
+           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores"]
 
 N_STAGE_EVENTS = 7
 STAGE_NAMES = ["gram", "factor", "score", "blend", "select", "compact"]
@@ -198,3 +200,10 @@ def score_builtin_scratch(shape: Shape, k_score: torch.Tensor, phi: torch.Tensor
     _check(LIB.compactor_score_builtin_scratch(byref(shape.c), mat(k_score), _ptr(phi), _ptr(attn), lam,
                                                _ptr(scores_out), _ptr(status), _stream()),
            "compactor_score_builtin_scratch")
+
+
+def attention_scores(shape: Shape, q: torch.Tensor, k: torch.Tensor, q_per_kv: int, attn_out: torch.Tensor,
+                     workspace: torch.Tensor, scale: float, pool: int = 1, chunk: int = 256) -> None:
+    """Eq. 5: chunked non-causal attention column sums of `q` [layers, heads*q_per_kv, tokens, d] against `k`."""
+    _check(LIB.compactor_attention_scores(byref(shape.c), mat(q), mat(k), q_per_kv, chunk, scale, pool, _ptr(attn_out),
+                                          _ptr(workspace), workspace.numel(), _stream()), "compactor_attention_scores")

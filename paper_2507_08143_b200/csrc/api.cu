@@ -399,3 +399,26 @@ int compactor_score_builtin_scratch(const compactor_shape* shape, compactor_mat 
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Attention term (Eq. 5).
+extern "C" int compactor_attention_scores(const compactor_shape* shape, compactor_mat q, compactor_mat k,
+                                          int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,
+                                          float* attn_out, void* workspace, size_t workspace_bytes, void* stream) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (chunk != 256) return COMPACTOR_E_UNSUPPORTED;
+    if (!mat_ok(q) || !mat_ok(k) || attn_out == nullptr || workspace == nullptr || q_per_kv < 1 ||
+        (long long)shape->heads * q_per_kv > 65535 || !(scale > 0.f) || !isfinite(scale) || pool < 1 || (pool & 1) == 0)
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (((uintptr_t)workspace & 255) != 0) return COMPACTOR_E_INVALID_ARGUMENT;
+    replan_chunk(shape, &hp, chunk);                 // one CTA per chunk of 256 tokens
+    const size_t raw_bytes = pool > 1 ? sizeof(float) * (size_t)hp.plan.total_tokens * shape->layers * shape->heads : 0;
+    if (workspace_bytes < hp.off_w + raw_bytes) return COMPACTOR_E_WORKSPACE;
+    if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CK(upload_tables(&hp, workspace, st));
+    float* raw = reinterpret_cast<float*>(static_cast<char*>(workspace) + hp.off_w);
+    CK(launch_attention(hp.plan, to_mat(q), to_mat(k), q_per_kv, scale, pool, raw, attn_out, st));
+    return COMPACTOR_OK;
+}

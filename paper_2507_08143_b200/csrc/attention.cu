@@ -1,0 +1,254 @@
+// Attention term of the score (Eq. 5): a = concat_i 1^T softmax(Q[i] K[i]^T) over chunks of 256
+// consecutive tokens, no causal mask, summed over the query heads that share a KV head, then
+// mean-pooled.  Readings where the paper is silent: logits are multiplied by a caller-given scale,
+// the last, shorter chunk is a softmax over its own keys, pooling is a centred window with zero
+// padding.
+//
+// One CTA per (chunk, layer, KV head).  Warp 0 loads the chunk's keys once and streams the query
+// heads' rows in halves of 128 through a two-slot ring (TMA, 128-byte swizzle).  One thread of
+// warp 1 issues, per half, S = Q_half K^T (tcgen05.mma, 128 x 256 fp32 in tensor memory).  Warps
+// 2-5 own one query row each: row maximum, e = exp(scale (s - max)) written as fp16 into shared
+// memory in the layout of an MN-major B operand, and the reciprocal of the row sum (two fp16 terms)
+// into rows 0 and 1 of a small A operand.  A second MMA then adds w^T E (1 x 256, the normalised column sums of the half)
+// into a second accumulator that runs over all halves and query heads; it is read out once.
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+#include "sm100.cuh"
+
+namespace compactor {
+namespace {
+
+using namespace sm100;
+
+constexpr int kChunk = 256;
+constexpr int kHalf = 128;
+constexpr int kThreads = 192;
+constexpr int kKBox = kChunk * 128;        // 64 channels x 256 tokens x 2 B
+constexpr int kQBox = kHalf * 128;         // 64 channels x 128 rows
+constexpr int kPBlock = kHalf * 128;       // 128 rows x 64 keys, fp16
+constexpr int kWBox = 64 * 128;            // 64 rows x 64 k, fp16
+constexpr uint32_t kTmemCols = 512;        // S at column 0, column sums at column 256
+
+struct __align__(1024) AttnSmem {
+    unsigned char k[2 * kKBox];
+    unsigned char q[2][2 * kQBox];
+    unsigned char p[4 * kPBlock];
+    unsigned char w[2 * kWBox];
+    uint64_t k_full, q_full[2], q_empty[2], s_full, p_ready, d_full;
+    uint32_t tmem_base;
+    int abort;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
+                 int q_per_kv, float scale_log2e, float* __restrict__ out) {
+    extern __shared__ unsigned char smem_raw[];
+    AttnSmem& s = *reinterpret_cast<AttnSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
+    const int chunk_id = blockIdx.x, lh = blockIdx.y;
+    const int layer = lh / p.heads, head = lh % p.heads;
+    const int b = find_segment(p.cu_chunks, p.batch, chunk_id);
+    const int tok_begin = p.cu_seqlens[b] + (chunk_id - p.cu_chunks[b]) * kChunk;
+    const int n_tok = min(kChunk, p.cu_seqlens[b + 1] - tok_begin);
+    const int n_iter = 2 * q_per_kv;                   // halves of 128 query rows
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        prefetch_tensormap(&qmap);
+        prefetch_tensormap(&kmap);
+        mbar_init(&s.k_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 1); }
+        mbar_init(&s.s_full, 1);
+        mbar_init(&s.p_ready, kHalf);
+        mbar_init(&s.d_full, 1);
+        s.abort = 0;
+        fence_barrier_init();
+    }
+    for (int i = threadIdx.x; i < 2 * kWBox / 16; i += kThreads)       // rows 1..63 of the weight operand stay zero
+        reinterpret_cast<uint4*>(s.w)[i] = make_uint4(0, 0, 0, 0);
+    fence_proxy_async_smem();
+    if (warp == 1) { tmem_alloc(&s.tmem_base, kTmemCols); tmem_relinquish(); }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = s.tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(&s.k_full, 2 * kKBox);
+            tma_load_4d(s.k, &kmap, &s.k_full, 0, tok_begin, head, layer);
+            tma_load_4d(s.k + kKBox, &kmap, &s.k_full, 64, tok_begin, head, layer);
+            for (int it = 0; it < n_iter; ++it) {
+                const int st = it & 1, use = it >> 1;
+                if (use > 0 && !mbar_wait(&s.q_empty[st], (use - 1) & 1)) { s.abort = 1; break; }
+                if (*(volatile int*)&s.abort) break;
+                mbar_arrive_expect_tx(&s.q_full[st], 2 * kQBox);
+                const int qhead = head * q_per_kv + (it >> 1);
+                const int row = tok_begin + (it & 1) * kHalf;
+                tma_load_4d(s.q[st], &qmap, &s.q_full[st], 0, row, qhead, layer);
+                tma_load_4d(s.q[st] + kQBox, &qmap, &s.q_full[st], 64, row, qhead, layer);
+            }
+        }
+    } else if (warp == 1) {
+        constexpr uint32_t idesc_s = umma_idesc_16bit(1, 128, kChunk, 0, 0);     // bf16: Q (K-major) x K^T (K-major)
+        constexpr uint32_t idesc_c = umma_idesc_16bit(0, 64, kChunk, 0, 1);      // fp16: w (K-major) x E (MN-major)
+        const uint32_t k_base = smem_u32(s.k), p_base = smem_u32(s.p), w_base = smem_u32(s.w);
+        auto column_sums = [&](int it) {           // adds w^T E of half `it` into the second accumulator
+#pragma unroll
+            for (int ks = 0; ks < kHalf / 16; ++ks) {
+                const uint64_t a_desc = umma_desc_sw128(w_base + (ks >> 2) * kWBox + (ks & 3) * 32, 16, 1024);
+                const uint64_t b_desc = umma_desc_sw128(p_base + ks * 2048, kPBlock, 1024);
+                umma_bf16(tmem + 256, a_desc, b_desc, idesc_c, (it > 0) || (ks > 0));
+            }
+        };
+        bool ok = mbar_wait(&s.k_full, 0);
+        for (int it = 0; it < n_iter && ok; ++it) {
+            const int st = it & 1, use = it >> 1;
+            ok = mbar_wait(&s.q_full[st], use & 1);
+            if (ok && it > 0) ok = mbar_wait(&s.p_ready, (it - 1) & 1);     // S consumed, E and w of the previous half written
+            ok = ok && !*(volatile int*)&s.abort;
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (lane == 0) {
+                if (it > 0) column_sums(it - 1);
+                const uint32_t q_base = smem_u32(s.q[st]);
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t a_desc = umma_desc_sw128(q_base + (ks >> 2) * kQBox + (ks & 3) * 32, 16, 1024);
+                    const uint64_t b_desc = umma_desc_sw128(k_base + (ks >> 2) * kKBox + (ks & 3) * 32, 16, 1024);
+                    umma_bf16(tmem, a_desc, b_desc, idesc_s, ks > 0);
+                }
+                umma_commit(&s.q_empty[st]);
+                umma_commit(&s.s_full);
+            }
+            __syncwarp();
+        }
+        if (ok) ok = mbar_wait(&s.p_ready, (n_iter - 1) & 1);
+        if (ok) {
+            tc_fence_after_sync();
+            if (lane == 0) { column_sums(n_iter - 1); umma_commit(&s.d_full); }
+            __syncwarp();
+        } else {
+            s.abort = 1;
+            if (lane == 0) { mbar_arrive(&s.s_full); mbar_arrive(&s.d_full); }     // wake the other warps
+        }
+    } else {
+        const int q = warp & 3;
+        const int row = q * 32 + lane;                       // query row within the half = TMEM lane
+        const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+        bool ok = true;
+        for (int it = 0; it < n_iter && ok; ++it) {
+            ok = mbar_wait(&s.s_full, it & 1) && !*(volatile int*)&s.abort;
+            if (!ok) break;
+            tc_fence_after_sync();
+            const bool row_valid = (it & 1) * kHalf + row < n_tok;
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kChunk; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(lane_addr + c0, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (c0 + i < n_tok) mx = fmaxf(mx, __uint_as_float(r[i]));
+            }
+            float sum = 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < kChunk; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(lane_addr + c0, r);
+                tmem_ld_wait();
+                uint32_t packed[16];
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    const float e0 = (row_valid && c0 + i < n_tok) ? exp2f((__uint_as_float(r[i]) - mx) * scale_log2e) : 0.f;
+                    const float e1 = (row_valid && c0 + i + 1 < n_tok) ? exp2f((__uint_as_float(r[i + 1]) - mx) * scale_log2e) : 0.f;
+                    const __half2 h = __floats2half2_rn(e0, e1);
+                    // the column sums use the rounded values, so the row sum does too
+                    sum += __low2float(h) + __high2float(h);
+                    packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                unsigned char* blk = s.p + (c0 >> 6) * kPBlock + row * 128;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int piece = ((c0 & 63) >> 3) + j;
+                    *reinterpret_cast<uint4*>(blk + ((piece ^ (row & 7)) << 4)) =
+                        make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                }
+            }
+            // 1 / (row sum) as two fp16 terms in rows 0 and 1 of the weight operand (row 1 is swizzled by its index)
+            const float wgt = (row_valid && sum > 0.f) ? 1.0f / sum : 0.f;
+            const __half w_hi = __float2half_rn(wgt);
+            const __half w_lo = __float2half_rn(wgt - __half2float(w_hi));
+            unsigned char* wbox = s.w + (row >> 6) * kWBox;
+            const int piece = (row & 63) >> 3, within = (row & 7) * 2;
+            *reinterpret_cast<__half*>(wbox + (piece << 4) + within) = w_hi;
+            *reinterpret_cast<__half*>(wbox + 128 + ((piece ^ 1) << 4) + within) = w_lo;
+            fence_proxy_async_smem();
+            tc_fence_before_sync();
+            mbar_arrive(&s.p_ready);
+        }
+        if (!ok) s.abort = 1;
+        if (q == 0) {                                        // lanes 0-31 of tensor memory: row 0 holds the column sums
+            const bool okd = ok && mbar_wait(&s.d_full, 0) && !*(volatile int*)&s.abort;
+            tc_fence_after_sync();
+            if (okd) {
+                float* dst = out + (size_t)lh * p.total_tokens + tok_begin;
+#pragma unroll 1
+                for (int c0 = 0; c0 < kChunk; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(tmem + 256 + c0, r);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float v = __uint_as_float(r[i]);
+                        const float total = v + __shfl_sync(0xffffffffu, v, 1);      // rows 0 and 1: hi and lo weights
+                        if (lane == 0 && c0 + i < n_tok) dst[c0 + i] = total;
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+}
+
+// Centred mean over `pool` tokens inside each sequence, zero beyond its ends.
+__global__ void pool_kernel(Plan p, const float* __restrict__ raw, float* __restrict__ out, int pool) {
+    const int lh = blockIdx.y;
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= p.total_tokens) return;
+    const int b = find_segment(p.cu_seqlens, p.batch, i);
+    const int lo = p.cu_seqlens[b], hi = p.cu_seqlens[b + 1];
+    const float* src = raw + (size_t)lh * p.total_tokens;
+    const int half = pool / 2;
+    float acc = 0.f;
+    for (int j = max(lo, i - half); j <= min(hi - 1, i + half); ++j) acc += src[j];
+    out[(size_t)lh * p.total_tokens + i] = acc / (float)pool;
+}
+
+}  // namespace
+
+cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_per_kv, float scale, int pool,
+                             float* raw, float* out, cudaStream_t stream) {
+    if (p.total_chunks == 0) return cudaSuccess;
+    CUtensorMap qmap, kmap;
+    if (!make_kv_tensor_map(&qmap, q.ptr, p.layers, p.heads * q_per_kv, p.total_tokens, q.stride_layer, q.stride_head,
+                            q.stride_token, kHalf) ||
+        !make_kv_tensor_map(&kmap, k.ptr, p.layers, p.heads, p.total_tokens, k.stride_layer, k.stride_head,
+                            k.stride_token, kChunk))
+        return cudaErrorInvalidValue;
+    const int smem = (int)sizeof(AttnSmem) + 1024;
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    float* dst = pool > 1 ? raw : out;
+    attention_kernel<<<dim3(p.total_chunks, p.layers * p.heads), kThreads, smem, stream>>>(
+        p, qmap, kmap, q_per_kv, scale * 1.4426950408889634f, dst);
+    e = cudaGetLastError();
+    if (e != cudaSuccess || pool <= 1) return e;
+    pool_kernel<<<dim3((p.total_tokens + 255) / 256, p.layers * p.heads), 256, 0, stream>>>(p, raw, out, pool);
+    return cudaGetLastError();
+}
+
+}  // namespace compactor

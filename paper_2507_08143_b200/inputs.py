@@ -196,3 +196,15 @@ def make_attention_scores(w: Workload, seed: int = 0, device="cpu") -> torch.Ten
     g.manual_seed(0xA77E0000 + seed)
     x = torch.randn(w.layers, w.heads, w.total_tokens, generator=g, dtype=torch.float32, device=dev)
     return torch.exp(0.75 * x)
+
+
+def make_queries(w: Workload, q_per_kv: int, device="cpu", seed: int = 0) -> torch.Tensor:
+    """Stand-in query vectors for the attention term: bf16 [L, H * q_per_kv, total_tokens, d], Gaussian with a
+    per-head channel scale (a few heads attend sharply, most diffusely)."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(0x9E7700 + 131 * w.seed + seed)
+    hq = w.heads * q_per_kv
+    q = torch.randn(w.layers, hq, w.total_tokens, w.d, generator=g, dtype=torch.float32, device=dev)
+    sharp = 0.5 + 2.0 * torch.rand(w.layers, hq, 1, 1, generator=g, dtype=torch.float32, device=dev)
+    return (q * sharp).to(torch.bfloat16)

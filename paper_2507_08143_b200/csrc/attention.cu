@@ -7,7 +7,7 @@
 // One CTA per (chunk, layer, KV head).  Warp 0 loads the chunk's keys once and streams the query
 // heads' rows in halves of 128 through a two-slot ring (TMA, 128-byte swizzle).  One thread of
 // warp 1 issues, per half, S = Q_half K^T (tcgen05.mma, 128 x 256 fp32 in tensor memory).  Warps
-// 2-5 own one query row each: row maximum, e = exp(scale (s - max)) written as fp16 into shared
+// 2-9 share the 128 query rows (a pair of warps per 32 rows, 128 keys each): row maximum, e = exp(scale (s - max)) written as fp16 into shared
 // memory in the layout of an MN-major B operand, and the reciprocal of the row sum (two fp16 terms)
 // into rows 0 and 1 of a small A operand.  A second MMA then adds w^T E (1 x 256, the normalised column sums of the half)
 // into a second accumulator that runs over all halves and query heads; it is read out once.
@@ -23,7 +23,8 @@ using namespace sm100;
 
 constexpr int kChunk = 256;
 constexpr int kHalf = 128;
-constexpr int kThreads = 192;
+constexpr int kSoftmaxWarps = 8;           // two warps per query row quadrant: each takes 128 of the 256 keys
+constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
 constexpr int kKBox = kChunk * 128;        // 64 channels x 256 tokens x 2 B
 constexpr int kQBox = kHalf * 128;         // 64 channels x 128 rows
 constexpr int kPBlock = kHalf * 128;       // 128 rows x 64 keys, fp16
@@ -36,9 +37,21 @@ struct __align__(1024) AttnSmem {
     unsigned char p[4 * kPBlock];
     unsigned char w[2 * kWBox];
     uint64_t k_full, q_full[2], q_empty[2], s_full, p_ready, d_full;
+    float xmax[2][kHalf];      // row maxima / row sums of the two column halves, exchanged between warp pairs
+    float xsum[2][kHalf];
     uint32_t tmem_base;
     int abort;
+    int abort_mma;             // set by the MMA warp alone, before it wakes the softmax warps: they all see the same value
 };
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void softmax_pair_sync() {          // the 256 softmax threads only
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
@@ -59,9 +72,10 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         mbar_init(&s.k_full, 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 1); }
         mbar_init(&s.s_full, 1);
-        mbar_init(&s.p_ready, kHalf);
+        mbar_init(&s.p_ready, 32 * kSoftmaxWarps);
         mbar_init(&s.d_full, 1);
         s.abort = 0;
+        s.abort_mma = 0;
         fence_barrier_init();
     }
     for (int i = threadIdx.x; i < 2 * kWBox / 16; i += kThreads)       // rows 1..63 of the weight operand stay zero
@@ -130,67 +144,91 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             __syncwarp();
         } else {
             s.abort = 1;
+            s.abort_mma = 1;
+            __threadfence_block();
+            __syncwarp();
             if (lane == 0) { mbar_arrive(&s.s_full); mbar_arrive(&s.d_full); }     // wake the other warps
         }
     } else {
-        const int q = warp & 3;
+        const int q = warp & 3;                              // TMEM lane quadrant
+        const int ch = (warp - 2) >> 2;                      // which 128 of the 256 keys
         const int row = q * 32 + lane;                       // query row within the half = TMEM lane
-        const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16);
+        const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + ch * 128;
+        const bool full = n_tok == kChunk;                   // only the last chunk of a sequence needs masks
         bool ok = true;
         for (int it = 0; it < n_iter && ok; ++it) {
-            ok = mbar_wait(&s.s_full, it & 1) && !*(volatile int*)&s.abort;
+            // every softmax thread takes the same decision here (they meet at a named barrier below)
+            ok = mbar_wait(&s.s_full, it & 1) && !*(volatile int*)&s.abort_mma;
             if (!ok) break;
             tc_fence_after_sync();
             const bool row_valid = (it & 1) * kHalf + row < n_tok;
             float mx = -INFINITY;
 #pragma unroll 1
-            for (int c0 = 0; c0 < kChunk; c0 += 32) {
+            for (int c0 = 0; c0 < 128; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld_32x32b_x32(lane_addr + c0, r);
                 tmem_ld_wait();
+                if (full) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (c0 + i < n_tok) mx = fmaxf(mx, __uint_as_float(r[i]));
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (ch * 128 + c0 + i < n_tok) mx = fmaxf(mx, __uint_as_float(r[i]));
+                }
             }
+            s.xmax[ch][row] = mx;
+            softmax_pair_sync();
+            mx = fmaxf(s.xmax[0][row], s.xmax[1][row]);      // finite: key 0 of the chunk always exists
+            const float bias = -mx * scale_log2e;
             float sum = 0.f;
 #pragma unroll 1
-            for (int c0 = 0; c0 < kChunk; c0 += 32) {
+            for (int c0 = 0; c0 < 128; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld_32x32b_x32(lane_addr + c0, r);
                 tmem_ld_wait();
                 uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const float e0 = (row_valid && c0 + i < n_tok) ? exp2f((__uint_as_float(r[i]) - mx) * scale_log2e) : 0.f;
-                    const float e1 = (row_valid && c0 + i + 1 < n_tok) ? exp2f((__uint_as_float(r[i + 1]) - mx) * scale_log2e) : 0.f;
+                    float e0 = ex2_approx(fmaf(__uint_as_float(r[i]), scale_log2e, bias));
+                    float e1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), scale_log2e, bias));
+                    if (!full) {
+                        if (!row_valid || ch * 128 + c0 + i >= n_tok) e0 = 0.f;
+                        if (!row_valid || ch * 128 + c0 + i + 1 >= n_tok) e1 = 0.f;
+                    }
+                    sum += e0 + e1;
                     const __half2 h = __floats2half2_rn(e0, e1);
-                    // the column sums use the rounded values, so the row sum does too
-                    sum += __low2float(h) + __high2float(h);
                     packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&h);
                 }
-                unsigned char* blk = s.p + (c0 >> 6) * kPBlock + row * 128;
+                const int col = ch * 128 + c0;
+                unsigned char* blk = s.p + (col >> 6) * kPBlock + row * 128;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    const int piece = ((c0 & 63) >> 3) + j;
+                    const int piece = ((col & 63) >> 3) + j;
                     *reinterpret_cast<uint4*>(blk + ((piece ^ (row & 7)) << 4)) =
                         make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
                 }
             }
-            // 1 / (row sum) as two fp16 terms in rows 0 and 1 of the weight operand (row 1 is swizzled by its index)
-            const float wgt = (row_valid && sum > 0.f) ? 1.0f / sum : 0.f;
-            const __half w_hi = __float2half_rn(wgt);
-            const __half w_lo = __float2half_rn(wgt - __half2float(w_hi));
-            unsigned char* wbox = s.w + (row >> 6) * kWBox;
-            const int piece = (row & 63) >> 3, within = (row & 7) * 2;
-            *reinterpret_cast<__half*>(wbox + (piece << 4) + within) = w_hi;
-            *reinterpret_cast<__half*>(wbox + 128 + ((piece ^ 1) << 4) + within) = w_lo;
+            s.xsum[ch][row] = sum;
+            softmax_pair_sync();
+            if (ch == 0) {
+                // 1 / (row sum) as two fp16 terms in rows 0 and 1 of the weight operand (row 1 is swizzled by its index)
+                sum = s.xsum[0][row] + s.xsum[1][row];
+                const float wgt = (row_valid && sum > 0.f) ? 1.0f / sum : 0.f;
+                const __half w_hi = __float2half_rn(wgt);
+                const __half w_lo = __float2half_rn(wgt - __half2float(w_hi));
+                unsigned char* wbox = s.w + (row >> 6) * kWBox;
+                const int piece = (row & 63) >> 3, within = (row & 7) * 2;
+                *reinterpret_cast<__half*>(wbox + (piece << 4) + within) = w_hi;
+                *reinterpret_cast<__half*>(wbox + 128 + ((piece ^ 1) << 4) + within) = w_lo;
+            }
             fence_proxy_async_smem();
             tc_fence_before_sync();
             mbar_arrive(&s.p_ready);
         }
         if (!ok) s.abort = 1;
-        if (q == 0) {                                        // lanes 0-31 of tensor memory: row 0 holds the column sums
-            const bool okd = ok && mbar_wait(&s.d_full, 0) && !*(volatile int*)&s.abort;
+        if (q == 0 && ch == 0) {                             // lanes 0-31 of tensor memory: rows 0 and 1 hold the column sums
+            const bool okd = ok && mbar_wait(&s.d_full, 0) && !*(volatile int*)&s.abort_mma;
             tc_fence_after_sync();
             if (okd) {
                 float* dst = out + (size_t)lh * p.total_tokens + tok_begin;

@@ -30,7 +30,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the dominant kernels per head-token, from ncu captures of a smaller case of
 # the same kernels (see profiles/); bytes read + written per token of one (layer, head).
-NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN = {"gram": 286.3, "score": 260.9, "compact": 316.3}   # compact: at 32 % kept
+NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN = {"gram": 257.1, "score": 260.7, "compact": 316.1}   # compact: at 32 % kept
 
 
 def parse_args():

@@ -92,9 +92,12 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
 #pragma unroll
             for (int q = 0; q < kPer; ++q) {
                 const int e = tid + q * kProjThreads;
-                pre[u][q] = (u < it.n_part && it.n_tok > kExactGramTokens)
-                                ? __ldcs(it.part + (size_t)u * kGramElems + (e / kRows) * kD + it.slice * kRows + (e % kRows))
-                                : 0.0;
+                pre[u][q] = 0.0;
+                if (u < it.n_part && it.n_tok > kExactGramTokens) {
+                    // volatile: keeps the load here, ahead of the matrix products, instead of at its first use
+                    const double* src = it.part + (size_t)u * kGramElems + (e / kRows) * kD + it.slice * kRows + (e % kRows);
+                    asm volatile("ld.global.cs.f64 %0, [%1];" : "=d"(pre[u][q]) : "l"(src));
+                }
             }
     };
 

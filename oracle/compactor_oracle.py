@@ -18,6 +18,8 @@ What follows the paper step by step:
   * `keep_count`             - the number of retained tokens, ceil(r N) (Section 3,
     Preliminaries; Section 3.4).
   * `top_k_indices`          - per-head top-k of the scores.
+  * `top_k_across_heads`     - the same budget spent over all heads of a layer
+    (Section 3.4's alternative; ties: lower head, then lower index).
   * `compact`                - the retained rows of K and V.
   * `calibrated_ratio`       - inverse of the fitted curve f_{alpha,beta}
     (Section 3.5).
@@ -208,6 +210,21 @@ def top_k_indices(s: np.ndarray, kk: int) -> np.ndarray:
     kk = int(kk)
     order = np.lexsort((np.arange(n), -s))            # primary key -s, then index
     return np.sort(order[:kk]).astype(np.int32)
+
+
+def top_k_across_heads(S: np.ndarray, budget: int):
+    """Selection across the heads of one layer (Section 3.4 allows the top scores to be taken over
+    all heads instead of per head): S [H, n] holds the heads' scores of one sequence; the `budget`
+    largest entries are kept, ranked by (score descending, head ascending, index ascending).
+    Returns one ascending index array per head; their lengths add up to `budget`."""
+    S = np.asarray(S)
+    H, n = S.shape
+    budget = int(budget)
+    heads = np.repeat(np.arange(H), n)
+    idxs = np.tile(np.arange(n), H)
+    order = np.lexsort((idxs, heads, -S.reshape(-1)))      # primary -score, then head, then index
+    chosen = order[:budget]
+    return [np.sort(idxs[chosen][heads[chosen] == h]).astype(np.int32) for h in range(H)]
 
 
 def compact(K_bits: np.ndarray, V_bits: np.ndarray, idx: np.ndarray):

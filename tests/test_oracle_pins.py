@@ -272,6 +272,24 @@ def test_topk_random_and_edges():
     assert orc.top_k_indices(np.array([-1.0, -3.0, -2.0]), 2).tolist() == [0, 2]
 
 
+def test_topk_across_heads_brute_force():
+    rng = _rng(13)
+    for H, n, budget in ((2, 5, 4), (3, 7, 10), (4, 6, 1), (3, 4, 12), (2, 9, 9)):
+        for trial in range(20):
+            S = np.round(rng.random((H, n)), 1)           # many ties, also across heads
+            got = orc.top_k_across_heads(S, budget)
+            triples = sorted(((-S[h, i], h, i) for h in range(H) for i in range(n)))[:budget]
+            want = [sorted(i for (_, hh, i) in triples if hh == h) for h in range(H)]
+            assert [g.tolist() for g in got] == want
+            assert sum(len(g) for g in got) == budget
+    # one head far above the others takes the whole budget; equal heads split like per-head selection
+    S = np.stack([np.linspace(10, 11, 8), np.linspace(0, 1, 8)])
+    assert [g.tolist() for g in orc.top_k_across_heads(S, 8)] == [list(range(8)), []]
+    S = np.tile(rng.permutation(8).astype(float), (3, 1))
+    per_head = orc.top_k_indices(S[0], 3).tolist()
+    assert [g.tolist() for g in orc.top_k_across_heads(S, 9)] == [per_head] * 3
+
+
 # ----------------------------------------------------------------------------- compaction / whole unit
 def test_compact_and_compress_unit():
     import torch

@@ -193,6 +193,30 @@ int compactor_attention_scores(const compactor_shape* shape, compactor_mat q, co
                                float* attn_out, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Selection across the heads of a layer (Section 3.4 allows the top scores to be taken over all
+ * heads instead of within each head; the paper's experiments use such head-adaptive budgets).
+ * For every (layer, sequence b) the heads * keep_counts[b] largest scores over all heads are kept,
+ * ranked by (score descending, head ascending, index ascending), so heads keep different numbers
+ * of tokens while the layer keeps as many as per-head selection would.
+ *   idx_out           device int32 [layers][heads * total_keep]: layer l, sequence b owns entries
+ *                     [heads * cu_keep[b], heads * cu_keep[b+1]); inside that block head h owns
+ *                     [off[h], off[h+1]) with off = head_offsets_out[l][b][0 .. heads]; indices are
+ *                     local to the sequence and ascending within a head.
+ *   head_offsets_out  device int32 [layers][batch][heads + 1], off[0] = 0, off[heads] = heads * keep_counts[b].
+ * heads must not exceed 64.  Workspace: compactor_across_heads_workspace_bytes().
+ * compactor_compact_across_heads gathers K/V rows in exactly that order into
+ * k_out / v_out [layers][heads * total_keep][d] (bit copies; out-of-range indices are skipped).
+ */
+size_t compactor_across_heads_workspace_bytes(const compactor_shape* shape);
+int compactor_select_across_heads(const compactor_shape* shape, const float* scores,
+                                  const int32_t* keep_counts, int32_t* idx_out, int32_t* head_offsets_out,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+int compactor_compact_across_heads(const compactor_shape* shape, compactor_mat k_cache, compactor_mat v_cache,
+                                   const int32_t* idx, const int32_t* head_offsets,
+                                   const int32_t* keep_counts, void* k_out, void* v_out,
+                                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * compactor_score for callers that cannot allocate device memory (the paper has no counterpart;
  * this is a deployment convenience).  Same inputs, outputs and results as compactor_score, but
  * no workspace argument: the scratch is a fixed array of compactor_builtin_scratch_bytes()

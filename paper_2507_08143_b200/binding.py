@@ -54,6 +54,12 @@ def _load() -> ctypes.CDLL:
     lib.compactor_compress_profiled.argtypes = lib.compactor_compress.argtypes + [POINTER(c_void_p), c_int32]
     lib.compactor_attention_scores.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_int32, c_int32,
                                                c_float, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_across_heads_workspace_bytes.restype = c_size_t
+    lib.compactor_across_heads_workspace_bytes.argtypes = [POINTER(CompactorShape)]
+    lib.compactor_select_across_heads.argtypes = [POINTER(CompactorShape), c_void_p, POINTER(c_int32), c_void_p, c_void_p,
+                                                  c_void_p, c_size_t, c_void_p]
+    lib.compactor_compact_across_heads.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_void_p, c_void_p,
+                                                   POINTER(c_int32), c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.compactor_builtin_scratch_bytes.restype = c_size_t
     lib.compactor_score_builtin_scratch.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_void_p, c_float,
                                                     c_void_p, c_void_p, c_void_p]
@@ -66,7 +72,8 @@ LIB_PATH = _build.LIB
 EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_keep_count",
            "compactor_calibrated_ratio", "compactor_workspace_bytes", "compactor_score", "compactor_select",
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
-           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores"]
+           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores",
+           "compactor_across_heads_workspace_bytes", "compactor_select_across_heads", "compactor_compact_across_heads"]
 
 N_STAGE_EVENTS = 7
 STAGE_NAMES = ["gram", "factor", "score", "blend", "select", "compact"]
@@ -207,3 +214,22 @@ def attention_scores(shape: Shape, q: torch.Tensor, k: torch.Tensor, q_per_kv: i
     """Eq. 5: chunked non-causal attention column sums of `q` [layers, heads*q_per_kv, tokens, d] against `k`."""
     _check(LIB.compactor_attention_scores(byref(shape.c), mat(q), mat(k), q_per_kv, chunk, scale, pool, _ptr(attn_out),
                                           _ptr(workspace), workspace.numel(), _stream()), "compactor_attention_scores")
+
+
+def across_heads_workspace_bytes(shape: Shape) -> int:
+    return int(LIB.compactor_across_heads_workspace_bytes(byref(shape.c)))
+
+
+def select_across_heads(shape: Shape, scores: torch.Tensor, keep_counts: Sequence[int], idx_out: torch.Tensor,
+                        head_offsets_out: torch.Tensor, workspace: torch.Tensor) -> None:
+    _check(LIB.compactor_select_across_heads(byref(shape.c), _ptr(scores), _keep_array(keep_counts), _ptr(idx_out),
+                                             _ptr(head_offsets_out), _ptr(workspace), workspace.numel(), _stream()),
+           "compactor_select_across_heads")
+
+
+def compact_across_heads(shape: Shape, k_cache: torch.Tensor, v_cache: torch.Tensor, idx: torch.Tensor,
+                         head_offsets: torch.Tensor, keep_counts: Sequence[int], k_out: torch.Tensor,
+                         v_out: torch.Tensor, workspace: torch.Tensor) -> None:
+    _check(LIB.compactor_compact_across_heads(byref(shape.c), mat(k_cache), mat(v_cache), _ptr(idx), _ptr(head_offsets),
+                                              _keep_array(keep_counts), _ptr(k_out), _ptr(v_out), _ptr(workspace),
+                                              workspace.numel(), _stream()), "compactor_compact_across_heads")

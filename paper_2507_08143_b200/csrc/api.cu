@@ -422,3 +422,52 @@ extern "C" int compactor_attention_scores(const compactor_shape* shape, compacto
     CK(launch_attention(hp.plan, to_mat(q), to_mat(k), q_per_kv, scale, pool, raw, attn_out, st));
     return COMPACTOR_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Selection across the heads of a layer and the matching gather.
+extern "C" size_t compactor_across_heads_workspace_bytes(const compactor_shape* shape) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return 0;
+    return hp.off_w + align_up(sizeof(int32_t) * (size_t)shape->layers * shape->batch * (shape->heads + 1));
+}
+
+extern "C" int compactor_select_across_heads(const compactor_shape* shape, const float* scores,
+                                             const int32_t* keep_counts, int32_t* idx_out, int32_t* head_offsets_out,
+                                             void* workspace, size_t workspace_bytes, void* stream) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (shape->heads > 64) return COMPACTOR_E_UNSUPPORTED;
+    if (scores == nullptr || idx_out == nullptr || head_offsets_out == nullptr || workspace == nullptr ||
+        !set_keep(shape, keep_counts, &hp) || ((uintptr_t)workspace & 255) != 0)
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if ((long long)shape->heads * hp.plan.total_keep > 0x7fffffffLL) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (workspace_bytes < compactor_across_heads_workspace_bytes(shape)) return COMPACTOR_E_WORKSPACE;
+    if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CK(upload_tables(&hp, workspace, st));
+    char* ws = static_cast<char*>(workspace) + hp.off_w;
+    uint32_t* thr = reinterpret_cast<uint32_t*>(ws);                                  // [layers * batch]
+    int* ties = reinterpret_cast<int*>(ws) + (size_t)shape->layers * shape->batch;    // [layers * batch * heads]
+    CK(launch_select_across(hp.plan, scores, idx_out, head_offsets_out, thr, ties, st));
+    return COMPACTOR_OK;
+}
+
+extern "C" int compactor_compact_across_heads(const compactor_shape* shape, compactor_mat k_cache, compactor_mat v_cache,
+                                              const int32_t* idx, const int32_t* head_offsets,
+                                              const int32_t* keep_counts, void* k_out, void* v_out,
+                                              void* workspace, size_t workspace_bytes, void* stream) {
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (!mat_ok(k_cache) || !mat_ok(v_cache) || idx == nullptr || head_offsets == nullptr || k_out == nullptr ||
+        v_out == nullptr || workspace == nullptr || !set_keep(shape, keep_counts, &hp))
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if ((((uintptr_t)k_out | (uintptr_t)v_out) & 15) != 0 || ((uintptr_t)workspace & 255) != 0)
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (workspace_bytes < hp.off_w) return COMPACTOR_E_WORKSPACE;
+    if (hp.plan.total_keep == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CK(upload_tables(&hp, workspace, st));
+    CK(launch_compact_across(hp.plan, to_mat(k_cache), to_mat(v_cache), idx, head_offsets,
+                             static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
+    return COMPACTOR_OK;
+}

@@ -58,6 +58,10 @@ cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStre
 cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int* idx,
                            __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream);
 
+cudaError_t launch_select_across(const Plan& p, const float* scores, int* idx, int* head_offsets, uint32_t* thr,
+                                 int* ties, cudaStream_t stream);
+cudaError_t launch_compact_across(const Plan& p, const Mat& k, const Mat& v, const int* idx, const int* head_offsets,
+                                  __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream);
 cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_per_kv, float scale, int pool,
                              float* raw, float* out, cudaStream_t stream);
 

@@ -130,24 +130,13 @@ __device__ uint32_t radix_select(SelectSmem& s, int want, int* ties, Visit visit
     return prefix;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
-select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_out) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
-    const int unit = blockIdx.x;
-    const int b = unit % p.batch, lh = unit / p.batch;
-    const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
-    const int kk = p.cu_keep[b + 1] - p.cu_keep[b];
-    if (kk <= 0 || n <= 0) return;
-    const float* sc = scores + (size_t)lh * p.total_tokens + p.cu_seqlens[b];
-    int* out = idx_out + (size_t)lh * p.total_keep + p.cu_keep[b];
+// Key of the `want`-th largest of the values that `visit(f)` enumerates (f(value) is called once per
+// value, in any order, by any thread), and through *ties how many values equal to that key belong
+// to the top `want`.  `sample` / `n_sample` are some of the values, used to guess their range.
+template <class Visit>
+__device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __restrict__ sample, int n_sample,
+                                   int want_total, int* ties) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-    if (kk >= n) {
-        for (int i = tid; i < n; i += kThreads) out[i] = i;
-        return;
-    }
-
     // ---- value range from a sample ------------------------------------------------------------
     {
         float lo = INFINITY, hi = -INFINITY;
@@ -156,7 +145,7 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
 #pragma unroll
         for (int u = 0; u < kSample / kThreads; ++u) {
             const int i = u * kThreads + tid;
-            smp[u] = sc[i < n ? i : 0];
+            smp[u] = sample[i < n_sample ? i : 0];
         }
 #pragma unroll
         for (int u = 0; u < kSample / kThreads; ++u) {
@@ -183,9 +172,6 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
         __syncthreads();
     }
 
-    uint32_t thr = 0;
-    int ties = 0;
-    bool found = false;
     if (!s.fallback) {
         const float lo = s.lo, scale = s.scale;
         // monotone in v: subtraction, multiplication by a positive constant, clamping and truncation all are
@@ -196,37 +182,41 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
         for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
         __syncthreads();
         int nonfinite = 0;
-        for_each_score(sc, n, [&](float v) {
+        visit([&](float v) {
             if (!isfinite(v)) nonfinite = 1;
             atomicAdd(&s.hist[bin_of(v)], 1);
         });
         const int any_nonfinite = __syncthreads_or(nonfinite);
-        pick_bin(s, kBins, kk);
+        pick_bin(s, kBins, want_total);
         const int tbin = s.bin, want = s.remaining;
         const int members = s.hist[tbin];
         __syncthreads();
         if (!any_nonfinite && members <= kCand) {
-            for_each_score(sc, n, [&](float v) {
+            visit([&](float v) {
                 if (bin_of(v) == tbin) s.cand[atomicAdd(&s.n_cand, 1)] = order_key(v);
             });
             __syncthreads();
             const int nc = s.n_cand;
-            thr = radix_select(s, want, &ties, [&](auto tally) {
+            return radix_select(s, want, ties, [&](auto tally) {
                 for (int i = tid; i < nc; i += kThreads) tally(s.cand[i]);
             });
-            found = true;
         }
     }
-    if (!found)
-        thr = radix_select(s, kk, &ties, [&](auto tally) {
-            for_each_score(sc, n, [&](float v) { tally(order_key(v)); });
-        });
+    return radix_select(s, want_total, ties, [&](auto tally) {
+        visit([&](float v) { tally(order_key(v)); });
+    });
+}
 
-    // ---- ordered pass: positions from ballots and a scan of per-warp counts ---------------------
+// Ordered pass over one score vector: writes, ascending, the indices of the scores whose key exceeds
+// `thr` and of the first `ties` scores whose key equals it.  Positions come from warp ballots and one
+// scan of per-warp counts per 8192 scores; the next iteration's scores are loaded one iteration ahead.
+__device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n, uint32_t thr, int ties,
+                             int* __restrict__ out) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int base_gt = 0, base_eq = 0;          // counts over the elements before this iteration
     const uint32_t lt_mask = (1u << lane) - 1u;
     int it = 0;
-    float nxt[kSub];                       // scores of the next iteration, loaded one iteration ahead
+    float nxt[kSub];
 #pragma unroll
     for (int u = 0; u < kSub; ++u) {
         const int i = u * kThreads + tid;
@@ -278,6 +268,114 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
         base_gt += run & 0xffff;
         base_eq += run >> 16;
     }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_out) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    const int unit = blockIdx.x;
+    const int b = unit % p.batch, lh = unit / p.batch;
+    const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+    const int kk = p.cu_keep[b + 1] - p.cu_keep[b];
+    if (kk <= 0 || n <= 0) return;
+    const float* sc = scores + (size_t)lh * p.total_tokens + p.cu_seqlens[b];
+    int* out = idx_out + (size_t)lh * p.total_keep + p.cu_keep[b];
+    if (kk >= n) {
+        for (int i = threadIdx.x; i < n; i += kThreads) out[i] = i;
+        return;
+    }
+    int ties = 0;
+    const uint32_t thr = find_threshold(s, [&](auto f) { for_each_score(sc, n, f); }, sc, n, kk, &ties);
+    emit_ordered(s, sc, n, thr, ties, out);
+}
+
+// ---- selection across the heads of a layer (Section 3.4's alternative) -------------------------
+// Step 1, one CTA per (layer, sequence): the key of the (heads * kk)-th largest score over all heads,
+// how many scores each head keeps (ties go to the lower head first, then to the lower index), and
+// the heads' offsets inside the sequence's block of the output.
+__global__ void __launch_bounds__(kThreads, 1)
+across_threshold_kernel(Plan p, const float* __restrict__ scores, uint32_t* __restrict__ thr_out,
+                        int* __restrict__ ties_out, int* __restrict__ head_offsets) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    __shared__ int head_gt[64], head_eq[64];
+    const int layer = blockIdx.x / p.batch, b = blockIdx.x % p.batch;
+    const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+    const int kk = p.cu_keep[b + 1] - p.cu_keep[b];
+    const int H = p.heads, tid = threadIdx.x;
+    int* offs = head_offsets + ((size_t)layer * p.batch + b) * (H + 1);
+    int* ties_h = ties_out + ((size_t)layer * p.batch + b) * H;
+    const float* base = scores + (size_t)layer * H * p.total_tokens + p.cu_seqlens[b];
+    if (kk <= 0 || n <= 0) {
+        for (int h = tid; h <= H; h += kThreads) offs[h] = 0;
+        return;
+    }
+    if (kk >= n) {                                         // everything is kept
+        for (int h = tid; h <= H; h += kThreads) offs[h] = h * n;
+        for (int h = tid; h < H; h += kThreads) ties_h[h] = n;
+        if (tid == 0) thr_out[blockIdx.x] = 0u;           // every key is >= 0: all scores count as ties or above
+        return;
+    }
+    auto visit_all = [&](auto f) {
+        for (int h = 0; h < H; ++h) for_each_score(base + (size_t)h * p.total_tokens, n, f);
+    };
+    int ties = 0;
+    const uint32_t thr = find_threshold(s, visit_all, base, n, H * kk, &ties);
+    // per-head counts above and at the threshold
+    for (int h = tid; h < H; h += kThreads) { head_gt[h] = 0; head_eq[h] = 0; }
+    __syncthreads();
+    for (int h = 0; h < H; ++h) {
+        int gt = 0, eq = 0;
+        for_each_score(base + (size_t)h * p.total_tokens, n, [&](float v) {
+            const uint32_t key = order_key(v);
+            gt += key > thr; eq += key == thr;
+        });
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            gt += __shfl_xor_sync(0xffffffffu, gt, d);
+            eq += __shfl_xor_sync(0xffffffffu, eq, d);
+        }
+        if ((tid & 31) == 0) { atomicAdd(&head_gt[h], gt); atomicAdd(&head_eq[h], eq); }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int left = ties, off = 0;
+        for (int h = 0; h < H; ++h) {
+            const int take = min(left, head_eq[h]);
+            left -= take;
+            ties_h[h] = take;
+            offs[h] = off;
+            off += head_gt[h] + take;
+        }
+        offs[H] = off;
+        thr_out[blockIdx.x] = thr;
+    }
+}
+
+// Step 2, one CTA per (layer, head, sequence): the head's kept indices, ascending.
+__global__ void __launch_bounds__(kThreads, 1)
+across_emit_kernel(Plan p, const float* __restrict__ scores, const uint32_t* __restrict__ thr_in,
+                   const int* __restrict__ ties_in, const int* __restrict__ head_offsets, int* __restrict__ idx_out) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    const int unit = blockIdx.x;
+    const int b = unit % p.batch, lh = unit / p.batch;
+    const int layer = lh / p.heads, head = lh % p.heads;
+    const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+    const int kk = p.cu_keep[b + 1] - p.cu_keep[b];
+    if (kk <= 0 || n <= 0) return;
+    const size_t lb = (size_t)layer * p.batch + b;
+    const int off = head_offsets[lb * (p.heads + 1) + head];
+    const int count = head_offsets[lb * (p.heads + 1) + head + 1] - off;
+    if (count <= 0) return;
+    const float* sc = scores + (size_t)lh * p.total_tokens + p.cu_seqlens[b];
+    int* out = idx_out + (size_t)layer * p.heads * p.total_keep + (size_t)p.heads * p.cu_keep[b] + off;
+    if (kk >= n) {
+        for (int i = threadIdx.x; i < n; i += kThreads) out[i] = i;
+        return;
+    }
+    emit_ordered(s, sc, n, thr_in[lb], ties_in[lb * p.heads + head], out);
 }
 
 // Eq. 6: s = z(a) + lambda z(o), population standard deviation, per unit.  Overwrites the
@@ -341,6 +439,22 @@ cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStre
     cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     select_kernel<<<units, kThreads, smem, stream>>>(p, scores, idx);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_select_across(const Plan& p, const float* scores, int* idx, int* head_offsets, uint32_t* thr,
+                                 int* ties, cudaStream_t stream) {
+    const int units = p.layers * p.heads * p.batch;
+    if (units == 0 || p.heads > 64) return units == 0 ? cudaSuccess : cudaErrorInvalidValue;
+    const int smem = (int)sizeof(SelectSmem);
+    cudaError_t e = cudaFuncSetAttribute(across_threshold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(across_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    across_threshold_kernel<<<p.layers * p.batch, kThreads, smem, stream>>>(p, scores, thr, ties, head_offsets);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    across_emit_kernel<<<units, kThreads, smem, stream>>>(p, scores, thr, ties, head_offsets, idx);
     return cudaGetLastError();
 }
 

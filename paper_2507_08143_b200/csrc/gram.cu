@@ -6,10 +6,11 @@
 // six-stage ring of shared memory with TMA (two 64-channel boxes per tile, 128-byte swizzle); one
 // thread issues tcgen05.mma with the same tile as both operands (the token axis is the
 // contraction axis, so both are MN-major) into one of two 128 x 128 fp32 accumulators in tensor
-// memory.  Every 2048 tokens the accumulator is handed to eight epilogue warps, which add it
+// memory.  Every 512 tokens the accumulator is handed to eight epilogue warps, which add it
 // into fp64 registers (64 columns of one row per thread) while the other accumulator fills; the
 // fp64 sums go to global memory once, at the end of the block.  So no fp32 sum is longer than
-// 2048 tokens, whatever the block length.
+// 512 tokens, whatever the block length: the tensor-core accumulator loses accuracy in proportion
+// to the length of the run.
 #include "common.cuh"
 #include "sm100.cuh"
 

@@ -85,6 +85,17 @@ const char* compactor_error_string(int code);
 int compactor_make_sketch(uint64_t seed, int32_t d, int32_t m, float* phi_host);
 
 /*
+ * Appendix D: a subsampled randomised Hadamard sketch, written out as a matrix Phi [d][m] (HOST,
+ * row-major fp32) that the scoring calls take like any other sketch: Phi = (1/sqrt(m)) D H R^T with
+ * D random signs, H the Sylvester-Walsh-Hadamard matrix of order d (d a power of two) and R a
+ * choice of m columns without replacement.  Random bits come from the splitmix64 stream of
+ * compactor_make_sketch: word i (i < d) gives the sign of row i (bit 0 set = minus); word d + j
+ * drives step j of a Fisher-Yates shuffle of 0..d-1 (swap position j with j + word mod (d - j)),
+ * whose first m entries are the chosen columns.
+ */
+int compactor_make_sketch_srht(uint64_t seed, int32_t d, int32_t m, float* phi_host);
+
+/*
  * Number of retained tokens for a sequence of n tokens at retention ratio r (Section 3,
  * Preliminaries: k = ceil(r N)): ceil evaluated on the double product, clamped to [1, n];
  * 0 when n <= 0.  Returns the count (never an error code).

@@ -95,6 +95,34 @@ def make_sketch(seed: int, d: int, m: int) -> np.ndarray:
     return (out[:count] / math.sqrt(m)).astype(np.float32).reshape(d, m)
 
 
+def make_sketch_srht(seed: int, d: int, m: int) -> np.ndarray:
+    """Appendix D: subsampled randomised Hadamard sketch Phi = c * D H R^T as an explicit [d, m] matrix
+    (D random signs, H the Sylvester-Walsh-Hadamard matrix, R a choice of m columns without
+    replacement).  The constant is 1/sqrt(m), which gives entries the variance of the Gaussian
+    sketch; scores do not depend on it.  Random bits come from the same splitmix64 stream as
+    `make_sketch`: word i (i < d) gives the sign of row i (bit 0: 1 = minus); word d + j drives step
+    j of a Fisher-Yates shuffle of 0..d-1 whose first m entries are the chosen columns."""
+    assert d & (d - 1) == 0 and 1 <= m <= d
+    mask = (1 << 64) - 1
+
+    def word(i):
+        z = (seed + (i + 1) * 0x9E3779B97F4A7C15) & mask
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & mask
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & mask
+        return z ^ (z >> 31)
+
+    sign = np.array([-1.0 if word(i) & 1 else 1.0 for i in range(d)])
+    perm = list(range(d))
+    for j in range(m):
+        r = j + word(d + j) % (d - j)
+        perm[j], perm[r] = perm[r], perm[j]
+    H = np.array([[1.0]])
+    while H.shape[0] < d:
+        H = np.block([[H, H], [H, -H]])
+    Phi = (sign[:, None] * H[:, perm[:m]]) / math.sqrt(m)
+    return Phi.astype(np.float32)
+
+
 # ----------------------------------------------------------------------------
 # Definition 1 / Eq. 1: exact leverage scores
 # ----------------------------------------------------------------------------

@@ -37,6 +37,7 @@ def _load() -> ctypes.CDLL:
     lib.compactor_error_string.restype = c_char_p
     lib.compactor_error_string.argtypes = [ctypes.c_int]
     lib.compactor_make_sketch.argtypes = [c_uint64, c_int32, c_int32, POINTER(c_float)]
+    lib.compactor_make_sketch_srht.argtypes = [c_uint64, c_int32, c_int32, POINTER(c_float)]
     lib.compactor_keep_count.restype = c_int64
     lib.compactor_keep_count.argtypes = [c_int64, c_double]
     lib.compactor_calibrated_ratio.argtypes = [c_double, c_double, c_double, c_double, POINTER(c_double)]
@@ -69,7 +70,7 @@ def _load() -> ctypes.CDLL:
 LIB = _load()
 LIB_PATH = _build.LIB
 
-EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_keep_count",
+EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_make_sketch_srht", "compactor_keep_count",
            "compactor_calibrated_ratio", "compactor_workspace_bytes", "compactor_score", "compactor_select",
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
            "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores",
@@ -132,6 +133,13 @@ def _keep_array(keep_counts: Sequence[int]):
 def make_sketch(seed: int, d: int, m: int) -> torch.Tensor:
     out = torch.empty(d, m, dtype=torch.float32)
     _check(LIB.compactor_make_sketch(seed, d, m, ctypes.cast(out.data_ptr(), POINTER(c_float))), "compactor_make_sketch")
+    return out
+
+
+def make_sketch_srht(seed: int, d: int, m: int) -> torch.Tensor:
+    out = torch.empty(d, m, dtype=torch.float32)
+    _check(LIB.compactor_make_sketch_srht(seed, d, m, ctypes.cast(out.data_ptr(), POINTER(c_float))),
+           "compactor_make_sketch_srht")
     return out
 
 

@@ -471,3 +471,30 @@ extern "C" int compactor_compact_across_heads(const compactor_shape* shape, comp
                              static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
     return COMPACTOR_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Appendix D: the subsampled randomised Hadamard sketch as an explicit matrix (host helper).
+extern "C" int compactor_make_sketch_srht(uint64_t seed, int32_t d, int32_t m, float* phi_host) {
+    if (phi_host == nullptr || d < 1 || (d & (d - 1)) != 0 || m < 1 || m > d) return COMPACTOR_E_INVALID_ARGUMENT;
+    auto word = [seed](uint64_t i) {
+        uint64_t z = seed + (i + 1) * 0x9E3779B97F4A7C15ull;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+        return z ^ (z >> 31);
+    };
+    std::vector<int> perm(d);
+    for (int i = 0; i < d; ++i) perm[i] = i;
+    for (int j = 0; j < m; ++j) {
+        const int r = j + (int)(word((uint64_t)d + j) % (uint64_t)(d - j));
+        const int tmp = perm[j]; perm[j] = perm[r]; perm[r] = tmp;
+    }
+    const float mag = (float)(1.0 / sqrt((double)m));
+    for (int i = 0; i < d; ++i) {
+        const bool minus_row = (word((uint64_t)i) & 1ull) != 0;
+        for (int j = 0; j < m; ++j) {
+            const bool minus_h = (__builtin_popcount((unsigned)(i & perm[j])) & 1) != 0;   // Sylvester: H[i][c] = (-1)^popcount(i & c)
+            phi_host[(size_t)i * m + j] = (minus_row != minus_h) ? -mag : mag;
+        }
+    }
+    return COMPACTOR_OK;
+}

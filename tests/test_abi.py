@@ -55,6 +55,13 @@ def test_make_sketch_matches_oracle_generator():
     assert abs(z.mean()) < 0.05 and abs(z.std() - 1) < 0.05
 
 
+def test_srht_sketch_matches_oracle_generator():
+    for seed, d, m in ((0, 128, 48), (9, 128, 64), (3, 16, 16), (4, 8, 1)):
+        np.testing.assert_array_equal(B.make_sketch_srht(seed, d, m).numpy(), orc.make_sketch_srht(seed, d, m))
+    with pytest.raises(B.CompactorError):
+        B.make_sketch_srht(0, 96, 48)                     # the Hadamard order must be a power of two
+
+
 def test_workspace_bytes():
     small = B.workspace_bytes(B.Shape(1, 2, 128, 48, [1024]))
     big = B.workspace_bytes(B.Shape(64, 8, 128, 48, [131072]))

@@ -61,6 +61,18 @@ def test_other_sketch_dimensions(B, m):
     _run_workload(B, w, mode="aliased", device="cpu")
 
 
+def test_srht_sketch(B):
+    # Appendix D's sketch is just another Phi for the same kernels
+    w = inputs.Workload("srht", 1, 2, 128, [3000, 900], [0.3, 0.5], p=1.0, seed=27)
+    kp, kr, v = [t.cuda() for t in inputs.make_tensors(w, device="cpu")]
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    phi = B.make_sketch_srht(11, w.d, w.m)
+    keep = _keep(B, w)
+    outs = H.run_compress(B, shape, kp, kr, v, phi, keep)
+    worst, _ = H.compare_all_units(shape, keep, outs, kp, kr, v, phi, what="srht")
+    print(f"srht sketch: max rel score err {worst:.2e}")
+
+
 def test_token_major_layout(B):
     # [layers, tokens, heads, d] storage (the layout of a serving engine's cache), passed by strides
     w = inputs.Workload("token-major", 2, 3, 128, [900, 411], [0.3, 0.6], p=0.7, seed=31)

@@ -165,6 +165,18 @@ def test_make_sketch_statistics_and_determinism():
     assert x == 0xE220A8397B1DCDAF
 
 
+def test_srht_sketch_structure():
+    P = orc.make_sketch_srht(5, 128, 48).astype(np.float64)
+    assert P.shape == (128, 48)
+    np.testing.assert_allclose(np.abs(P), 1 / math.sqrt(48))                  # entries are +-1/sqrt(m)
+    np.testing.assert_allclose(P.T @ P, (128 / 48) * np.eye(48), atol=1e-9)    # distinct Hadamard columns are orthogonal
+    assert not np.array_equal(P, orc.make_sketch_srht(6, 128, 48))
+    # m = d: D H R^T is a scaled orthogonal matrix, so Algorithm 1 returns the exact leverage scores
+    K = _rng(14).standard_normal((300, 16)) * (np.arange(1, 17) ** -1.0)
+    np.testing.assert_allclose(orc.approx_leverage_scores(K, orc.make_sketch_srht(1, 16, 16)),
+                               orc.exact_leverage_scores(K), rtol=1e-8)
+
+
 # ----------------------------------------------------------------------------- attention term (Eq. 5)
 def test_attention_scores_pins():
     import torch

@@ -250,6 +250,16 @@ int compactor_score_builtin_scratch(const compactor_shape* shape, compactor_mat 
                                     const float* attn_scores, float lambda, float* scores_out,
                                     int32_t* status, void* stream);
 
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper).  Enqueues a one-warp
+ * kernel that waits, with a limit of about a millisecond, once on a barrier that completes and
+ * once on a barrier that nothing completes, through the same wait routine the streaming kernels
+ * use.  status_out (device int32[1]) receives COMPACTOR_STATUS_TIMEOUT (4) when the first wait
+ * succeeded and the second gave up as designed; any other value is a defect.  The context stays
+ * usable: nothing traps or hangs.
+ */
+int compactor_wait_selftest(int32_t* status_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -61,6 +61,7 @@ def _load() -> ctypes.CDLL:
                                                   c_void_p, c_size_t, c_void_p]
     lib.compactor_compact_across_heads.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_void_p, c_void_p,
                                                    POINTER(c_int32), c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_wait_selftest.argtypes = [c_void_p, c_void_p]
     lib.compactor_builtin_scratch_bytes.restype = c_size_t
     lib.compactor_score_builtin_scratch.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_void_p, c_float,
                                                     c_void_p, c_void_p, c_void_p]
@@ -73,7 +74,7 @@ LIB_PATH = _build.LIB
 EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_make_sketch_srht", "compactor_keep_count",
            "compactor_calibrated_ratio", "compactor_workspace_bytes", "compactor_score", "compactor_select",
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
-           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores",
+           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores", "compactor_wait_selftest",
            "compactor_across_heads_workspace_bytes", "compactor_select_across_heads", "compactor_compact_across_heads"]
 
 N_STAGE_EVENTS = 7
@@ -241,3 +242,11 @@ def compact_across_heads(shape: Shape, k_cache: torch.Tensor, v_cache: torch.Ten
     _check(LIB.compactor_compact_across_heads(byref(shape.c), mat(k_cache), mat(v_cache), _ptr(idx), _ptr(head_offsets),
                                               _keep_array(keep_counts), _ptr(k_out), _ptr(v_out), _ptr(workspace),
                                               workspace.numel(), _stream()), "compactor_compact_across_heads")
+
+
+def wait_selftest() -> int:
+    """Runs the bounded-wait self-test and returns the status word (4 = the wait gave up as designed)."""
+    out = torch.full((1,), -1, dtype=torch.int32, device="cuda")
+    _check(LIB.compactor_wait_selftest(_ptr(out), _stream()), "compactor_wait_selftest")
+    torch.cuda.synchronize()
+    return int(out.item())

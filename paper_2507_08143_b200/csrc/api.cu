@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "sm100.cuh"
 
 using namespace compactor;
 
@@ -497,4 +498,32 @@ extern "C" int compactor_make_sketch_srht(uint64_t seed, int32_t d, int32_t m, f
         }
     }
     return COMPACTOR_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded waits.  Every spin of the streaming kernels goes through
+// sm100::mbar_wait, which gives up after a cycle limit and lets the kernel report
+// COMPACTOR_STATUS_TIMEOUT instead of hanging the device.  This entry point runs that same wait on
+// a barrier that nothing will ever complete, with a limit of about one millisecond, and writes what
+// the wait returned, so that the give-up path can be exercised without faulting or hanging a GPU.
+namespace {
+__global__ void wait_selftest_kernel(int* status_out, long long limit_cycles) {
+    __shared__ uint64_t never;
+    __shared__ uint64_t once;
+    if (threadIdx.x == 0) {
+        compactor::sm100::mbar_init(&never, 1);
+        compactor::sm100::mbar_init(&once, 1);
+        compactor::sm100::fence_barrier_init();
+        compactor::sm100::mbar_arrive(&once);                                  // this one does complete
+        const bool completed = compactor::sm100::mbar_wait(&once, 0, limit_cycles);
+        const bool hung = compactor::sm100::mbar_wait(&never, 0, limit_cycles);   // runs out
+        status_out[0] = (completed ? 0 : 8) | (hung ? 0 : COMPACTOR_STATUS_TIMEOUT);
+    }
+}
+}  // namespace
+
+extern "C" int compactor_wait_selftest(int32_t* status_out, void* stream) {
+    if (status_out == nullptr) return COMPACTOR_E_INVALID_ARGUMENT;
+    wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status_out, 2000000LL);
+    return cudaGetLastError() == cudaSuccess ? COMPACTOR_OK : COMPACTOR_E_CUDA;
 }

@@ -224,3 +224,11 @@ def test_c3_long_context_units(B):
     w.heads = 2
     worst, band, _ = _run_workload(B, w, mode="paper", device="cuda")
     print(f"c3 (n=131072, 2 units): max rel score err {worst:.2e}, boundary band {band}")
+
+
+def test_bounded_wait_gives_up_and_context_survives(B):
+    # failure detection without a fault: a wait that nothing satisfies returns after its limit
+    assert B.wait_selftest() == 4
+    x = torch.ones(8, device="cuda")
+    assert float(x.sum()) == 8.0                       # the context is still usable
+    assert B.wait_selftest() == 4

@@ -110,6 +110,18 @@ int64_t compactor_keep_count(int64_t n, double r);
 int compactor_calibrated_ratio(double nll, double alpha, double beta, double tau, double* r_out);
 
 /*
+ * Fit of the calibration curve (Section 3.5): finds (alpha, beta) minimising the asymmetric mean
+ * squared error sum_i w_i (f_{alpha,beta}(r_i, nll_i) - y_i)^2 / n over n training triples, where
+ * f is the curve of compactor_calibrated_ratio with b = alpha*nll_i + beta, y_i is the measured
+ * NLL ratio at retention r_i, and w_i = under_weight (>= 1) when the curve predicts more quality
+ * than was measured (which would make r* too small), else 1; the paper weights those errors
+ * higher without giving the weight.  Host arrays, host computation (Levenberg-Marquardt from a
+ * grid of starting points); loss_out may be NULL.
+ */
+int compactor_fit_calibration(int64_t n, const double* r, const double* nll, const double* y,
+                              double under_weight, double* alpha_out, double* beta_out, double* loss_out);
+
+/*
  * Bytes of device workspace that compactor_score and compactor_compress need for this shape.
  * compactor_select and compactor_compact only use a small table at its start and accept any
  * workspace of at least 12*(batch+1) bytes rounded up to 256.  The workspace must be 256-byte

@@ -22,7 +22,8 @@ What follows the paper step by step:
     (Section 3.4's alternative; ties: lower head, then lower index).
   * `compact`                - the retained rows of K and V.
   * `calibrated_ratio`       - inverse of the fitted curve f_{alpha,beta}
-    (Section 3.5).
+    (Section 3.5); `fit_calibration` - the asymmetric least-squares fit of
+    (alpha, beta) on (r, NLL, y) triples.
 
 Readings taken where the paper is silent or inconsistent:
   * Eq. 1 prints diag(U^T U); Definition 1 and Algorithm 1's last line make it
@@ -278,6 +279,33 @@ def calibrated_ratio(nll: float, alpha: float, beta: float, tau: float) -> float
     if b == 0.0:
         return float(tau)
     return math.log1p(float(tau) * math.expm1(b)) / b
+
+
+def calibration_loss(alpha: float, beta: float, r, nll, y, under_weight: float = 1.0) -> float:
+    """Asymmetric mean squared error of the fitted curve (Section 3.5): residual e_i =
+    f_{alpha,beta}(r_i, NLL_i) - y_i; a positive residual predicts more quality than was measured,
+    which would make r* too small, and is weighted by `under_weight` >= 1 (the paper says such
+    errors are weighted higher but not by how much)."""
+    r = np.asarray(r, dtype=np.float64); nll = np.asarray(nll, dtype=np.float64); y = np.asarray(y, dtype=np.float64)
+    total = 0.0
+    for ri, ci, yi in zip(r, nll, y):
+        e = calibration_curve(float(ri), alpha * float(ci) + beta) - float(yi)
+        total += (under_weight if e > 0.0 else 1.0) * e * e
+    return total / max(1, r.size)
+
+
+def fit_calibration(r, nll, y, under_weight: float = 1.0):
+    """(alpha, beta) minimising `calibration_loss` over the training triples (r_i, NLL_i, y_i): a
+    derivative-free simplex search from a coarse grid of starting points (slow and plain)."""
+    from scipy.optimize import minimize
+    best = None
+    for a0 in (-4.0, -1.0, 0.0, 1.0):
+        for b0 in (-6.0, -2.0, 0.5):
+            res = minimize(lambda p: calibration_loss(p[0], p[1], r, nll, y, under_weight), x0=[a0, b0],
+                           method="Nelder-Mead", options={"xatol": 1e-10, "fatol": 1e-16, "maxiter": 4000})
+            if best is None or res.fun < best.fun:
+                best = res
+    return float(best.x[0]), float(best.x[1]), float(best.fun)
 
 
 # ----------------------------------------------------------------------------

@@ -41,6 +41,8 @@ def _load() -> ctypes.CDLL:
     lib.compactor_keep_count.restype = c_int64
     lib.compactor_keep_count.argtypes = [c_int64, c_double]
     lib.compactor_calibrated_ratio.argtypes = [c_double, c_double, c_double, c_double, POINTER(c_double)]
+    lib.compactor_fit_calibration.argtypes = [c_int64, POINTER(c_double), POINTER(c_double), POINTER(c_double), c_double,
+                                              POINTER(c_double), POINTER(c_double), POINTER(c_double)]
     lib.compactor_workspace_bytes.restype = c_size_t
     lib.compactor_workspace_bytes.argtypes = [POINTER(CompactorShape)]
     lib.compactor_score.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_void_p, c_float, c_void_p,
@@ -72,7 +74,7 @@ LIB = _load()
 LIB_PATH = _build.LIB
 
 EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_make_sketch_srht", "compactor_keep_count",
-           "compactor_calibrated_ratio", "compactor_workspace_bytes", "compactor_score", "compactor_select",
+           "compactor_calibrated_ratio", "compactor_fit_calibration", "compactor_workspace_bytes", "compactor_score", "compactor_select",
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
            "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores", "compactor_wait_selftest",
            "compactor_across_heads_workspace_bytes", "compactor_select_across_heads", "compactor_compact_across_heads"]
@@ -152,6 +154,16 @@ def calibrated_ratio(nll: float, alpha: float, beta: float, tau: float) -> float
     r = c_double()
     _check(LIB.compactor_calibrated_ratio(nll, alpha, beta, tau, byref(r)), "compactor_calibrated_ratio")
     return r.value
+
+
+def fit_calibration(r: Sequence[float], nll: Sequence[float], y: Sequence[float], under_weight: float = 1.0):
+    """Returns (alpha, beta, loss) of the asymmetric least-squares fit of the calibration curve."""
+    n = len(r)
+    arr = lambda v: (c_double * n)(*[float(x) for x in v])
+    al, be, loss = c_double(), c_double(), c_double()
+    _check(LIB.compactor_fit_calibration(n, arr(r), arr(nll), arr(y), under_weight, byref(al), byref(be), byref(loss)),
+           "compactor_fit_calibration")
+    return al.value, be.value, loss.value
 
 
 def workspace_bytes(shape: Shape) -> int:

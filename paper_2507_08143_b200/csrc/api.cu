@@ -527,3 +527,73 @@ extern "C" int compactor_wait_selftest(int32_t* status_out, void* stream) {
     wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(status_out, 2000000LL);
     return cudaGetLastError() == cudaSuccess ? COMPACTOR_OK : COMPACTOR_E_CUDA;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Section 3.5: fit of the calibration curve's two parameters (host helper).
+namespace {
+
+double curve(double r, double b) {                  // f(r) = (e^{br} - 1) / (e^b - 1), f = r at b = 0
+    if (fabs(b) < 1e-8) return r + 0.5 * b * r * (r - 1.0);
+    return expm1(b * r) / expm1(b);
+}
+double curve_db(double r, double b) {               // d f / d b
+    if (fabs(b) < 1e-4) return 0.5 * r * (r - 1.0) + b * r * (r - 1.0) * (2.0 * r - 1.0) / 6.0;
+    const double eb = expm1(b), er = expm1(b * r);
+    return (r * (er + 1.0) * eb - er * (eb + 1.0)) / (eb * eb);
+}
+double fit_loss(long long n, const double* r, const double* c, const double* y, double w_under, double al, double be) {
+    double s = 0.0;
+    for (long long i = 0; i < n; ++i) {
+        const double e = curve(r[i], al * c[i] + be) - y[i];
+        s += (e > 0.0 ? w_under : 1.0) * e * e;
+    }
+    return s / (double)n;
+}
+
+}  // namespace
+
+extern "C" int compactor_fit_calibration(int64_t n, const double* r, const double* nll, const double* y,
+                                         double under_weight, double* alpha_out, double* beta_out, double* loss_out) {
+    if (n < 2 || r == nullptr || nll == nullptr || y == nullptr || alpha_out == nullptr || beta_out == nullptr ||
+        !(under_weight >= 1.0))
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    double best = 1e300, best_a = 0.0, best_b = 0.0;
+    const double a_starts[4] = {-4.0, -1.0, 0.0, 1.0}, b_starts[3] = {-6.0, -2.0, 0.5};
+    for (double a0 : a_starts)
+        for (double b0 : b_starts) {
+            // Levenberg-Marquardt on (alpha, beta); the asymmetric weights are those of the current residuals
+            double al = a0, be = b0, mu = 1e-3, cur = fit_loss(n, r, nll, y, under_weight, al, be);
+            for (int iter = 0; iter < 500; ++iter) {
+                double jaa = 0, jab = 0, jbb = 0, ga = 0, gb = 0;
+                for (long long i = 0; i < n; ++i) {
+                    const double b = al * nll[i] + be;
+                    const double e = curve(r[i], b) - y[i];
+                    const double w = e > 0.0 ? under_weight : 1.0;
+                    const double db = curve_db(r[i], b), da = db * nll[i];
+                    jaa += w * da * da; jab += w * da * db; jbb += w * db * db;
+                    ga += w * da * e; gb += w * db * e;
+                }
+                bool improved = false;
+                for (int tries = 0; tries < 30 && !improved; ++tries) {
+                    const double haa = jaa * (1.0 + mu) + 1e-300, hbb = jbb * (1.0 + mu) + 1e-300;
+                    const double det = haa * hbb - jab * jab;
+                    if (!(fabs(det) > 0.0)) { mu *= 10.0; continue; }
+                    const double sa = -(hbb * ga - jab * gb) / det, sb = -(haa * gb - jab * ga) / det;
+                    const double trial = fit_loss(n, r, nll, y, under_weight, al + sa, be + sb);
+                    if (trial < cur) {
+                        al += sa; be += sb; improved = true;
+                        const bool tiny = fabs(sa) + fabs(sb) < 1e-13 || cur - trial < 1e-18 * (1.0 + cur);
+                        cur = trial; mu = fmax(mu * 0.3, 1e-12);
+                        if (tiny) iter = 500;
+                    } else {
+                        mu *= 10.0;
+                    }
+                }
+                if (!improved) break;
+            }
+            if (cur < best) { best = cur; best_a = al; best_b = be; }
+        }
+    *alpha_out = best_a; *beta_out = best_b;
+    if (loss_out != nullptr) *loss_out = best;
+    return COMPACTOR_OK;
+}

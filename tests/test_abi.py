@@ -45,6 +45,23 @@ def test_calibrated_ratio_matches_oracle():
         B.calibrated_ratio(1.0, 1.0, 0.0, 1.5)
 
 
+def test_fit_calibration_matches_oracle():
+    rng = np.random.default_rng(21)
+    nll = rng.uniform(0.5, 3.0, 80); r = rng.uniform(0.05, 1.0, 80)
+    y_true = np.array([orc.calibration_curve(ri, -1.7 * ci - 0.8) for ri, ci in zip(r, nll)])
+    a, b, loss = B.fit_calibration(r, nll, y_true)
+    assert abs(a + 1.7) < 1e-6 and abs(b + 0.8) < 1e-6 and loss < 1e-20            # noise-free: exact recovery
+    y = np.clip(y_true + 0.05 * rng.standard_normal(80), 0, 1)
+    for w in (1.0, 4.0):
+        a, b, loss = B.fit_calibration(r, nll, y, under_weight=w)
+        ao, bo, lo = orc.fit_calibration(r, nll, y, under_weight=w)
+        assert abs(loss - orc.calibration_loss(a, b, r, nll, y, w)) < 1e-12       # same objective
+        assert loss <= lo * (1 + 1e-6) + 1e-15                                      # at least as good as the oracle's search
+        assert abs(a - ao) < 2e-3 and abs(b - bo) < 2e-3
+    with pytest.raises(B.CompactorError):
+        B.fit_calibration([0.5], [1.0], [0.5])
+
+
 def test_make_sketch_matches_oracle_generator():
     for seed, d, m in ((0, 128, 48), (12345, 128, 64), (7, 5, 3)):
         got = B.make_sketch(seed, d, m).numpy()

@@ -261,6 +261,26 @@ def test_calibrated_ratio():
     assert orc.calibrated_ratio(1.0, -10, 0, 0.95) < orc.calibrated_ratio(1.0, -4, 0, 0.95)
 
 
+def test_fit_calibration_recovers_known_parameters():
+    rng = _rng(15)
+    alpha, beta = -1.7, -0.8
+    nll = rng.uniform(0.5, 3.0, 60); r = rng.uniform(0.05, 1.0, 60)
+    y = np.array([orc.calibration_curve(ri, alpha * ci + beta) for ri, ci in zip(r, nll)])
+    a, b, loss = orc.fit_calibration(r, nll, y)
+    assert abs(a - alpha) < 1e-4 and abs(b - beta) < 1e-4 and loss < 1e-12     # noise-free triples: exact recovery
+    assert orc.calibration_loss(alpha, beta, r, nll, y) < 1e-30
+    # with noise, weighting over-predicted quality more moves the curve down: larger r* for the same tau
+    y_noisy = np.clip(y + 0.05 * rng.standard_normal(60), 0.0, 1.0)
+    a1, b1, _ = orc.fit_calibration(r, nll, y_noisy, under_weight=1.0)
+    a4, b4, _ = orc.fit_calibration(r, nll, y_noisy, under_weight=8.0)
+    r1 = np.mean([orc.calibrated_ratio(c, a1, b1, 0.9) for c in (1.0, 2.0)])
+    r4 = np.mean([orc.calibrated_ratio(c, a4, b4, 0.9) for c in (1.0, 2.0)])
+    assert r4 > r1
+    # the loss counts a positive residual `under_weight` times
+    assert abs(orc.calibration_loss(0.0, 0.0, [0.5], [1.0], [0.4], 3.0) - 3.0 * 0.01) < 1e-12
+    assert abs(orc.calibration_loss(0.0, 0.0, [0.5], [1.0], [0.6], 3.0) - 0.01) < 1e-12
+
+
 # ----------------------------------------------------------------------------- top-k
 def _brute_topk(s, kk):
     order = sorted(range(len(s)), key=lambda i: (-s[i], i))

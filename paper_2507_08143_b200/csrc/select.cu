@@ -21,7 +21,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kBins = 2048;
 constexpr int kSample = 4096;          // scores used to estimate the value range
 constexpr int kCand = 8192;            // capacity of the candidate list
-constexpr int kSub = 8;                // 1024-element sub-blocks per iteration of the ordered pass
+constexpr int kSub = 8;                // rows of the small shared count table
 
 // Monotone map float -> uint32: larger float <=> larger key; -0 and +0 share a key (adding +0
 // turns -0 into +0) and a NaN with the sign bit clear ranks highest.
@@ -208,65 +208,119 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
 }
 
 // Ordered pass over one score vector: writes, ascending, the indices of the scores whose key exceeds
-// `thr` and of the first `ties` scores whose key equals it.  Positions come from warp ballots and one
-// scan of per-warp counts per 8192 scores; the next iteration's scores are loaded one iteration ahead.
+// `thr` and of the first `ties` scores whose key equals it.  The vector is cut into an unaligned
+// head (0-3 scores), a 16-byte aligned body and a tail (0-3 scores).  Every warp owns a contiguous
+// stretch of the body, read as float4 (four consecutive scores per lane): it first counts its
+// scores above and at the threshold, one block-wide scan turns the counts into output offsets, and
+// then each warp emits its stretch on its own (a shuffle scan of per-lane counts per 128 scores).
+// The pass is bound by instruction issue, hence four scores per load and per scan.
 __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n, uint32_t thr, int ties,
                              int* __restrict__ out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    int base_gt = 0, base_eq = 0;          // counts over the elements before this iteration
-    const uint32_t lt_mask = (1u << lane) - 1u;
-    int it = 0;
-    float nxt[kSub];
-#pragma unroll
-    for (int u = 0; u < kSub; ++u) {
-        const int i = u * kThreads + tid;
-        nxt[u] = (i < n) ? sc[i] : 0.f;
+    const int head = min(n, (int)((4 - ((reinterpret_cast<uintptr_t>(sc) >> 2) & 3)) & 3));
+    const int n_vec = (n - head) >> 2;
+    const int tail_begin = head + 4 * n_vec;
+    const float4* body = reinterpret_cast<const float4*>(sc + head);
+    const int per_warp = (((n_vec + kWarps - 1) / kWarps) + 31) & ~31;   // vectors per stretch, a multiple of 32
+    const int vbegin = min(n_vec, warp * per_warp), vend = min(n_vec, vbegin + per_warp);
+    constexpr int kAhead = 4;                                             // vector steps loaded together
+
+    auto flags = [&](const float4& q, int& g, int& e) {                   // 4-bit masks: above / at the threshold
+        const uint32_t k0 = order_key(q.x), k1 = order_key(q.y), k2 = order_key(q.z), k3 = order_key(q.w);
+        g = (k0 > thr) | ((k1 > thr) << 1) | ((k2 > thr) << 2) | ((k3 > thr) << 3);
+        e = (k0 == thr) | ((k1 == thr) << 1) | ((k2 == thr) << 2) | ((k3 == thr) << 3);
+    };
+
+    // ---- counts: head (warp 0), the warp's stretch, tail (last warp) ----------------------------
+    int head_gt = 0, head_eq = 0;                       // head scores precede everything; every thread counts them
+    for (int i = 0; i < head; ++i) {
+        const uint32_t key = order_key(sc[i]);
+        head_gt += key > thr; head_eq += key == thr;
     }
-    for (int start = 0; start < n; start += kThreads * kSub, ++it) {
-        const int buf = it & 1;
-        uint32_t keys[kSub], bg[kSub], be[kSub];
+    int cnt = 0;                                        // packed: above | at << 16
+    for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
+        float4 q[kAhead];
 #pragma unroll
-        for (int u = 0; u < kSub; ++u) keys[u] = order_key(nxt[u]);
-#pragma unroll
-        for (int u = 0; u < kSub; ++u) {
-            const int i = start + kThreads * kSub + u * kThreads + tid;
-            nxt[u] = (i < n) ? sc[i] : 0.f;
+        for (int u = 0; u < kAhead; ++u) {
+            const int vi = v0 + u * 32 + lane;
+            q[u] = vi < vend ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int u = 0; u < kSub; ++u) {
-            const int i = start + u * kThreads + tid;
-            bg[u] = __ballot_sync(0xffffffffu, i < n && keys[u] > thr);
-            be[u] = __ballot_sync(0xffffffffu, i < n && keys[u] == thr);
-            if (lane == 0) s.cnt[buf][u][warp] = __popc(bg[u]) | (__popc(be[u]) << 16);
+        for (int u = 0; u < kAhead; ++u) {
+            int g, e;
+            flags(q[u], g, e);
+            if (v0 + u * 32 + lane < vend) cnt += __popc(g) | (__popc(e) << 16);
         }
-        __syncthreads();
-        if (warp < kSub) {
-            const int v = s.cnt[buf][warp][lane];
-            int incl = v;
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+    __syncthreads();                                    // earlier users of the shared arrays are done
+    if (lane == 0) s.cnt[0][0][warp] = cnt;
+    __syncthreads();
+    int base_gt, base_eq;
+    {
+        const int c = s.cnt[0][0][lane];                // kWarps == 32: one packed count per lane
+        int incl = c;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += t;
+        }
+        const int excl = __shfl_sync(0xffffffffu, incl - c, warp);          // exclusive prefix of this warp
+        base_gt = head_gt + (excl & 0xffff);
+        base_eq = head_eq + (excl >> 16);
+    }
+
+    // ---- emission: head, stretches, tail ----------------------------------------------------------
+    if (tid == 0) {
+        int g = 0, e = 0;
+        for (int i = 0; i < head; ++i) {
+            const uint32_t key = order_key(sc[i]);
+            if (key > thr) out[g + min(e, ties)] = i;
+            else if (key == thr && e < ties) out[g + e] = i;
+            g += key > thr; e += key == thr;
+        }
+    }
+    for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
+        float4 q[kAhead];
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+            const int vi = v0 + u * 32 + lane;
+            q[u] = vi < vend ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+            const int vi = v0 + u * 32 + lane;
+            int g, e;
+            flags(q[u], g, e);
+            if (vi >= vend) { g = 0; e = 0; }
+            const int mine = __popc(g) | (__popc(e) << 16);
+            int incl = mine;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                int t = __shfl_up_sync(0xffffffffu, incl, off);
+                const int t = __shfl_up_sync(0xffffffffu, incl, off);
                 if (lane >= off) incl += t;
             }
-            s.cnt[buf][warp][lane] = incl - v;
-            if (lane == 31) s.row_total[buf][warp] = incl;
-        }
-        __syncthreads();
-        int run = 0;                        // packed count of the sub-blocks before u in this iteration
+            int gt_before = base_gt + ((incl - mine) & 0xffff);
+            int eq_before = base_eq + ((incl - mine) >> 16);
+            const int i0 = head + 4 * vi;
 #pragma unroll
-        for (int u = 0; u < kSub; ++u) {
-            const int i = start + u * kThreads + tid;
-            const int before = run + s.cnt[buf][u][warp];
-            const int gt_before = base_gt + (before & 0xffff) + __popc(bg[u] & lt_mask);
-            const int eq_before = base_eq + (before >> 16) + __popc(be[u] & lt_mask);
-            if (i < n) {
-                if (keys[u] > thr) out[gt_before + min(eq_before, ties)] = i;
-                else if (keys[u] == thr && eq_before < ties) out[gt_before + eq_before] = i;
+            for (int j = 0; j < 4; ++j) {
+                if ((g >> j) & 1) { out[gt_before + min(eq_before, ties)] = i0 + j; ++gt_before; }
+                else if ((e >> j) & 1) { if (eq_before < ties) out[gt_before + eq_before] = i0 + j; ++eq_before; }
             }
-            run += s.row_total[buf][u];
+            const int total = __shfl_sync(0xffffffffu, incl, 31);
+            base_gt += total & 0xffff;
+            base_eq += total >> 16;
         }
-        base_gt += run & 0xffff;
-        base_eq += run >> 16;
+    }
+    if (warp == kWarps - 1 && lane == 0) {                // the tail follows the last stretch
+        for (int i = tail_begin; i < n; ++i) {
+            const uint32_t key = order_key(sc[i]);
+            if (key > thr) out[base_gt + min(base_eq, ties)] = i;
+            else if (key == thr && base_eq < ties) out[base_gt + base_eq] = i;
+            base_gt += key > thr; base_eq += key == thr;
+        }
     }
 }
 

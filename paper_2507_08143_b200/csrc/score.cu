@@ -20,6 +20,9 @@ constexpr int kStages = 6;
 constexpr int kBoxBytes = kTile * 128;
 constexpr int kTileBytes = 2 * kBoxBytes;
 constexpr int kThreads = 192;
+// Tiles whose scores are stored together (4 KB bursts instead of 512 B); at MP = 64 the W operand
+// leaves no shared memory for that.
+template <int MP> struct OutTiles { static constexpr int value = MP <= 48 ? 8 : 1; };
 constexpr int kBufs = 4;                  // accumulators of up to 64 columns each
 constexpr uint32_t kTmemCols = 64 * kBufs;
 
@@ -32,8 +35,10 @@ struct __align__(1024) ScoreSmem {
     uint64_t w_full;
     uint64_t d_full[kBufs];
     uint64_t d_empty[kBufs];
+    float obuf[2][OutTiles<MP>::value * kTile];     // scores of a group of tiles, written to global memory in one burst
     uint32_t tmem_base;
     int abort;
+    int abort_mma;                        // set by the MMA warp alone before it wakes the epilogue: seen alike by all its threads
 };
 
 template <int MP>
@@ -61,6 +66,7 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
         mbar_init(&s.w_full, 1);
         for (int i = 0; i < kBufs; ++i) { mbar_init(&s.d_full[i], 1); mbar_init(&s.d_empty[i], 4); }
         s.abort = 0;
+        s.abort_mma = 0;
         fence_barrier_init();
     }
     if (warp == 1) { tmem_alloc(&s.tmem_base, kTmemCols); tmem_relinquish(); }
@@ -117,17 +123,22 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
         }
         if (!ok) {
             s.abort = 1;
+            s.abort_mma = 1;
+            __threadfence_block();
+            __syncwarp();
             if (lane == 0)
                 for (int i = 0; i < kBufs; ++i) mbar_arrive(&s.d_full[i]);   // wake the epilogue
         }
     } else {
         const int q = warp & 3;
         float* out = scores + (size_t)lh * p.total_tokens + tok_begin;
+        constexpr int kOutTiles = OutTiles<MP>::value;
+        const int et = threadIdx.x - 64;                     // 0..127 among the epilogue threads
         for (int t = 0; t < n_tiles; ++t) {
             const int buf = t % kBufs, use = t / kBufs;
-            const bool ok = mbar_wait(&s.d_full[buf], use & 1);
-            if (!ok) s.abort = 1;
-            if (!ok || *(volatile int*)&s.abort) break;
+            // all 128 epilogue threads take the same decision (they meet at a named barrier below)
+            const bool ok = mbar_wait(&s.d_full[buf], use & 1) && !*(volatile int*)&s.abort_mma;
+            if (!ok) { s.abort = 1; break; }
             tc_fence_after_sync();
             float acc = 0.f;
 #pragma unroll
@@ -141,8 +152,14 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&s.d_empty[buf]);
-            const int tok = t * kTile + q * 32 + lane;
-            if (tok < n_tok) out[tok] = acc;
+            const int group = t / kOutTiles, in_group = t % kOutTiles;
+            s.obuf[group & 1][in_group * kTile + q * 32 + lane] = acc;
+            if (in_group == kOutTiles - 1 || t == n_tiles - 1) {
+                asm volatile("bar.sync 2, 128;" ::: "memory");         // the group's scores are in shared memory
+                const int g0 = group * kOutTiles * kTile;
+                const int count = min(n_tok - g0, (in_group + 1) * kTile);
+                for (int i = et; i < count; i += 128) out[g0 + i] = s.obuf[group & 1][i];
+            }
         }
     }
     tc_fence_before_sync();

@@ -163,11 +163,9 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             tc_fence_after_sync();
             const bool row_valid = (it & 1) * kHalf + row < n_tok;
             float mx = -INFINITY;
-#pragma unroll 1
-            for (int c0 = 0; c0 < 128; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld_32x32b_x32(lane_addr + c0, r);
-                tmem_ld_wait();
+            // the load of the next 32 columns is in flight while this thread works on the current ones
+            uint32_t ra[32], rb[32];
+            auto max_of = [&](const uint32_t (&r)[32], int c0) {
                 if (full) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
@@ -176,17 +174,25 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                     for (int i = 0; i < 32; ++i)
                         if (ch * 128 + c0 + i < n_tok) mx = fmaxf(mx, __uint_as_float(r[i]));
                 }
-            }
+            };
+            tmem_ld_32x32b_x32(lane_addr, ra);
+            tmem_ld_wait_for(ra);
+            tmem_ld_32x32b_x32(lane_addr + 32, rb);
+            max_of(ra, 0);
+            tmem_ld_wait_for(rb);
+            tmem_ld_32x32b_x32(lane_addr + 64, ra);
+            max_of(rb, 32);
+            tmem_ld_wait_for(ra);
+            tmem_ld_32x32b_x32(lane_addr + 96, rb);
+            max_of(ra, 64);
+            tmem_ld_wait_for(rb);
+            max_of(rb, 96);
             s.xmax[ch][row] = mx;
             softmax_pair_sync();
             mx = fmaxf(s.xmax[0][row], s.xmax[1][row]);      // finite: key 0 of the chunk always exists
             const float bias = -mx * scale_log2e;
             float sum = 0.f;
-#pragma unroll 1
-            for (int c0 = 0; c0 < 128; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld_32x32b_x32(lane_addr + c0, r);
-                tmem_ld_wait();
+            auto exp_of = [&](const uint32_t (&r)[32], int c0) {
                 uint32_t packed[16];
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
@@ -208,7 +214,19 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                     *reinterpret_cast<uint4*>(blk + ((piece ^ (row & 7)) << 4)) =
                         make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
                 }
-            }
+            };
+            tmem_ld_32x32b_x32(lane_addr, ra);
+            tmem_ld_wait_for(ra);
+            tmem_ld_32x32b_x32(lane_addr + 32, rb);
+            exp_of(ra, 0);
+            tmem_ld_wait_for(rb);
+            tmem_ld_32x32b_x32(lane_addr + 64, ra);
+            exp_of(rb, 32);
+            tmem_ld_wait_for(ra);
+            tmem_ld_32x32b_x32(lane_addr + 96, rb);
+            exp_of(ra, 64);
+            tmem_ld_wait_for(rb);
+            exp_of(rb, 96);
             s.xsum[ch][row] = sum;
             softmax_pair_sync();
             if (ch == 0) {

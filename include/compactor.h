@@ -50,6 +50,10 @@ extern "C" {
 #define COMPACTOR_STATUS_RANK        2
 #define COMPACTOR_STATUS_TIMEOUT     4
 
+/* Small factorisations for compactor_score_variant (Appendix C). */
+#define COMPACTOR_FACTOR_CHOLESKY    0    /* G = L L^T: the R factor of the QR route          */
+#define COMPACTOR_FACTOR_EIG         1    /* G = V Lambda V^T with a floor on the eigenvalues */
+
 /* A strided bf16 tensor [layers][heads][total_tokens][d] in device memory. */
 typedef struct compactor_mat {
     const void* ptr;          /* device, 16-byte aligned                           */
@@ -139,11 +143,29 @@ size_t compactor_workspace_bytes(const compactor_shape* shape);
  *   scores_out   device fp32 [layers][heads][total_tokens].
  * The small factorisation is a Cholesky factorisation of G = (K Phi)^T (K Phi) in fp64 - one of
  * the algebraically equal routes the paper allows (Section 3.2, Appendix C); Gram sums are fp32
- * within runs of 2048 tokens and fp64 beyond.
+ * within runs of 512 tokens and fp64 beyond.
  */
 int compactor_score(const compactor_shape* shape, compactor_mat k_score, const float* phi,
                     const float* attn_scores, float lambda, float* scores_out,
                     int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * compactor_score with the small factorisation chosen by the caller (Appendix C).
+ *   factorization  COMPACTOR_FACTOR_CHOLESKY: exactly compactor_score.  Cholesky of G is the R
+ *                  factor of the appendix's QR route (K Phi = Q R, score = squared row norm of Q).
+ *                  COMPACTOR_FACTOR_EIG: the appendix's eigendecomposition route.  G = V Lambda V^T
+ *                  (cyclic Jacobi, fp64), every eigenvalue raised to at least eig_floor,
+ *                  score_i = || k_i Phi V Lambda^-1/2 ||^2.  Unlike the other routes the result
+ *                  depends on the scale of Phi once the floor is active; the status bit
+ *                  COMPACTOR_STATUS_RANK then reports that some eigenvalue was below the floor.
+ *   eig_floor      the floor (the paper suggests about 1e-6); must be positive and finite;
+ *                  ignored for COMPACTOR_FACTOR_CHOLESKY.
+ * All other arguments, the workspace and the error behaviour are those of compactor_score.
+ */
+int compactor_score_variant(const compactor_shape* shape, compactor_mat k_score, const float* phi,
+                            int32_t factorization, double eig_floor,
+                            const float* attn_scores, float lambda, float* scores_out,
+                            int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Per-unit top-k (Section 3.4: the ceil(r N) highest-scoring tokens are kept, here per head).

@@ -11,6 +11,9 @@ What follows the paper step by step:
     small SVD, back-projection, squared row norms).
   * `exact_leverage_scores`  - Definition 1 / Eq. 1 (the quantity Algorithm 1
     approximates; used to pin the oracle, and as the m = d special case).
+  * `approx_leverage_scores_eig`, `approx_leverage_scores_qr` - Appendix C's
+    two other routes to the same scores (eigendecomposition of G with clamped
+    eigenvalues; reduced QR of K Phi).
   * `attention_scores`       - Eq. 5 (column sums of chunked non-causal softmax
     attention, mean-pooled).
   * `blend`                  - Eq. 6 (z-scored attention term + lambda * z-scored
@@ -163,6 +166,33 @@ def approx_leverage_scores(K: np.ndarray, Phi: np.ndarray) -> np.ndarray:
     sigma = np.sqrt(lam[keep])
     U_t = (K_hat @ V_t[:, keep]) / sigma[None, :]     # line 5
     return np.sum(U_t * U_t, axis=1)                  # line 6: diag(U U^T)
+
+
+def approx_leverage_scores_eig(K: np.ndarray, Phi: np.ndarray, eps: float = 1e-6) -> np.ndarray:
+    """Appendix C, eigendecomposition route: G = V Lambda V^T, every eigenvalue raised to at
+    least eps (an absolute floor on the eigenvalues of G, so the result depends on the scale
+    of K Phi once the floor is active), U~ = K^ V Lambda^-1/2, scores = squared row norms."""
+    K = np.asarray(K, dtype=np.float64)
+    Phi = np.asarray(Phi, dtype=np.float64)
+    if K.shape[0] == 0:
+        return np.zeros(0)
+    K_hat = K @ Phi
+    G = K_hat.T @ K_hat
+    lam, V = np.linalg.eigh(G)
+    lam = np.maximum(lam, float(eps))
+    U_t = (K_hat @ V) / np.sqrt(lam)[None, :]
+    return np.sum(U_t * U_t, axis=1)
+
+
+def approx_leverage_scores_qr(K: np.ndarray, Phi: np.ndarray) -> np.ndarray:
+    """Appendix C, QR route: K^ = Q R (reduced), scores = squared row norms of Q.  Defined for
+    K^ of full column rank; rank-deficient input is left to the routes above."""
+    K = np.asarray(K, dtype=np.float64)
+    Phi = np.asarray(Phi, dtype=np.float64)
+    if K.shape[0] == 0:
+        return np.zeros(0)
+    Q, _ = np.linalg.qr(K @ Phi, mode="reduced")
+    return np.sum(Q * Q, axis=1)
 
 
 # ----------------------------------------------------------------------------

@@ -47,6 +47,8 @@ def _load() -> ctypes.CDLL:
     lib.compactor_workspace_bytes.argtypes = [POINTER(CompactorShape)]
     lib.compactor_score.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_void_p, c_float, c_void_p,
                                     c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_score_variant.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_int32, c_double, c_void_p,
+                                            c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.compactor_select.argtypes = [POINTER(CompactorShape), c_void_p, POINTER(c_int32), c_void_p, c_void_p,
                                      c_void_p, c_size_t, c_void_p]
     lib.compactor_compact.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_void_p, POINTER(c_int32),
@@ -77,7 +79,11 @@ EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch
            "compactor_calibrated_ratio", "compactor_fit_calibration", "compactor_workspace_bytes", "compactor_score", "compactor_select",
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
            "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores", "compactor_wait_selftest",
-           "compactor_across_heads_workspace_bytes", "compactor_select_across_heads", "compactor_compact_across_heads"]
+           "compactor_across_heads_workspace_bytes", "compactor_select_across_heads", "compactor_compact_across_heads",
+           "compactor_score_variant"]
+
+FACTOR_CHOLESKY = 0
+FACTOR_EIG = 1
 
 N_STAGE_EVENTS = 7
 STAGE_NAMES = ["gram", "factor", "score", "blend", "select", "compact"]
@@ -178,6 +184,15 @@ def score(shape: Shape, k_score: torch.Tensor, phi: torch.Tensor, scores_out: to
           attn: Optional[torch.Tensor] = None, lam: float = 0.3, status: Optional[torch.Tensor] = None) -> None:
     _check(LIB.compactor_score(byref(shape.c), mat(k_score), _ptr(phi), _ptr(attn), lam, _ptr(scores_out),
                                _ptr(status), _ptr(workspace), workspace.numel(), _stream()), "compactor_score")
+
+
+def score_variant(shape: Shape, k_score: torch.Tensor, phi: torch.Tensor, scores_out: torch.Tensor,
+                  workspace: torch.Tensor, factorization: int, eig_floor: float = 1e-6,
+                  attn: Optional[torch.Tensor] = None, lam: float = 0.3, status: Optional[torch.Tensor] = None) -> None:
+    """Appendix C: `score` with the small factorisation chosen (FACTOR_CHOLESKY or FACTOR_EIG)."""
+    _check(LIB.compactor_score_variant(byref(shape.c), mat(k_score), _ptr(phi), factorization, eig_floor, _ptr(attn), lam,
+                                       _ptr(scores_out), _ptr(status), _ptr(workspace), workspace.numel(), _stream()),
+           "compactor_score_variant")
 
 
 def select(shape: Shape, scores: torch.Tensor, keep_counts: Sequence[int], idx_out: torch.Tensor,

@@ -145,14 +145,16 @@ struct Marks {
 };
 
 int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn, float lambda,
-                float* scores, int32_t* status, char* ws, cudaStream_t stream, const Marks& mk = Marks()) {
+                float* scores, int32_t* status, char* ws, cudaStream_t stream, const Marks& mk = Marks(),
+                int factorization = COMPACTOR_FACTOR_CHOLESKY, double eig_floor = 0.0) {
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(ws + hp.off_w);
     double* partials = reinterpret_cast<double*>(ws + hp.off_partials);
     if (status != nullptr) CK(cudaMemsetAsync(status, 0, sizeof(int32_t) * hp.units, stream));
     CK(mk.mark(0, stream));
     CK(launch_gram(hp.plan, k, partials, status, stream));
     CK(mk.mark(1, stream));
-    CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, status, stream));
+    CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, status,
+                     factorization, eig_floor, stream));
     CK(mk.mark(2, stream));
     CK(launch_score(hp.plan, k, w, scores, status, stream));
     CK(mk.mark(3, stream));
@@ -236,6 +238,28 @@ int compactor_score(const compactor_shape* shape, compactor_mat k_score, const f
     CK(upload_tables(&hp, workspace, st));
     return run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores_out, status,
                        static_cast<char*>(workspace), st);
+}
+
+int compactor_score_variant(const compactor_shape* shape, compactor_mat k_score, const float* phi,
+                            int32_t factorization, double eig_floor, const float* attn_scores, float lambda,
+                            float* scores_out, int32_t* status, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+    if (factorization == COMPACTOR_FACTOR_CHOLESKY)
+        return compactor_score(shape, k_score, phi, attn_scores, lambda, scores_out, status, workspace,
+                               workspace_bytes, stream);
+    if (factorization != COMPACTOR_FACTOR_EIG) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (!(eig_floor > 0.0) || !std::isfinite(eig_floor)) return COMPACTOR_E_INVALID_ARGUMENT;
+    HostPlan hp; int err = 0;
+    if (!make_plan(shape, &hp, &err)) return err;
+    if (!mat_ok(k_score) || phi == nullptr || scores_out == nullptr || workspace == nullptr)
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (((uintptr_t)workspace & 255) != 0) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (workspace_bytes < hp.total_bytes) return COMPACTOR_E_WORKSPACE;
+    if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CK(upload_tables(&hp, workspace, st));
+    return run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores_out, status,
+                       static_cast<char*>(workspace), st, Marks(), factorization, eig_floor);
 }
 
 int compactor_select(const compactor_shape* shape, const float* scores, const int32_t* keep_counts,

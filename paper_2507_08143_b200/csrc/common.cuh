@@ -50,7 +50,7 @@ __device__ __forceinline__ int find_segment(const int* __restrict__ table, int n
 // launch status.
 cudaError_t launch_gram(const Plan& p, const Mat& k, double* partials, int* status, cudaStream_t stream);
 cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* g_partials,
-                          __nv_bfloat16* w, int* status, cudaStream_t stream);
+                          __nv_bfloat16* w, int* status, int factorization, double eig_floor, cudaStream_t stream);
 cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
                          cudaStream_t stream);
 cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* scores, cudaStream_t stream);

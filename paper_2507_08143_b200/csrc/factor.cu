@@ -297,9 +297,160 @@ cholesky_kernel(Plan p, const double* __restrict__ g_partials, const float* __re
     if (tid == 0 && status != nullptr && s.flags != 0) atomicOr(&status[unit], s.flags);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Appendix C, eigendecomposition route: G = V Lambda V^T by cyclic two-sided Jacobi rotations in
+// fp64 (all disjoint index pairs of a round-robin step are rotated at once), every eigenvalue
+// raised to at least `floor`, W = Phi V Lambda^-1/2 split into two bf16 terms.  One CTA per unit.
+constexpr int kEigThreads = kD;
+constexpr int kEigMaxSweeps = 16;
+
+template <int MP>
+struct EigSmem {
+    static constexpr int kLd = MP + 1;
+    double a[MP * kLd];          // G, driven to diagonal form
+    double v[MP * kLd];          // accumulated rotations: columns are the eigenvectors
+    double rot_c[MP / 2], rot_s[MP / 2];
+    int rot_p[MP / 2], rot_q[MP / 2];
+    double inv_sqrt[MP];
+    double red[kEigThreads / 32][2];
+    int flags;
+};
+
+template <int MP>
+__global__ void __launch_bounds__(kEigThreads, 3)
+eig_kernel(Plan p, const double* __restrict__ g_partials, const float* __restrict__ phi, double floor,
+           __nv_bfloat16* __restrict__ w_out, int* __restrict__ status) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    using Smem = EigSmem<MP>;
+    Smem& s = *reinterpret_cast<Smem*>(smem_raw);
+    constexpr int LD = Smem::kLd;
+    const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int m = p.m;
+    const int n = (m + 1) & ~1;                 // an even number of indices to pair; the padding row is zero
+    const int half = n >> 1;
+
+    if (tid == 0) s.flags = 0;
+    __syncthreads();
+    {
+        const double* src = g_partials + (size_t)unit * kSlices * (MP * MP);
+        bool finite = true;
+        for (int e = tid; e < MP * MP; e += kEigThreads) {
+            double x = 0.0;
+#pragma unroll
+            for (int r = 0; r < kSlices; ++r) x += src[(size_t)r * (MP * MP) + e];
+            const int i = e / MP, j = e % MP;
+            s.a[i * LD + j] = x;
+            s.v[i * LD + j] = (i == j) ? 1.0 : 0.0;
+            finite = finite && isfinite(x);
+        }
+        if (!finite) atomicOr(&s.flags, COMPACTOR_STATUS_NONFINITE);
+    }
+    __syncthreads();
+    const bool bad = (s.flags & COMPACTOR_STATUS_NONFINITE) != 0;
+
+    for (int sweep = 0; sweep < kEigMaxSweeps && !bad; ++sweep) {
+        // off-diagonal mass against the whole: the same value in every thread, so all leave together
+        double off = 0.0, all = 0.0;
+        for (int e = tid; e < n * n; e += kEigThreads) {
+            const int i = e / n, j = e % n;
+            const double x = s.a[i * LD + j];
+            all = fma(x, x, all);
+            if (i != j) off = fma(x, x, off);
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            off += __shfl_xor_sync(0xffffffffu, off, d);
+            all += __shfl_xor_sync(0xffffffffu, all, d);
+        }
+        if (lane == 0) { s.red[warp][0] = off; s.red[warp][1] = all; }
+        __syncthreads();
+        off = 0.0; all = 0.0;
+#pragma unroll
+        for (int w = 0; w < kEigThreads / 32; ++w) { off += s.red[w][0]; all += s.red[w][1]; }
+        __syncthreads();
+        if (!(off > 1e-26 * all)) break;
+
+        for (int step = 0; step < n - 1; ++step) {
+            if (tid < half) {
+                // round-robin pairing: index n-1 stays, the others move round a ring of n-1 seats
+                int a0, a1;
+                if (tid == 0) { a0 = n - 1; a1 = step % (n - 1); }
+                else { a0 = (step + tid) % (n - 1); a1 = (step - tid + (n - 1)) % (n - 1); }
+                const int pp = min(a0, a1), qq = max(a0, a1);
+                const double apq = s.a[pp * LD + qq], app = s.a[pp * LD + pp], aqq = s.a[qq * LD + qq];
+                double c = 1.0, sn = 0.0;
+                if (fabs(apq) > 1e-300 && fabs(apq) > 1e-19 * sqrt(fabs(app) * fabs(aqq))) {
+                    const double theta = (aqq - app) / (2.0 * apq);
+                    const double t = copysign(1.0, theta) / (fabs(theta) + sqrt(fma(theta, theta, 1.0)));
+                    c = rsqrt(fma(t, t, 1.0));
+                    sn = t * c;
+                }
+                s.rot_c[tid] = c; s.rot_s[tid] = sn; s.rot_p[tid] = pp; s.rot_q[tid] = qq;
+            }
+            __syncthreads();
+            // columns: A <- A J and V <- V J
+            for (int e = tid; e < 2 * n * half; e += kEigThreads) {
+                const int which = e / (n * half), r = e % (n * half);
+                const int i = r / half, k = r % half;
+                const int pp = s.rot_p[k], qq = s.rot_q[k];
+                const double c = s.rot_c[k], sn = s.rot_s[k];
+                double* mat = which ? s.v : s.a;
+                const double x = mat[i * LD + pp], y = mat[i * LD + qq];
+                mat[i * LD + pp] = fma(c, x, -sn * y);
+                mat[i * LD + qq] = fma(sn, x, c * y);
+            }
+            __syncthreads();
+            // rows: A <- J^T A
+            for (int e = tid; e < n * half; e += kEigThreads) {
+                const int k = e / n, i = e % n;
+                const int pp = s.rot_p[k], qq = s.rot_q[k];
+                const double c = s.rot_c[k], sn = s.rot_s[k];
+                const double x = s.a[pp * LD + i], y = s.a[qq * LD + i];
+                s.a[pp * LD + i] = fma(c, x, -sn * y);
+                s.a[qq * LD + i] = fma(sn, x, c * y);
+            }
+            __syncthreads();
+        }
+    }
+
+    if (tid < MP) {
+        double inv = 0.0;
+        if (tid < m && !bad) {
+            const double lam = s.a[tid * LD + tid];
+            if (lam < floor) atomicOr(&s.flags, COMPACTOR_STATUS_RANK);
+            inv = rsqrt(fmax(lam, floor));
+        }
+        s.inv_sqrt[tid] = inv;
+    }
+    __syncthreads();
+
+    {   // W = Phi V Lambda^-1/2: one thread per row of Phi
+        const int row = tid;
+        double r[MP];
+#pragma unroll
+        for (int c = 0; c < MP; ++c) r[c] = (c < m && !bad) ? (double)phi[row * m + c] : 0.0;
+        __nv_bfloat16* w_hi = w_out + (size_t)unit * w_elems_per_unit(MP);
+        __nv_bfloat16* w_lo = w_hi + (size_t)MP * kD;
+        for (int j = 0; j < MP; ++j) {
+            double acc0 = 0.0, acc1 = 0.0;
+#pragma unroll
+            for (int c = 0; c < MP; c += 2) {
+                acc0 = fma(r[c], s.v[c * LD + j], acc0);
+                acc1 = fma(r[c + 1], s.v[(c + 1) * LD + j], acc1);
+            }
+            const double wj = (j < m) ? (acc0 + acc1) * s.inv_sqrt[j] : 0.0;
+            const __nv_bfloat16 hi = __double2bfloat16(wj);
+            w_hi[j * kD + row] = hi;
+            w_lo[j * kD + row] = __double2bfloat16(wj - (double)__bfloat162float(hi));
+        }
+    }
+    if (tid == 0 && status != nullptr && s.flags != 0) atomicOr(&status[unit], s.flags);
+}
+
 template <int MP>
 cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials, const float* phi,
-                             double* g_partials, __nv_bfloat16* w, int* status, cudaStream_t stream) {
+                             double* g_partials, __nv_bfloat16* w, int* status, int factorization, double eig_floor,
+                             cudaStream_t stream) {
     const int units = p.layers * p.heads * p.batch;
     const int smem = (int)sizeof(ProjectSmem<MP>);
     cudaError_t e = cudaFuncSetAttribute(project_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -309,20 +460,27 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
     project_kernel<MP><<<grid, kProjThreads, smem, stream>>>(p, k, partials, phi, g_partials, n_items);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    cholesky_kernel<MP><<<units, kCholThreads, 0, stream>>>(p, g_partials, phi, w, status);
+    if (factorization == COMPACTOR_FACTOR_EIG) {
+        const int esmem = (int)sizeof(EigSmem<MP>);
+        e = cudaFuncSetAttribute(eig_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, esmem);
+        if (e != cudaSuccess) return e;
+        eig_kernel<MP><<<units, kEigThreads, esmem, stream>>>(p, g_partials, phi, eig_floor, w, status);
+    } else {
+        cholesky_kernel<MP><<<units, kCholThreads, 0, stream>>>(p, g_partials, phi, w, status);
+    }
     return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* g_partials,
-                          __nv_bfloat16* w, int* status, cudaStream_t stream) {
+                          __nv_bfloat16* w, int* status, int factorization, double eig_floor, cudaStream_t stream) {
     if (p.layers * p.heads * p.batch == 0) return cudaSuccess;
     switch (p.mp) {
-        case 16: return launch_factor_mp<16>(p, k, partials, phi, g_partials, w, status, stream);
-        case 32: return launch_factor_mp<32>(p, k, partials, phi, g_partials, w, status, stream);
-        case 48: return launch_factor_mp<48>(p, k, partials, phi, g_partials, w, status, stream);
-        case 64: return launch_factor_mp<64>(p, k, partials, phi, g_partials, w, status, stream);
+        case 16: return launch_factor_mp<16>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
+        case 32: return launch_factor_mp<32>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
+        case 48: return launch_factor_mp<48>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
+        case 64: return launch_factor_mp<64>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
         default: return cudaErrorInvalidValue;
     }
 }

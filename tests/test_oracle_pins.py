@@ -141,6 +141,41 @@ def test_alg1_detects_a_transposed_or_dropped_factor():
     np.testing.assert_allclose(orc.approx_leverage_scores(K, Phi), want, rtol=1e-9)
 
 
+def test_appendix_c_routes_agree_on_full_rank_input():
+    # Full column rank and a floor far below the spectrum: all three routes give Algorithm 1's scores.
+    rng = _rng(21)
+    K = rng.standard_normal((300, 20)); Phi = rng.standard_normal((20, 7))
+    o = orc.approx_leverage_scores(K, Phi)
+    np.testing.assert_allclose(orc.approx_leverage_scores_qr(K, Phi), o, rtol=1e-9)
+    np.testing.assert_allclose(orc.approx_leverage_scores_eig(K, Phi, 1e-6), o, rtol=1e-9)
+    np.testing.assert_allclose(orc.approx_leverage_scores_qr(K, np.eye(20)), orc.exact_leverage_scores(K), rtol=1e-9)
+    assert orc.approx_leverage_scores_eig(np.zeros((0, 20)), Phi).shape == (0,)
+    assert orc.approx_leverage_scores_qr(np.zeros((0, 20)), Phi).shape == (0,)
+
+
+def test_eig_route_clamp_closed_form():
+    # K = Q diag(sigma) with orthonormal Q and Phi = the first m columns of the identity:
+    # G = diag(sigma_j^2), so score_i = sum_j Q_ij^2 sigma_j^2 / max(sigma_j^2, eps).  Directions
+    # above the floor count fully, directions below it are scaled by sigma_j^2 / eps.
+    rng = _rng(22)
+    n, d, m = 40, 6, 4
+    Q, _ = np.linalg.qr(rng.standard_normal((n, d)))
+    sigma = np.array([3.0, 1.0, 1e-2, 1e-4, 5.0, 2.0])
+    K = Q * sigma[None, :]
+    Phi = np.eye(d)[:, :m]
+    for eps in (1e-12, 1e-6, 1e-3, 4.0):
+        lam = sigma[:m] ** 2
+        want = np.sum(Q[:, :m] ** 2 * (lam / np.maximum(lam, eps))[None, :], axis=1)
+        np.testing.assert_allclose(orc.approx_leverage_scores_eig(K, Phi, eps), want, rtol=1e-7, atol=1e-12)
+    # a floor above every eigenvalue turns the score into ||k_hat_i||^2 / eps
+    big = orc.approx_leverage_scores_eig(K, Phi, 100.0)
+    np.testing.assert_allclose(big, np.sum((K @ Phi) ** 2, axis=1) / 100.0, rtol=1e-9)
+    # exactly rank-deficient input: the null directions contribute (numerically) nothing
+    K2 = np.hstack([K[:, :3], K[:, :3]])
+    got = orc.approx_leverage_scores_eig(K2, np.eye(6), 1e-6)
+    np.testing.assert_allclose(got, orc.exact_leverage_scores(K2), atol=1e-7)
+
+
 def test_bf16_widening_is_exact():
     import torch
     x = torch.randn(1000, dtype=torch.float32).to(torch.bfloat16)

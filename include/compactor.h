@@ -41,7 +41,7 @@ extern "C" {
 
 #define COMPACTOR_OK                  0
 #define COMPACTOR_E_INVALID_ARGUMENT -1   /* null pointer, bad size, bad stride or alignment      */
-#define COMPACTOR_E_UNSUPPORTED      -2   /* d != 128 or m outside [1, 64]                       */
+#define COMPACTOR_E_UNSUPPORTED      -2   /* d != 128 or m outside [1, 128]                      */
 #define COMPACTOR_E_WORKSPACE        -3   /* workspace smaller than compactor_workspace_bytes()  */
 #define COMPACTOR_E_CUDA             -4   /* a CUDA runtime call failed (see cudaGetLastError)   */
 #define COMPACTOR_E_TOO_LARGE        -5   /* problem exceeds the library's built-in scratch      */
@@ -67,7 +67,7 @@ typedef struct compactor_shape {
     int32_t layers;
     int32_t heads;
     int32_t d;                /* head dimension; must be 128                       */
-    int32_t m;                /* sketch dimension (the paper uses 48)              */
+    int32_t m;                /* sketch dimension, 1..128 (the paper uses 48)      */
     int32_t batch;            /* number of packed sequences                        */
     const int32_t* cu_seqlens;/* host, [batch+1]                                   */
 } compactor_shape;
@@ -141,6 +141,9 @@ size_t compactor_workspace_bytes(const compactor_shape* shape);
  *                s = z(attn) + lambda * z(o) per unit (population std; a term with zero std
  *                contributes 0); if NULL the output is the outlier score o itself.
  *   scores_out   device fp32 [layers][heads][total_tokens].
+ * With m = d and any invertible phi (the identity, say) the result is the exact leverage score
+ * of Definition 1 / Eq. 1, the paper's "exact" ablation; sketches wider than 64 columns run in a
+ * slower configuration of the same kernels.
  * The small factorisation is a Cholesky factorisation of G = (K Phi)^T (K Phi) in fp64 - one of
  * the algebraically equal routes the paper allows (Section 3.2, Appendix C); Gram sums are fp32
  * within runs of 512 tokens and fp64 beyond.
@@ -160,6 +163,7 @@ int compactor_score(const compactor_shape* shape, compactor_mat k_score, const f
  *                  COMPACTOR_STATUS_RANK then reports that some eigenvalue was below the floor.
  *   eig_floor      the floor (the paper suggests about 1e-6); must be positive and finite;
  *                  ignored for COMPACTOR_FACTOR_CHOLESKY.
+ * The eigendecomposition route takes m <= 64 (COMPACTOR_E_UNSUPPORTED beyond).
  * All other arguments, the workspace and the error behaviour are those of compactor_score.
  */
 int compactor_score_variant(const compactor_shape* shape, compactor_mat k_score, const float* phi,

@@ -43,7 +43,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     Plan& p = hp->plan;
     memset(&p, 0, sizeof(p));
     p.layers = s->layers; p.heads = s->heads; p.batch = s->batch;
-    p.m = s->m; p.mp = (s->m + 15) / 16 * 16;
+    p.m = s->m; p.mp = s->m <= 64 ? (s->m + 15) / 16 * 16 : 128;
     p.total_tokens = s->cu_seqlens[s->batch];
     hp->units = s->layers * s->heads * s->batch;
 
@@ -251,6 +251,7 @@ int compactor_score_variant(const compactor_shape* shape, compactor_mat k_score,
     if (!(eig_floor > 0.0) || !std::isfinite(eig_floor)) return COMPACTOR_E_INVALID_ARGUMENT;
     HostPlan hp; int err = 0;
     if (!make_plan(shape, &hp, &err)) return err;
+    if (hp.plan.mp > 64) return COMPACTOR_E_UNSUPPORTED;
     if (!mat_ok(k_score) || phi == nullptr || scores_out == nullptr || workspace == nullptr)
         return COMPACTOR_E_INVALID_ARGUMENT;
     if (((uintptr_t)workspace & 255) != 0) return COMPACTOR_E_INVALID_ARGUMENT;

@@ -9,7 +9,7 @@
 namespace compactor {
 
 constexpr int kD = 128;            // head dimension the kernels are written for
-constexpr int kMaxM = 64;          // largest sketch dimension
+constexpr int kMaxM = 128;          // largest sketch dimension
 constexpr int kMaxChunk = 32768;   // most tokens per block (one CTA of the two streaming kernels)
 constexpr int kMinChunk = 256;
 constexpr int kGramFlushTokens = 512;    // most tokens whose Gram matrix is summed in fp32 (tensor-core accumulators) before going to fp64

@@ -200,19 +200,27 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
 
 constexpr int kCholThreads = kD;           // one thread per row of Phi
 
+// Columns of W that a thread holds in registers at a time; a wider sketch is solved block by block,
+// with the finished blocks parked in shared memory (fp64) for the updates of the later ones.
+template <int MP> struct WBlock { static constexpr int value = MP <= 64 ? MP : 64; };
+
 template <int MP>
 struct CholSmem {
+    static constexpr int kParked = MP - WBlock<MP>::value;      // columns of W kept for later blocks
     double g[MP * (MP + 1)];     // G, then L in the lower triangle; odd row stride spreads a column over the banks
     double inv_diag[MP];         // 1 / L_jj of kept columns, 0 for dropped or padded ones
+    double parked[kParked > 0 ? kParked * kCholThreads : 1];
     int flags;
 };
 
 template <int MP>
-__global__ void __launch_bounds__(kCholThreads, 4)
+__global__ void __launch_bounds__(kCholThreads, MP <= 48 ? 4 : (MP <= 64 ? 2 : 1))
 cholesky_kernel(Plan p, const double* __restrict__ g_partials, const float* __restrict__ phi,
                 __nv_bfloat16* __restrict__ w_out, int* __restrict__ status) {
-    __shared__ CholSmem<MP> s;
+    extern __shared__ __align__(16) unsigned char chol_smem_raw[];
+    CholSmem<MP>& s = *reinterpret_cast<CholSmem<MP>*>(chol_smem_raw);
     constexpr int LD = MP + 1;
+    constexpr int kH = (MP + 31) / 32;          // rows of a column per lane
     const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = p.m;
 
@@ -234,13 +242,13 @@ cholesky_kernel(Plan p, const double* __restrict__ g_partials, const float* __re
     __syncthreads();
     const bool bad = (s.flags & COMPACTOR_STATUS_NONFINITE) != 0;
 
-    // ---- Cholesky, left-looking, one warp: at column j lane l owns rows j+l and j+l+32 ----------
+    // ---- Cholesky, left-looking, one warp: at column j lane l owns rows j+l, j+l+32, ... ---------
     if (warp == 0 && !bad) {
         int rank_flag = 0;
         for (int j = 0; j < m; ++j) {
-            double v[2];
+            double v[kH];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
+            for (int h = 0; h < kH; ++h) {
                 const int i = j + lane + 32 * h;
                 double a0 = 0.0, a1 = 0.0;
                 if (i < m) {
@@ -261,7 +269,7 @@ cholesky_kernel(Plan p, const double* __restrict__ g_partials, const float* __re
             if (!keep) rank_flag = 1;
             __syncwarp();
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
+            for (int h = 0; h < kH; ++h) {
                 const int i = j + lane + 32 * h;
                 if (i < m) s.g[i * LD + j] = (i == j) ? piv * inv : v[h] * inv;
             }
@@ -272,26 +280,39 @@ cholesky_kernel(Plan p, const double* __restrict__ g_partials, const float* __re
     }
     __syncthreads();
 
-    // ---- W = Phi L^-T: forward substitution along the row, which is held in registers ------------
+    // ---- W = Phi L^-T: forward substitution along the row, a block of columns in registers --------
     {
+        constexpr int kWB = WBlock<MP>::value;
         const int row = tid;
-        double r[MP];
-#pragma unroll
-        for (int c = 0; c < MP; ++c) r[c] = (c < m && !bad) ? (double)phi[row * m + c] : 0.0;
-#pragma unroll
-        for (int j = 0; j < MP; ++j) {
-            const double wj = r[j] * s.inv_diag[j];
-            r[j] = wj;
-#pragma unroll
-            for (int c = j + 1; c < MP; ++c) r[c] = fma(-wj, s.g[c * LD + j], r[c]);
-        }
         __nv_bfloat16* w_hi = w_out + (size_t)unit * w_elems_per_unit(MP);
         __nv_bfloat16* w_lo = w_hi + (size_t)MP * kD;
+#pragma unroll 1
+        for (int c0 = 0; c0 < MP; c0 += kWB) {
+            double r[kWB];
 #pragma unroll
-        for (int j = 0; j < MP; ++j) {
-            const __nv_bfloat16 hi = __double2bfloat16(r[j]);
-            w_hi[j * kD + row] = hi;
-            w_lo[j * kD + row] = __double2bfloat16(r[j] - (double)__bfloat162float(hi));
+            for (int c = 0; c < kWB; ++c) r[c] = (c0 + c < m && !bad) ? (double)phi[row * m + c0 + c] : 0.0;
+            for (int j = 0; j < c0; ++j) {                  // what the finished blocks take out of this one
+                const double wj = s.parked[j * kCholThreads + tid];
+#pragma unroll
+                for (int c = 0; c < kWB; ++c) r[c] = fma(-wj, s.g[(c0 + c) * LD + j], r[c]);
+            }
+#pragma unroll
+            for (int j = 0; j < kWB; ++j) {
+                const double wj = r[j] * s.inv_diag[c0 + j];
+                r[j] = wj;
+#pragma unroll
+                for (int c = j + 1; c < kWB; ++c) r[c] = fma(-wj, s.g[(c0 + c) * LD + c0 + j], r[c]);
+            }
+            if (c0 + kWB < MP) {
+#pragma unroll
+                for (int j = 0; j < kWB; ++j) s.parked[(c0 + j) * kCholThreads + tid] = r[j];
+            }
+#pragma unroll
+            for (int j = 0; j < kWB; ++j) {
+                const __nv_bfloat16 hi = __double2bfloat16(r[j]);
+                w_hi[(c0 + j) * kD + row] = hi;
+                w_lo[(c0 + j) * kD + row] = __double2bfloat16(r[j] - (double)__bfloat162float(hi));
+            }
         }
     }
     if (tid == 0 && status != nullptr && s.flags != 0) atomicOr(&status[unit], s.flags);
@@ -461,12 +482,19 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (factorization == COMPACTOR_FACTOR_EIG) {
-        const int esmem = (int)sizeof(EigSmem<MP>);
-        e = cudaFuncSetAttribute(eig_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, esmem);
-        if (e != cudaSuccess) return e;
-        eig_kernel<MP><<<units, kEigThreads, esmem, stream>>>(p, g_partials, phi, eig_floor, w, status);
+        if constexpr (MP <= 64) {
+            const int esmem = (int)sizeof(EigSmem<MP>);
+            e = cudaFuncSetAttribute(eig_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, esmem);
+            if (e != cudaSuccess) return e;
+            eig_kernel<MP><<<units, kEigThreads, esmem, stream>>>(p, g_partials, phi, eig_floor, w, status);
+        } else {
+            return cudaErrorInvalidValue;        // two m x m fp64 matrices no longer fit in shared memory
+        }
     } else {
-        cholesky_kernel<MP><<<units, kCholThreads, 0, stream>>>(p, g_partials, phi, w, status);
+        const int csmem = (int)sizeof(CholSmem<MP>);
+        e = cudaFuncSetAttribute(cholesky_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, csmem);
+        if (e != cudaSuccess) return e;
+        cholesky_kernel<MP><<<units, kCholThreads, csmem, stream>>>(p, g_partials, phi, w, status);
     }
     return cudaGetLastError();
 }
@@ -481,6 +509,7 @@ cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, c
         case 32: return launch_factor_mp<32>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
         case 48: return launch_factor_mp<48>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
         case 64: return launch_factor_mp<64>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
+        case 128: return launch_factor_mp<128>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -16,18 +16,20 @@ namespace {
 using namespace sm100;
 
 constexpr int kTile = 128;
-constexpr int kStages = 6;
+// Ring depth: six 32 KB stages, four when the W operand of a 128-column sketch takes 64 KB.
+template <int MP> struct Stages { static constexpr int value = MP <= 64 ? 6 : 4; };
 constexpr int kBoxBytes = kTile * 128;
 constexpr int kTileBytes = 2 * kBoxBytes;
 constexpr int kThreads = 192;
 // Tiles whose scores are stored together (4 KB bursts instead of 512 B); at MP = 64 the W operand
 // leaves no shared memory for that.
 template <int MP> struct OutTiles { static constexpr int value = MP <= 48 ? 8 : 1; };
-constexpr int kBufs = 4;                  // accumulators of up to 64 columns each
-constexpr uint32_t kTmemCols = 64 * kBufs;
+constexpr int kBufs = 4;                  // accumulators in rotation
+template <int MP> struct BufCols { static constexpr uint32_t value = MP <= 64 ? 64 : 128; };   // tensor-memory columns each
 
 template <int MP>
 struct __align__(1024) ScoreSmem {
+    static constexpr int kStages = Stages<MP>::value;
     unsigned char tiles[kStages][kTileBytes];
     unsigned char w[2][2][MP * 128];      // [term][channel half][MP rows x 64 channels]
     uint64_t full[kStages];
@@ -47,6 +49,9 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
              float* __restrict__ scores, int* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
     using Smem = ScoreSmem<MP>;
+    constexpr int kStages = Smem::kStages;
+    constexpr uint32_t kCols = BufCols<MP>::value;
+    constexpr uint32_t kTmemCols = kCols * kBufs;
     Smem& s = *reinterpret_cast<Smem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
     const int chunk_id = blockIdx.x;
     const int lh = blockIdx.y;
@@ -106,7 +111,7 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
             tc_fence_after_sync();
             if (lane == 0) {
                 const uint32_t a_base = smem_u32(s.tiles[stage]);
-                const uint32_t d_addr = tmem + buf * 64;
+                const uint32_t d_addr = tmem + buf * kCols;
 #pragma unroll
                 for (int term = 0; term < 2; ++term)
 #pragma unroll
@@ -144,7 +149,7 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
 #pragma unroll
             for (int c0 = 0; c0 < MP; c0 += 16) {
                 uint32_t r[16];
-                tmem_ld_32x32b_x16(tmem + ((uint32_t)(q * 32) << 16) + buf * 64 + c0, r);
+                tmem_ld_32x32b_x16(tmem + ((uint32_t)(q * 32) << 16) + buf * kCols + c0, r);
                 tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) { float v = __uint_as_float(r[i]); acc = fmaf(v, v, acc); }
@@ -195,6 +200,7 @@ cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, fl
         case 32: return launch_score_mp<32>(p, kmap, wmap, scores, status, stream);
         case 48: return launch_score_mp<48>(p, kmap, wmap, scores, status, stream);
         case 64: return launch_score_mp<64>(p, kmap, wmap, scores, status, stream);
+        case 128: return launch_score_mp<128>(p, kmap, wmap, scores, status, stream);
         default: return cudaErrorInvalidValue;
     }
 }

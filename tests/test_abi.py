@@ -85,7 +85,8 @@ def test_workspace_bytes():
     assert 0 < small < big < 4 << 30
     assert small % 256 == 0
     assert B.workspace_bytes(B.Shape(1, 2, 64, 48, [1024])) == 0          # d != 128
-    assert B.workspace_bytes(B.Shape(1, 2, 128, 65, [1024])) == 0         # m too large
+    assert B.workspace_bytes(B.Shape(1, 2, 128, 129, [1024])) == 0        # m too large
+    assert B.workspace_bytes(B.Shape(1, 2, 128, 128, [1024])) > small      # m = d: exact scores
     assert B.workspace_bytes(B.Shape(1, 2, 128, 48, [1024, 0, 77])) > 0   # empty sequences are fine
 
 

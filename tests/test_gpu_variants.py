@@ -131,3 +131,69 @@ def test_variant_argument_checks(B):
         with pytest.raises(B.CompactorError) as e:
             B.score_variant(shape, kr.cuda(), phi, out, ws, fact, floor)
         assert e.value.code == -1
+
+
+# ----------------------------------------------------------------------------- m = d: exact leverage scores
+def _score_with_phi(B, w, phi):
+    _, kr, _ = inputs.make_tensors(w, device="cpu", want_pre=False)
+    shape = B.Shape(w.layers, w.heads, w.d, phi.shape[1], w.seqlens)
+    ws = torch.empty(B.workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    scores = torch.full((w.layers, w.heads, sum(w.seqlens)), -1.0, dtype=torch.float32, device="cuda")
+    status = torch.full((w.layers * w.heads * len(w.seqlens),), -1, dtype=torch.int32, device="cuda")
+    B.score(shape, kr.cuda(), phi.cuda(), scores, ws, status=status)
+    torch.cuda.synchronize()
+    return kr, scores.cpu().numpy(), status.cpu().numpy().reshape(w.layers, w.heads, -1)
+
+
+@pytest.mark.parametrize("sketch", ["identity", "rotation"])
+def test_full_width_sketch_gives_exact_leverage_scores(B, sketch):
+    # Definition 1 / Eq. 1 (the "exact" row of the ablation): any invertible 128 x 128 sketch
+    # leaves the column space of K unchanged, so Algorithm 1 returns the exact scores.  The second
+    # sketch is a well-conditioned one (orthogonal times a mild column scaling): a square Gaussian
+    # matrix squares its own condition number into G, below what fp32 Gram sums resolve.
+    w = inputs.Workload("exact", 1, 2, 128, [1500, 5000, 300], [0.3, 0.3, 0.3], p=0.5, seed=51)
+    if sketch == "identity":
+        phi = torch.eye(128)
+    else:
+        q, _ = torch.linalg.qr(inputs.make_sketch_matrix(128, 128, 51).double())
+        phi = (q * torch.linspace(0.5, 2.0, 128, dtype=torch.float64)[None, :]).float()
+    k, got, status = _score_with_phi(B, w, phi)
+    worst = 0.0
+    for layer, head, b, t0, n in _units(w):
+        K = orc.bf16_bits_to_f64(_bits(k, layer, head, t0, n))
+        want = orc.exact_leverage_scores(K)
+        g = got[layer, head, t0:t0 + n]
+        worst = max(worst, np.max(np.abs(g - want) / want))
+        assert abs(g.sum() - 128.0) < 0.05                              # sum of leverage scores = rank
+        assert status[layer, head, b] == 0
+    print(f"exact scores ({sketch}): max rel err {worst:.2e}")
+    assert worst <= H.SCORE_RTOL
+
+
+def test_wide_sketch_between_64_and_128_columns(B):
+    w = inputs.Workload("m100", 1, 2, 128, [2100, 640], [0.3, 0.3], p=0.5, seed=52, m=100)
+    phi = inputs.make_sketch_matrix(128, 100, 52)
+    k, got, status = _score_with_phi(B, w, phi)
+    for layer, head, b, t0, n in _units(w):
+        K = orc.bf16_bits_to_f64(_bits(k, layer, head, t0, n))
+        np.testing.assert_allclose(got[layer, head, t0:t0 + n], orc.approx_leverage_scores(K, phi.double().numpy()),
+                                   rtol=H.SCORE_RTOL)
+
+
+def test_exact_scores_of_a_short_rank_deficient_sequence(B):
+    # fewer tokens than channels: rank n, every exact score is 1
+    w = inputs.Workload("exact-short", 1, 1, 128, [90], [0.5], p=0.5, seed=53)
+    k, got, status = _score_with_phi(B, w, torch.eye(128))
+    np.testing.assert_allclose(got[0, 0], np.ones(90), rtol=H.SCORE_RTOL)
+    assert status[0, 0, 0] & 2                                          # rank deficiency is reported
+
+
+def test_eig_route_rejects_wide_sketches(B):
+    w = inputs.Workload("eig-wide", 1, 1, 128, [300], [0.3], p=0.7, seed=54)
+    _, kr, _ = inputs.make_tensors(w, device="cpu", want_pre=False)
+    shape = B.Shape(1, 1, 128, 128, w.seqlens)
+    ws = torch.empty(B.workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    out = torch.empty((1, 1, 300), dtype=torch.float32, device="cuda")
+    with pytest.raises(B.CompactorError) as e:
+        B.score_variant(shape, kr.cuda(), torch.eye(128).cuda(), out, ws, B.FACTOR_EIG, 1e-6)
+    assert e.value.code == -2

@@ -126,6 +126,29 @@ int compactor_fit_calibration(int64_t n, const double* r, const double* nll, con
                               double under_weight, double* alpha_out, double* beta_out, double* loss_out);
 
 /*
+ * Token-averaged negative log-likelihood (Section 3.5): for each of `batch` sequences, the mean
+ * over its scored rows of -log softmax(logits_i)[targets_i].  This is the context statistic NLL(c)
+ * that compactor_calibrated_ratio turns into a retention ratio.
+ *   logits       device, [rows][vocab] with `row_stride` elements between rows; bf16
+ *                (logits_dtype COMPACTOR_DTYPE_BF16) or fp32 (COMPACTOR_DTYPE_F32); 16-byte aligned,
+ *                row_stride * element size a multiple of 16.
+ *   targets      device int32 [rows]: the token each row is scored on; a negative id (or one
+ *                >= vocab) leaves the row unscored: its row result is 0 and it does not count in
+ *                the average.
+ *   cu_rows      HOST int32 [batch+1], non-decreasing from 0 to rows: the rows of each sequence.
+ *   row_nll_out  device fp32 [rows], required: the per-row terms (also the kernel's scratch).
+ *   nll_out      device fp64 [batch]: the averages (0 for a sequence with no scored row).
+ * Arithmetic: one streaming pass in fp32 (running maximum, base-2 exponentials), averages in fp64
+ * in a fixed order.  No workspace.  Errors: COMPACTOR_E_INVALID_ARGUMENT for null pointers, bad
+ * alignment, vocab < 1, an unknown dtype or an inconsistent cu_rows.
+ */
+#define COMPACTOR_DTYPE_BF16 0
+#define COMPACTOR_DTYPE_F32  1
+int compactor_nll(const void* logits, int32_t logits_dtype, int64_t rows, int32_t vocab, int64_t row_stride,
+                  const int32_t* targets, int32_t batch, const int32_t* cu_rows,
+                  float* row_nll_out, double* nll_out, void* stream);
+
+/*
  * Bytes of device workspace that compactor_score and compactor_compress need for this shape.
  * compactor_select and compactor_compact only use a small table at its start and accept any
  * workspace of at least 12*(batch+1) bytes rounded up to 256.  The workspace must be 256-byte

@@ -24,6 +24,8 @@ What follows the paper step by step:
   * `top_k_across_heads`     - the same budget spent over all heads of a layer
     (Section 3.4's alternative; ties: lower head, then lower index).
   * `compact`                - the retained rows of K and V.
+  * `token_nll`, `mean_nll`  - the token-averaged negative log-likelihood of
+    Section 3.5, from logits and target ids.
   * `calibrated_ratio`       - inverse of the fitted curve f_{alpha,beta}
     (Section 3.5); `fit_calibration` - the asymmetric least-squares fit of
     (alpha, beta) on (r, NLL, y) triples.
@@ -295,6 +297,32 @@ def compact(K_bits: np.ndarray, V_bits: np.ndarray, idx: np.ndarray):
 # ----------------------------------------------------------------------------
 # Section 3.5: context-calibrated ratio
 # ----------------------------------------------------------------------------
+def token_nll(logits: np.ndarray, targets: np.ndarray) -> np.ndarray:
+    """-log softmax(logits_i)[targets_i] for every row i (Section 3.5: the summand of the
+    token-averaged NLL).  Rows whose target is negative are not scored and give 0."""
+    x = np.asarray(logits, dtype=np.float64)
+    t = np.asarray(targets, dtype=np.int64)
+    out = np.zeros(x.shape[0])
+    for i in range(x.shape[0]):
+        if t[i] < 0:
+            continue
+        row = x[i]
+        top = np.max(row)
+        log_z = top + math.log(float(np.sum(np.exp(row - top))))     # log of the softmax denominator
+        out[i] = log_z - row[t[i]]
+    return out
+
+
+def mean_nll(logits: np.ndarray, targets: np.ndarray) -> float:
+    """NLL(t; c) = -(1/L) sum_i log LM(t_i | ...) (Section 3.5), L counting the scored rows;
+    0 when no row is scored."""
+    t = np.asarray(targets, dtype=np.int64)
+    scored = int(np.sum(t >= 0))
+    if scored == 0:
+        return 0.0
+    return float(np.sum(token_nll(logits, targets)) / scored)
+
+
 def calibration_curve(r: float, b: float) -> float:
     """f(r) = (exp(r b - b) - exp(-b)) / (1 - exp(-b)); f(r) = r in the limit b -> 0."""
     if b == 0.0:

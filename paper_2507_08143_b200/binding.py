@@ -49,6 +49,8 @@ def _load() -> ctypes.CDLL:
                                     c_void_p, c_void_p, c_size_t, c_void_p]
     lib.compactor_score_variant.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_int32, c_double, c_void_p,
                                             c_float, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_nll.argtypes = [c_void_p, c_int32, c_int64, c_int32, c_int64, c_void_p, c_int32, POINTER(c_int32),
+                                  c_void_p, c_void_p, c_void_p]
     lib.compactor_select.argtypes = [POINTER(CompactorShape), c_void_p, POINTER(c_int32), c_void_p, c_void_p,
                                      c_void_p, c_size_t, c_void_p]
     lib.compactor_compact.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_void_p, POINTER(c_int32),
@@ -80,7 +82,7 @@ EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
            "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores", "compactor_wait_selftest",
            "compactor_across_heads_workspace_bytes", "compactor_select_across_heads", "compactor_compact_across_heads",
-           "compactor_score_variant"]
+           "compactor_score_variant", "compactor_nll"]
 
 FACTOR_CHOLESKY = 0
 FACTOR_EIG = 1
@@ -193,6 +195,26 @@ def score_variant(shape: Shape, k_score: torch.Tensor, phi: torch.Tensor, scores
     _check(LIB.compactor_score_variant(byref(shape.c), mat(k_score), _ptr(phi), factorization, eig_floor, _ptr(attn), lam,
                                        _ptr(scores_out), _ptr(status), _ptr(workspace), workspace.numel(), _stream()),
            "compactor_score_variant")
+
+
+def nll(logits: torch.Tensor, targets: torch.Tensor, seq_rows: Sequence[int], row_nll_out: torch.Tensor,
+        nll_out: torch.Tensor) -> None:
+    """Section 3.5: token-averaged NLL of each sequence from `logits` [rows, vocab] (bf16 or fp32,
+    unit stride along the vocabulary) and `targets` [rows] (int32, negative = unscored)."""
+    if logits.dtype == torch.bfloat16:
+        dtype = 0
+    elif logits.dtype == torch.float32:
+        dtype = 1
+    else:
+        raise TypeError("logits must be bf16 or fp32")
+    if logits.dim() != 2 or logits.stride(1) != 1 or targets.dtype != torch.int32:
+        raise ValueError("logits [rows, vocab] with unit inner stride and int32 targets expected")
+    cu = [0]
+    for n in seq_rows:
+        cu.append(cu[-1] + int(n))
+    cu_arr = (c_int32 * len(cu))(*cu)
+    _check(LIB.compactor_nll(_ptr(logits), dtype, logits.shape[0], logits.shape[1], logits.stride(0), _ptr(targets),
+                             len(seq_rows), cu_arr, _ptr(row_nll_out), _ptr(nll_out), _stream()), "compactor_nll")
 
 
 def select(shape: Shape, scores: torch.Tensor, keep_counts: Sequence[int], idx_out: torch.Tensor,

@@ -427,6 +427,26 @@ int compactor_score_builtin_scratch(const compactor_shape* shape, compactor_mat 
 }  // extern "C"
 
 // ---------------------------------------------------------------------------------------------
+// Token-averaged negative log-likelihood (Section 3.5).
+extern "C" int compactor_nll(const void* logits, int32_t logits_dtype, int64_t rows, int32_t vocab, int64_t row_stride,
+                             const int32_t* targets, int32_t batch, const int32_t* cu_rows, float* row_nll_out,
+                             double* nll_out, void* stream) {
+    if (logits_dtype != COMPACTOR_DTYPE_BF16 && logits_dtype != COMPACTOR_DTYPE_F32) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (rows < 0 || vocab < 1 || batch < 0 || cu_rows == nullptr || row_stride < vocab) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (cu_rows[0] != 0 || cu_rows[batch] != rows) return COMPACTOR_E_INVALID_ARGUMENT;
+    for (int b = 0; b < batch; ++b)
+        if (cu_rows[b + 1] < cu_rows[b]) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (batch == 0) return COMPACTOR_OK;
+    if (nll_out == nullptr) return COMPACTOR_E_INVALID_ARGUMENT;
+    if (rows > 0 && (logits == nullptr || targets == nullptr || row_nll_out == nullptr)) return COMPACTOR_E_INVALID_ARGUMENT;
+    const size_t esize = logits_dtype == COMPACTOR_DTYPE_F32 ? 4 : 2;
+    if (((uintptr_t)logits & 15) != 0 || ((size_t)row_stride * esize) % 16 != 0) return COMPACTOR_E_INVALID_ARGUMENT;
+    CK(launch_nll(logits, logits_dtype == COMPACTOR_DTYPE_F32, rows, vocab, row_stride, targets, batch, cu_rows,
+                  row_nll_out, nll_out, static_cast<cudaStream_t>(stream)));
+    return COMPACTOR_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Attention term (Eq. 5).
 extern "C" int compactor_attention_scores(const compactor_shape* shape, compactor_mat q, compactor_mat k,
                                           int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,

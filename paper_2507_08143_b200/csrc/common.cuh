@@ -58,6 +58,10 @@ cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStre
 cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int* idx,
                            __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream);
 
+cudaError_t launch_nll(const void* logits, int is_fp32, long long rows, int vocab, long long row_stride,
+                       const int* targets, int batch, const int* cu_rows_host, float* row_nll, double* nll_out,
+                       cudaStream_t stream);
+
 cudaError_t launch_select_across(const Plan& p, const float* scores, int* idx, int* head_offsets, uint32_t* thr,
                                  int* ties, cudaStream_t stream);
 cudaError_t launch_compact_across(const Plan& p, const Mat& k, const Mat& v, const int* idx, const int* head_offsets,

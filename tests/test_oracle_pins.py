@@ -296,6 +296,35 @@ def test_calibrated_ratio():
     assert orc.calibrated_ratio(1.0, -10, 0, 0.95) < orc.calibrated_ratio(1.0, -4, 0, 0.95)
 
 
+def test_nll_pins():
+    rng = _rng(61)
+    # equal logits: every token has probability 1/V
+    np.testing.assert_allclose(orc.token_nll(np.full((3, 50), 2.5), [0, 7, 49]), np.full(3, math.log(50)), rtol=1e-14)
+    # two-way softmax is the logistic function: -log sigmoid(a - b)
+    a, b = 1.3, -0.4
+    np.testing.assert_allclose(orc.token_nll([[a, b]], [0]), [math.log1p(math.exp(b - a))], rtol=1e-14)
+    np.testing.assert_allclose(orc.token_nll([[a, b]], [1]), [math.log1p(math.exp(a - b))], rtol=1e-14)
+    # a dominant logit: picking it costs nothing, picking another costs the gap
+    row = np.zeros(10); row[4] = 800.0
+    np.testing.assert_allclose(orc.token_nll([row, row], [4, 2]), [0.0, 800.0], atol=1e-12)
+    # brute force against probabilities multiplied out, and invariance under a shift of a row
+    x = rng.standard_normal((6, 9)) * 3
+    t = rng.integers(0, 9, size=6)
+    p = np.exp(x) / np.sum(np.exp(x), axis=1, keepdims=True)
+    want = -np.log(p[np.arange(6), t])
+    np.testing.assert_allclose(orc.token_nll(x, t), want, rtol=1e-12)
+    np.testing.assert_allclose(orc.token_nll(x + 1000.0, t), want, rtol=1e-9)
+    assert abs(orc.mean_nll(x, t) - want.mean()) < 1e-12
+    # the probabilities of all targets of one row sum to one
+    full = np.tile(x[0], (9, 1))
+    assert abs(np.sum(np.exp(-orc.token_nll(full, np.arange(9)))) - 1.0) < 1e-12
+    # unscored rows: excluded from the average, and an average over nothing is 0
+    t2 = t.copy(); t2[[1, 4]] = -1
+    assert abs(orc.mean_nll(x, t2) - want[[0, 2, 3, 5]].mean()) < 1e-12
+    assert orc.token_nll(x, t2)[1] == 0.0
+    assert orc.mean_nll(x, np.full(6, -1)) == 0.0
+
+
 def test_fit_calibration_recovers_known_parameters():
     rng = _rng(15)
     alpha, beta = -1.7, -0.8

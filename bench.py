@@ -46,6 +46,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-units", type=int, default=16, help="units in the CPU-baseline sample")
+    ap.add_argument("--fig1-n", type=int, default=None, help="with --fig1: only this context length")
+    ap.add_argument("--nll", action="store_true",
+                    help="time the NLL reduction of Section 3.5 on 8192 x 128256 bf16 logits instead of the headline")
     ap.add_argument("--fig1", action="store_true",
                     help="context-length sweep of the paper's Fig. 1 setting (one layer, 8 KV heads, batch 1)")
     return ap.parse_args()
@@ -229,6 +232,8 @@ def run_fig1(args):
     torch.cuda.set_device(0)
     rows = []
     for n in sorted(FIG1_PAPER_MS_H100):
+        if args.fig1_n is not None and n != args.fig1_n:
+            continue
         w = inputs.Workload(f"fig1-n{n}", 1, 8, 128, [n], [0.3], p=0.7, n_out=4, theta=5e5, seed=100)
         _, kr, v = inputs.make_tensors(w, device="cuda", want_pre=False)
         shape = B.Shape(1, 8, 128, 48, [n])
@@ -274,8 +279,37 @@ def run_fig1(args):
                       "timing": "median of CUDA-event times, L2 flushed before every call"}))
 
 
+def run_nll(args):
+    """Streaming rate of compactor_nll on synthetic logits of a 128K-entry vocabulary."""
+    import torch
+    from paper_2507_08143_b200 import binding as B
+    torch.cuda.set_device(0)
+    rows, vocab = 8192, 128256
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    logits = (torch.randn(rows, vocab, device="cuda", generator=g) * 4).to(torch.bfloat16)
+    targets = torch.randint(0, vocab, (rows,), device="cuda", generator=g, dtype=torch.int32)
+    row_nll = torch.empty(rows, dtype=torch.float32, device="cuda")
+    out = torch.empty(1, dtype=torch.float64, device="cuda")
+    for _ in range(max(3, args.warmup)):
+        B.nll(logits, targets, [rows], row_nll, out)
+    times = []
+    for _ in range(max(5, args.steps)):                     # 2.1 GB of logits per call: larger than L2
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); B.nll(logits, targets, [rows], row_nll, out); e1.record(); torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ms = statistics.median(times)
+    peak, kind = measured_peak()
+    gbs = rows * vocab * 2 / ms / 1e6
+    print(json.dumps({"nll": {"rows": rows, "vocab": vocab, "dtype": "bf16", "ms": round(ms, 4), "GB/s": round(gbs, 1),
+                              "frac": round(gbs / peak, 4), "peak": peak, "peak_kind": "of " + kind,
+                              "mean_nll": float(out.cpu()[0])}}))
+
+
 def main():
     args = parse_args()
+    if args.nll:
+        run_nll(args)
+        return
     if args.impl == "reference":
         run_reference(args)
         return

@@ -9,8 +9,10 @@
 // warp 1 issues, per half, S = Q_half K^T (tcgen05.mma, 128 x 256 fp32 in tensor memory).  Warps
 // 2-9 share the 128 query rows (a pair of warps per 32 rows, 128 keys each): row maximum, e = exp(scale (s - max)) written as fp16 into shared
 // memory in the layout of an MN-major B operand, and the reciprocal of the row sum (two fp16 terms)
-// into rows 0 and 1 of a small A operand.  A second MMA then adds w^T E (1 x 256, the normalised column sums of the half)
-// into a second accumulator that runs over all halves and query heads; it is read out once.
+// into rows 0 and 1 of a small K-major operand w.  A second MMA, E^T w (keys x 2: the half's normalised column sums),
+// lands in 32 columns of the half's own S accumulator once the softmax warps are done with S; four warps
+// add it to two registers per thread and write the chunk's result at the end.  S has two accumulators, so
+// that the products of the next half run beside the softmax of the current one.
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -29,14 +31,18 @@ constexpr int kKBox = kChunk * 128;        // 64 channels x 256 tokens x 2 B
 constexpr int kQBox = kHalf * 128;         // 64 channels x 128 rows
 constexpr int kPBlock = kHalf * 128;       // 128 rows x 64 keys, fp16
 constexpr int kWBox = 64 * 128;            // 64 rows x 64 k, fp16
-constexpr uint32_t kTmemCols = 512;        // S at column 0, column sums at column 256
+constexpr uint32_t kTmemCols = 512;        // two S accumulators of 256 columns; a half's column sums reuse 32 columns of its own
 
 struct __align__(1024) AttnSmem {
     unsigned char k[2 * kKBox];
     unsigned char q[2][2 * kQBox];
     unsigned char p[4 * kPBlock];
     unsigned char w[2 * kWBox];
-    uint64_t k_full, q_full[2], q_empty[2], s_full, p_ready, d_full;
+    uint64_t k_full, q_full[2], q_empty[2];
+    uint64_t s_full[2];        // S of a half is in accumulator (half & 1)
+    uint64_t p_ready;          // E and the weights of a half are in shared memory, its S is consumed
+    uint64_t c_full[2];        // the half's column sums are in its accumulator; E and the weights may be overwritten
+    uint64_t drained[2];       // the column sums have been taken out: the accumulator may be overwritten
     float xmax[2][kHalf];      // row maxima / row sums of the two column halves, exchanged between warp pairs
     float xsum[2][kHalf];
     uint32_t tmem_base;
@@ -71,14 +77,13 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         prefetch_tensormap(&kmap);
         mbar_init(&s.k_full, 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 1); }
-        mbar_init(&s.s_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&s.s_full[i], 1); mbar_init(&s.c_full[i], 1); mbar_init(&s.drained[i], 4); }
         mbar_init(&s.p_ready, 32 * kSoftmaxWarps);
-        mbar_init(&s.d_full, 1);
         s.abort = 0;
         s.abort_mma = 0;
         fence_barrier_init();
     }
-    for (int i = threadIdx.x; i < 2 * kWBox / 16; i += kThreads)       // rows 1..63 of the weight operand stay zero
+    for (int i = threadIdx.x; i < 2 * kWBox / 16; i += kThreads)       // rows 2.. of the weight operand stay zero
         reinterpret_cast<uint4*>(s.w)[i] = make_uint4(0, 0, 0, 0);
     fence_proxy_async_smem();
     if (warp == 1) { tmem_alloc(&s.tmem_base, kTmemCols); tmem_relinquish(); }
@@ -105,74 +110,96 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         }
     } else if (warp == 1) {
         constexpr uint32_t idesc_s = umma_idesc_16bit(1, 128, kChunk, 0, 0);     // bf16: Q (K-major) x K^T (K-major)
-        constexpr uint32_t idesc_c = umma_idesc_16bit(0, 64, kChunk, 0, 1);      // fp16: w (K-major) x E (MN-major)
+        constexpr uint32_t idesc_c = umma_idesc_16bit(0, 128, 16, 1, 0);         // fp16: E^T (MN-major: keys x rows) x w (K-major)
         const uint32_t k_base = smem_u32(s.k), p_base = smem_u32(s.p), w_base = smem_u32(s.w);
-        auto column_sums = [&](int it) {           // adds w^T E of half `it` into the second accumulator
+        // Column sums of half `it`: D[key][0..1] = sum_rows E[row][key] * (hi, lo of 1 / row sum), keys 0-127 in
+        // columns 0-15 and keys 128-255 in columns 16-31 of the half's own accumulator, whose S is consumed.
+        auto column_sums = [&](int it) {
+            const uint32_t d = tmem + (uint32_t)(it & 1) * 256;
 #pragma unroll
-            for (int ks = 0; ks < kHalf / 16; ++ks) {
-                const uint64_t a_desc = umma_desc_sw128(w_base + (ks >> 2) * kWBox + (ks & 3) * 32, 16, 1024);
-                const uint64_t b_desc = umma_desc_sw128(p_base + ks * 2048, kPBlock, 1024);
-                umma_bf16(tmem + 256, a_desc, b_desc, idesc_c, (it > 0) || (ks > 0));
-            }
+            for (int kh = 0; kh < 2; ++kh)
+#pragma unroll
+                for (int ks = 0; ks < kHalf / 16; ++ks) {
+                    const uint64_t a_desc = umma_desc_sw128(p_base + kh * 2 * kPBlock + ks * 2048, kPBlock, 1024);
+                    const uint64_t b_desc = umma_desc_sw128(w_base + (ks >> 2) * kWBox + (ks & 3) * 32, 16, 1024);
+                    umma_bf16(d + kh * 16, a_desc, b_desc, idesc_c, ks > 0);
+                }
         };
         bool ok = mbar_wait(&s.k_full, 0);
         for (int it = 0; it < n_iter && ok; ++it) {
             const int st = it & 1, use = it >> 1;
             ok = mbar_wait(&s.q_full[st], use & 1);
-            if (ok && it > 0) ok = mbar_wait(&s.p_ready, (it - 1) & 1);     // S consumed, E and w of the previous half written
+            if (ok && it >= 2) ok = mbar_wait(&s.drained[st], (use - 1) & 1);  // the accumulator's previous column sums are out
             ok = ok && !*(volatile int*)&s.abort;
             if (!ok) break;
             tc_fence_after_sync();
             if (lane == 0) {
-                if (it > 0) column_sums(it - 1);
                 const uint32_t q_base = smem_u32(s.q[st]);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t a_desc = umma_desc_sw128(q_base + (ks >> 2) * kQBox + (ks & 3) * 32, 16, 1024);
                     const uint64_t b_desc = umma_desc_sw128(k_base + (ks >> 2) * kKBox + (ks & 3) * 32, 16, 1024);
-                    umma_bf16(tmem, a_desc, b_desc, idesc_s, ks > 0);
+                    umma_bf16(tmem + (uint32_t)st * 256, a_desc, b_desc, idesc_s, ks > 0);
                 }
                 umma_commit(&s.q_empty[st]);
-                umma_commit(&s.s_full);
+                umma_commit(&s.s_full[st]);
             }
             __syncwarp();
+            if (it > 0) {                                   // the previous half's softmax ran beside the products above
+                ok = mbar_wait(&s.p_ready, (it - 1) & 1);
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (lane == 0) { column_sums(it - 1); umma_commit(&s.c_full[(it - 1) & 1]); }
+                __syncwarp();
+            }
         }
         if (ok) ok = mbar_wait(&s.p_ready, (n_iter - 1) & 1);
         if (ok) {
             tc_fence_after_sync();
-            if (lane == 0) { column_sums(n_iter - 1); umma_commit(&s.d_full); }
+            if (lane == 0) { column_sums(n_iter - 1); umma_commit(&s.c_full[(n_iter - 1) & 1]); }
             __syncwarp();
         } else {
             s.abort = 1;
             s.abort_mma = 1;
             __threadfence_block();
             __syncwarp();
-            if (lane == 0) { mbar_arrive(&s.s_full); mbar_arrive(&s.d_full); }     // wake the other warps
+            if (lane == 0)                                  // wake the other warps
+                for (int i = 0; i < 2; ++i) { mbar_arrive(&s.s_full[i]); mbar_arrive(&s.c_full[i]); }
         }
     } else {
         const int q = warp & 3;                              // TMEM lane quadrant
         const int ch = (warp - 2) >> 2;                      // which 128 of the 256 keys
         const int row = q * 32 + lane;                       // query row within the half = TMEM lane
-        const uint32_t lane_addr = tmem + ((uint32_t)(q * 32) << 16) + ch * 128;
+        const uint32_t quad_addr = tmem + ((uint32_t)(q * 32) << 16);
         const bool full = n_tok == kChunk;                   // only the last chunk of a sequence needs masks
+        float col0 = 0.f, col1 = 0.f;                        // ch == 0: column sums of keys `row` and 128 + `row`
+        auto take_column_sums = [&](int it) {                // TMEM lane = key within its half of the chunk
+            uint32_t c[2], d[2];
+            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(it & 1) * 256, c);
+            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(it & 1) * 256 + 16, d);
+            tmem_ld_wait();
+            col0 += __uint_as_float(c[0]) + __uint_as_float(c[1]);       // hi and lo weights
+            col1 += __uint_as_float(d[0]) + __uint_as_float(d[1]);
+        };
         bool ok = true;
         for (int it = 0; it < n_iter && ok; ++it) {
-            // every softmax thread takes the same decision here (they meet at a named barrier below)
-            ok = mbar_wait(&s.s_full, it & 1) && !*(volatile int*)&s.abort_mma;
+            // every softmax thread takes the same decisions here (they meet at a named barrier below)
+            ok = mbar_wait(&s.s_full[it & 1], (it >> 1) & 1) && !*(volatile int*)&s.abort_mma;
             if (!ok) break;
             tc_fence_after_sync();
+            const uint32_t lane_addr = quad_addr + (uint32_t)(it & 1) * 256 + ch * 128;
             const bool row_valid = (it & 1) * kHalf + row < n_tok;
-            float mx = -INFINITY;
             // the load of the next 32 columns is in flight while this thread works on the current ones
             uint32_t ra[32], rb[32];
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
             auto max_of = [&](const uint32_t (&r)[32], int c0) {
                 if (full) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+                    for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (ch * 128 + c0 + i < n_tok) mx = fmaxf(mx, __uint_as_float(r[i]));
+                        if (ch * 128 + c0 + i < n_tok) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
                 }
             };
             tmem_ld_32x32b_x32(lane_addr, ra);
@@ -187,11 +214,24 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             max_of(ra, 64);
             tmem_ld_wait_for(rb);
             max_of(rb, 96);
-            s.xmax[ch][row] = mx;
+            s.xmax[ch][row] = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
             softmax_pair_sync();
-            mx = fmaxf(s.xmax[0][row], s.xmax[1][row]);      // finite: key 0 of the chunk always exists
+            const float mx = fmaxf(s.xmax[0][row], s.xmax[1][row]);      // finite: key 0 of the chunk always exists
             const float bias = -mx * scale_log2e;
-            float sum = 0.f;
+            if (it > 0) {
+                // E and the weights of the previous half have been multiplied: they may be overwritten,
+                // and its column sums are waiting in its accumulator
+                ok = mbar_wait(&s.c_full[(it - 1) & 1], ((it - 1) >> 1) & 1) && !*(volatile int*)&s.abort_mma;
+                if (!ok) break;
+                if (ch == 0) {
+                    tc_fence_after_sync();
+                    take_column_sums(it - 1);
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&s.drained[(it - 1) & 1]);
+                }
+            }
+            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
             auto exp_of = [&](const uint32_t (&r)[32], int c0) {
                 uint32_t packed[16];
 #pragma unroll
@@ -202,7 +242,7 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                         if (!row_valid || ch * 128 + c0 + i >= n_tok) e0 = 0.f;
                         if (!row_valid || ch * 128 + c0 + i + 1 >= n_tok) e1 = 0.f;
                     }
-                    sum += e0 + e1;
+                    sum4[(i >> 1) & 3] += e0 + e1;
                     const __half2 h = __floats2half2_rn(e0, e1);
                     packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&h);
                 }
@@ -227,11 +267,11 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             exp_of(ra, 64);
             tmem_ld_wait_for(rb);
             exp_of(rb, 96);
-            s.xsum[ch][row] = sum;
+            s.xsum[ch][row] = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
             softmax_pair_sync();
             if (ch == 0) {
                 // 1 / (row sum) as two fp16 terms in rows 0 and 1 of the weight operand (row 1 is swizzled by its index)
-                sum = s.xsum[0][row] + s.xsum[1][row];
+                const float sum = s.xsum[0][row] + s.xsum[1][row];
                 const float wgt = (row_valid && sum > 0.f) ? 1.0f / sum : 0.f;
                 const __half w_hi = __float2half_rn(wgt);
                 const __half w_lo = __float2half_rn(wgt - __half2float(w_hi));
@@ -245,23 +285,15 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             mbar_arrive(&s.p_ready);
         }
         if (!ok) s.abort = 1;
-        if (q == 0 && ch == 0) {                             // lanes 0-31 of tensor memory: rows 0 and 1 hold the column sums
-            const bool okd = ok && mbar_wait(&s.d_full, 0) && !*(volatile int*)&s.abort_mma;
+        if (ch == 0) {                                       // the last half's column sums, then the chunk's result
+            const int last = n_iter - 1;
+            const bool okd = ok && mbar_wait(&s.c_full[last & 1], (last >> 1) & 1) && !*(volatile int*)&s.abort_mma;
             tc_fence_after_sync();
             if (okd) {
+                take_column_sums(last);
                 float* dst = out + (size_t)lh * p.total_tokens + tok_begin;
-#pragma unroll 1
-                for (int c0 = 0; c0 < kChunk; c0 += 32) {
-                    uint32_t r[32];
-                    tmem_ld_32x32b_x32(tmem + 256 + c0, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float v = __uint_as_float(r[i]);
-                        const float total = v + __shfl_sync(0xffffffffu, v, 1);      // rows 0 and 1: hi and lo weights
-                        if (lane == 0 && c0 + i < n_tok) dst[c0 + i] = total;
-                    }
-                }
+                if (row < n_tok) dst[row] = col0;
+                if (kHalf + row < n_tok) dst[kHalf + row] = col1;
             }
         }
     }

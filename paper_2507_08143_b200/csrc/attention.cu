@@ -38,7 +38,7 @@ struct __align__(1024) AttnSmem {
     unsigned char q[2][2 * kQBox];
     unsigned char p[4 * kPBlock];
     unsigned char w[2 * kWBox];
-    uint64_t k_full, q_full[2], q_empty[2];
+    uint64_t k_full, k_empty, q_full[2], q_empty[2];
     uint64_t s_full[2];        // S of a half is in accumulator (half & 1)
     uint64_t p_ready;          // E and the weights of a half are in shared memory, its S is consumed
     uint64_t c_full[2];        // the half's column sums are in its accumulator; E and the weights may be overwritten
@@ -55,27 +55,39 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void softmax_pair_sync() {          // the 256 softmax threads only
-    asm volatile("bar.sync 1, 256;" ::: "memory");
+__device__ __forceinline__ void softmax_pair_sync(int q) {     // the two warps that share 32 query rows
+    asm volatile("bar.sync %0, 64;" :: "r"(q + 1) : "memory");
 }
 
+// Where a work item (one chunk of one layer and KV head) lies.
+struct AttnItem { int layer, head, lh, tok_begin, n_tok; };
+__device__ __forceinline__ AttnItem attn_item(const Plan& p, int item) {
+    AttnItem a;
+    a.lh = item / p.total_chunks;
+    const int chunk_id = item % p.total_chunks;
+    a.layer = a.lh / p.heads; a.head = a.lh % p.heads;
+    const int b = find_segment(p.cu_chunks, p.batch, chunk_id);
+    a.tok_begin = p.cu_seqlens[b] + (chunk_id - p.cu_chunks[b]) * kChunk;
+    a.n_tok = min(kChunk, p.cu_seqlens[b + 1] - a.tok_begin);
+    return a;
+}
+
+// Persistent: CTA c takes items c, c + grid, ...; barriers, tensor memory and the zeroed weight operand are set
+// up once.  Halves are numbered through all of a CTA's items (g), which fixes every barrier's phase.
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
-                 int q_per_kv, float scale_log2e, float* __restrict__ out) {
+                 int q_per_kv, float scale_log2e, int n_items, float* __restrict__ out) {
     extern __shared__ unsigned char smem_raw[];
     AttnSmem& s = *reinterpret_cast<AttnSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
-    const int chunk_id = blockIdx.x, lh = blockIdx.y;
-    const int layer = lh / p.heads, head = lh % p.heads;
-    const int b = find_segment(p.cu_chunks, p.batch, chunk_id);
-    const int tok_begin = p.cu_seqlens[b] + (chunk_id - p.cu_chunks[b]) * kChunk;
-    const int n_tok = min(kChunk, p.cu_seqlens[b + 1] - tok_begin);
-    const int n_iter = 2 * q_per_kv;                   // halves of 128 query rows
+    const int n_iter = 2 * q_per_kv;                   // halves of 128 query rows per item (even)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int my_items = ((int)blockIdx.x < n_items) ? (n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
     if (threadIdx.x == 0) {
         prefetch_tensormap(&qmap);
         prefetch_tensormap(&kmap);
         mbar_init(&s.k_full, 1);
+        mbar_init(&s.k_empty, 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&s.s_full[i], 1); mbar_init(&s.c_full[i], 1); mbar_init(&s.drained[i], 4); }
         mbar_init(&s.p_ready, 32 * kSoftmaxWarps);
@@ -94,28 +106,33 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_arrive_expect_tx(&s.k_full, 2 * kKBox);
-            tma_load_4d(s.k, &kmap, &s.k_full, 0, tok_begin, head, layer);
-            tma_load_4d(s.k + kKBox, &kmap, &s.k_full, 64, tok_begin, head, layer);
-            for (int it = 0; it < n_iter; ++it) {
-                const int st = it & 1, use = it >> 1;
-                if (use > 0 && !mbar_wait(&s.q_empty[st], (use - 1) & 1)) { s.abort = 1; break; }
-                if (*(volatile int*)&s.abort) break;
-                mbar_arrive_expect_tx(&s.q_full[st], 2 * kQBox);
-                const int qhead = head * q_per_kv + (it >> 1);
-                const int row = tok_begin + (it & 1) * kHalf;
-                tma_load_4d(s.q[st], &qmap, &s.q_full[st], 0, row, qhead, layer);
-                tma_load_4d(s.q[st] + kQBox, &qmap, &s.q_full[st], 64, row, qhead, layer);
+            bool ok = true;
+            for (int r = 0; r < my_items && ok; ++r) {
+                const AttnItem a = attn_item(p, blockIdx.x + r * gridDim.x);
+                if (r > 0 && !mbar_wait(&s.k_empty, (r - 1) & 1)) { s.abort = 1; break; }   // the previous item's S products are done
+                mbar_arrive_expect_tx(&s.k_full, 2 * kKBox);
+                tma_load_4d(s.k, &kmap, &s.k_full, 0, a.tok_begin, a.head, a.layer);
+                tma_load_4d(s.k + kKBox, &kmap, &s.k_full, 64, a.tok_begin, a.head, a.layer);
+                for (int it = 0; it < n_iter; ++it) {
+                    const int g = r * n_iter + it, st = g & 1, use = g >> 1;
+                    if (use > 0 && !mbar_wait(&s.q_empty[st], (use - 1) & 1)) { s.abort = 1; ok = false; break; }
+                    if (*(volatile int*)&s.abort) { ok = false; break; }
+                    mbar_arrive_expect_tx(&s.q_full[st], 2 * kQBox);
+                    const int qhead = a.head * q_per_kv + (it >> 1);
+                    const int row = a.tok_begin + (it & 1) * kHalf;
+                    tma_load_4d(s.q[st], &qmap, &s.q_full[st], 0, row, qhead, a.layer);
+                    tma_load_4d(s.q[st] + kQBox, &qmap, &s.q_full[st], 64, row, qhead, a.layer);
+                }
             }
         }
     } else if (warp == 1) {
         constexpr uint32_t idesc_s = umma_idesc_16bit(1, 128, kChunk, 0, 0);     // bf16: Q (K-major) x K^T (K-major)
         constexpr uint32_t idesc_c = umma_idesc_16bit(0, 128, 16, 1, 0);         // fp16: E^T (MN-major: keys x rows) x w (K-major)
         const uint32_t k_base = smem_u32(s.k), p_base = smem_u32(s.p), w_base = smem_u32(s.w);
-        // Column sums of half `it`: D[key][0..1] = sum_rows E[row][key] * (hi, lo of 1 / row sum), keys 0-127 in
+        // Column sums of half g: D[key][0..1] = sum_rows E[row][key] * (hi, lo of 1 / row sum), keys 0-127 in
         // columns 0-15 and keys 128-255 in columns 16-31 of the half's own accumulator, whose S is consumed.
-        auto column_sums = [&](int it) {
-            const uint32_t d = tmem + (uint32_t)(it & 1) * 256;
+        auto column_sums = [&](int g) {
+            const uint32_t d = tmem + (uint32_t)(g & 1) * 256;
 #pragma unroll
             for (int kh = 0; kh < 2; ++kh)
 #pragma unroll
@@ -125,11 +142,13 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                     umma_bf16(d + kh * 16, a_desc, b_desc, idesc_c, ks > 0);
                 }
         };
-        bool ok = mbar_wait(&s.k_full, 0);
-        for (int it = 0; it < n_iter && ok; ++it) {
-            const int st = it & 1, use = it >> 1;
-            ok = mbar_wait(&s.q_full[st], use & 1);
-            if (ok && it >= 2) ok = mbar_wait(&s.drained[st], (use - 1) & 1);  // the accumulator's previous column sums are out
+        const int n_halves = my_items * n_iter;
+        bool ok = true;
+        for (int g = 0; g < n_halves && ok; ++g) {
+            const int r = g / n_iter, it = g - r * n_iter, st = g & 1, use = g >> 1;
+            if (it == 0) ok = mbar_wait(&s.k_full, r & 1);
+            if (ok) ok = mbar_wait(&s.q_full[st], use & 1);
+            if (ok && g >= 2) ok = mbar_wait(&s.drained[st], (use - 1) & 1);   // the accumulator's previous column sums are out
             ok = ok && !*(volatile int*)&s.abort;
             if (!ok) break;
             tc_fence_after_sync();
@@ -143,21 +162,24 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                 }
                 umma_commit(&s.q_empty[st]);
                 umma_commit(&s.s_full[st]);
+                if (it == n_iter - 1) umma_commit(&s.k_empty);                // the item's keys are no longer needed
             }
             __syncwarp();
-            if (it > 0) {                                   // the previous half's softmax ran beside the products above
-                ok = mbar_wait(&s.p_ready, (it - 1) & 1);
+            if (g > 0) {                                    // the previous half's softmax ran beside the products above
+                ok = mbar_wait(&s.p_ready, (g - 1) & 1);
                 if (!ok) break;
                 tc_fence_after_sync();
-                if (lane == 0) { column_sums(it - 1); umma_commit(&s.c_full[(it - 1) & 1]); }
+                if (lane == 0) { column_sums(g - 1); umma_commit(&s.c_full[(g - 1) & 1]); }
                 __syncwarp();
             }
         }
-        if (ok) ok = mbar_wait(&s.p_ready, (n_iter - 1) & 1);
+        if (ok && n_halves > 0) ok = mbar_wait(&s.p_ready, (n_halves - 1) & 1);
         if (ok) {
-            tc_fence_after_sync();
-            if (lane == 0) { column_sums(n_iter - 1); umma_commit(&s.c_full[(n_iter - 1) & 1]); }
-            __syncwarp();
+            if (n_halves > 0) {
+                tc_fence_after_sync();
+                if (lane == 0) { column_sums(n_halves - 1); umma_commit(&s.c_full[(n_halves - 1) & 1]); }
+                __syncwarp();
+            }
         } else {
             s.abort = 1;
             s.abort_mma = 1;
@@ -171,35 +193,46 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         const int ch = (warp - 2) >> 2;                      // which 128 of the 256 keys
         const int row = q * 32 + lane;                       // query row within the half = TMEM lane
         const uint32_t quad_addr = tmem + ((uint32_t)(q * 32) << 16);
-        const bool full = n_tok == kChunk;                   // only the last chunk of a sequence needs masks
         float col0 = 0.f, col1 = 0.f;                        // ch == 0: column sums of keys `row` and 128 + `row`
-        auto take_column_sums = [&](int it) {                // TMEM lane = key within its half of the chunk
+        auto take_column_sums = [&](int g) {                 // TMEM lane = key within its half of the chunk
             uint32_t c[2], d[2];
-            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(it & 1) * 256, c);
-            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(it & 1) * 256 + 16, d);
+            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(g & 1) * 256, c);
+            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(g & 1) * 256 + 16, d);
             tmem_ld_wait();
             col0 += __uint_as_float(c[0]) + __uint_as_float(c[1]);       // hi and lo weights
             col1 += __uint_as_float(d[0]) + __uint_as_float(d[1]);
         };
+        auto write_result = [&](const AttnItem& a) {         // an item's column sums are complete
+            float* dst = out + (size_t)a.lh * p.total_tokens + a.tok_begin;
+            if (row < a.n_tok) dst[row] = col0;
+            if (kHalf + row < a.n_tok) dst[kHalf + row] = col1;
+            col0 = 0.f; col1 = 0.f;
+        };
+        const int n_halves = my_items * n_iter;
+        AttnItem cur = attn_item(p, blockIdx.x), prev = cur;
         bool ok = true;
-        for (int it = 0; it < n_iter && ok; ++it) {
-            // every softmax thread takes the same decisions here (they meet at a named barrier below)
-            ok = mbar_wait(&s.s_full[it & 1], (it >> 1) & 1) && !*(volatile int*)&s.abort_mma;
+        for (int g = 0; g < n_halves && ok; ++g) {
+            const int r = g / n_iter, it = g - r * n_iter;
+            if (it == 0 && r > 0) { prev = cur; cur = attn_item(p, blockIdx.x + r * gridDim.x); }
+            const int n_tok = cur.n_tok;
+            const bool full = n_tok == kChunk;               // only the last chunk of a sequence needs masks
+            // the two warps of a pair take the same decisions here (they meet at a named barrier below)
+            ok = mbar_wait(&s.s_full[g & 1], (g >> 1) & 1) && !*(volatile int*)&s.abort_mma;
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t lane_addr = quad_addr + (uint32_t)(it & 1) * 256 + ch * 128;
+            const uint32_t lane_addr = quad_addr + (uint32_t)(g & 1) * 256 + ch * 128;
             const bool row_valid = (it & 1) * kHalf + row < n_tok;
             // the load of the next 32 columns is in flight while this thread works on the current ones
             uint32_t ra[32], rb[32];
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            auto max_of = [&](const uint32_t (&r)[32], int c0) {
+            auto max_of = [&](const uint32_t (&x)[32], int c0) {
                 if (full) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
+                    for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(x[i]));
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (ch * 128 + c0 + i < n_tok) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
+                        if (ch * 128 + c0 + i < n_tok) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(x[i]));
                 }
             };
             tmem_ld_32x32b_x32(lane_addr, ra);
@@ -215,20 +248,21 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             tmem_ld_wait_for(rb);
             max_of(rb, 96);
             s.xmax[ch][row] = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-            softmax_pair_sync();
+            softmax_pair_sync(q);
             const float mx = fmaxf(s.xmax[0][row], s.xmax[1][row]);      // finite: key 0 of the chunk always exists
             const float bias = -mx * scale_log2e;
-            if (it > 0) {
+            if (g > 0) {
                 // E and the weights of the previous half have been multiplied: they may be overwritten,
                 // and its column sums are waiting in its accumulator
-                ok = mbar_wait(&s.c_full[(it - 1) & 1], ((it - 1) >> 1) & 1) && !*(volatile int*)&s.abort_mma;
+                ok = mbar_wait(&s.c_full[(g - 1) & 1], ((g - 1) >> 1) & 1) && !*(volatile int*)&s.abort_mma;
                 if (!ok) break;
                 if (ch == 0) {
                     tc_fence_after_sync();
-                    take_column_sums(it - 1);
+                    take_column_sums(g - 1);
                     tc_fence_before_sync();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&s.drained[(it - 1) & 1]);
+                    if (lane == 0) mbar_arrive(&s.drained[(g - 1) & 1]);
+                    if (it == 0) write_result(prev);         // that was the last half of the previous item
                 }
             }
             float sum4[4] = {0.f, 0.f, 0.f, 0.f};
@@ -268,7 +302,7 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             tmem_ld_wait_for(rb);
             exp_of(rb, 96);
             s.xsum[ch][row] = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-            softmax_pair_sync();
+            softmax_pair_sync(q);
             if (ch == 0) {
                 // 1 / (row sum) as two fp16 terms in rows 0 and 1 of the weight operand (row 1 is swizzled by its index)
                 const float sum = s.xsum[0][row] + s.xsum[1][row];
@@ -285,15 +319,13 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             mbar_arrive(&s.p_ready);
         }
         if (!ok) s.abort = 1;
-        if (ch == 0) {                                       // the last half's column sums, then the chunk's result
-            const int last = n_iter - 1;
+        if (ch == 0 && n_halves > 0) {                       // the last half's column sums, then the last item's result
+            const int last = n_halves - 1;
             const bool okd = ok && mbar_wait(&s.c_full[last & 1], (last >> 1) & 1) && !*(volatile int*)&s.abort_mma;
             tc_fence_after_sync();
             if (okd) {
                 take_column_sums(last);
-                float* dst = out + (size_t)lh * p.total_tokens + tok_begin;
-                if (row < n_tok) dst[row] = col0;
-                if (kHalf + row < n_tok) dst[kHalf + row] = col1;
+                write_result(cur);
             }
         }
     }
@@ -331,8 +363,13 @@ cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_pe
     cudaError_t e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     float* dst = pool > 1 ? raw : out;
-    attention_kernel<<<dim3(p.total_chunks, p.layers * p.heads), kThreads, smem, stream>>>(
-        p, qmap, kmap, q_per_kv, scale * 1.4426950408889634f, dst);
+    const long long n_items = (long long)p.total_chunks * p.layers * p.heads;
+    if (n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
+    int dev = 0, n_sm = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+    const int grid = (int)(n_items < n_sm ? n_items : n_sm);          // one CTA per SM (shared memory)
+    attention_kernel<<<grid, kThreads, smem, stream>>>(p, qmap, kmap, q_per_kv, scale * 1.4426950408889634f,
+                                                       (int)n_items, dst);
     e = cudaGetLastError();
     if (e != cudaSuccess || pool <= 1) return e;
     pool_kernel<<<dim3((p.total_tokens + 255) / 256, p.layers * p.heads), 256, 0, stream>>>(p, raw, out, pool);

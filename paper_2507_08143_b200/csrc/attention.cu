@@ -55,6 +55,30 @@ __device__ __forceinline__ float ex2_approx(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Two fp32 values per instruction (the softmax warps are bound by instruction issue).
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 __device__ __forceinline__ void softmax_pair_sync(int q) {     // the two warps that share 32 query rows
     asm volatile("bar.sync %0, 64;" :: "r"(q + 1) : "memory");
 }
@@ -228,7 +252,8 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             auto max_of = [&](const uint32_t (&x)[32], int c0) {
                 if (full) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(x[i]));
+                    for (int i = 0; i < 32; i += 2)
+                        m4[(i >> 1) & 3] = max3(m4[(i >> 1) & 3], __uint_as_float(x[i]), __uint_as_float(x[i + 1]));
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
@@ -251,6 +276,38 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             softmax_pair_sync(q);
             const float mx = fmaxf(s.xmax[0][row], s.xmax[1][row]);      // finite: key 0 of the chunk always exists
             const float bias = -mx * scale_log2e;
+            uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};     // four pairs of partial row sums
+            const uint64_t scale2 = pack2(scale_log2e, scale_log2e), bias2 = pack2(bias, bias);
+            uint32_t packed[16];
+            auto exp_of = [&](const uint32_t (&r)[32], int c0) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    float y0, y1;
+                    unpack2(fma2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), scale2, bias2), y0, y1);
+                    float e0 = ex2_approx(y0), e1 = ex2_approx(y1);
+                    if (!full) {
+                        if (!row_valid || ch * 128 + c0 + i >= n_tok) e0 = 0.f;
+                        if (!row_valid || ch * 128 + c0 + i + 1 >= n_tok) e1 = 0.f;
+                    }
+                    sum2[(i >> 1) & 3] = add2(sum2[(i >> 1) & 3], pack2(e0, e1));
+                    const __half2 h = __floats2half2_rn(e0, e1);
+                    packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+            };
+            auto store = [&](int c0) {
+                const int col = ch * 128 + c0;
+                unsigned char* blk = s.p + (col >> 6) * kPBlock + row * 128;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int piece = ((col & 63) >> 3) + j;
+                    *reinterpret_cast<uint4*>(blk + ((piece ^ (row & 7)) << 4)) =
+                        make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
+                }
+            };
+            tmem_ld_32x32b_x32(lane_addr, ra);
+            tmem_ld_wait_for(ra);
+            tmem_ld_32x32b_x32(lane_addr + 32, rb);
+            exp_of(ra, 0);                                   // the first exponentials need no room in shared memory yet
             if (g > 0) {
                 // E and the weights of the previous half have been multiplied: they may be overwritten,
                 // and its column sums are waiting in its accumulator
@@ -265,43 +322,23 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                     if (it == 0) write_result(prev);         // that was the last half of the previous item
                 }
             }
-            float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-            auto exp_of = [&](const uint32_t (&r)[32], int c0) {
-                uint32_t packed[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    float e0 = ex2_approx(fmaf(__uint_as_float(r[i]), scale_log2e, bias));
-                    float e1 = ex2_approx(fmaf(__uint_as_float(r[i + 1]), scale_log2e, bias));
-                    if (!full) {
-                        if (!row_valid || ch * 128 + c0 + i >= n_tok) e0 = 0.f;
-                        if (!row_valid || ch * 128 + c0 + i + 1 >= n_tok) e1 = 0.f;
-                    }
-                    sum4[(i >> 1) & 3] += e0 + e1;
-                    const __half2 h = __floats2half2_rn(e0, e1);
-                    packed[i >> 1] = *reinterpret_cast<const uint32_t*>(&h);
-                }
-                const int col = ch * 128 + c0;
-                unsigned char* blk = s.p + (col >> 6) * kPBlock + row * 128;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int piece = ((col & 63) >> 3) + j;
-                    *reinterpret_cast<uint4*>(blk + ((piece ^ (row & 7)) << 4)) =
-                        make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
-                }
-            };
-            tmem_ld_32x32b_x32(lane_addr, ra);
-            tmem_ld_wait_for(ra);
-            tmem_ld_32x32b_x32(lane_addr + 32, rb);
-            exp_of(ra, 0);
+            store(0);
             tmem_ld_wait_for(rb);
             tmem_ld_32x32b_x32(lane_addr + 64, ra);
             exp_of(rb, 32);
+            store(32);
             tmem_ld_wait_for(ra);
             tmem_ld_32x32b_x32(lane_addr + 96, rb);
             exp_of(ra, 64);
+            store(64);
             tmem_ld_wait_for(rb);
             exp_of(rb, 96);
-            s.xsum[ch][row] = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+            store(96);
+            {
+                float lo, hi;
+                unpack2(add2(add2(sum2[0], sum2[1]), add2(sum2[2], sum2[3])), lo, hi);
+                s.xsum[ch][row] = lo + hi;
+            }
             softmax_pair_sync(q);
             if (ch == 0) {
                 // 1 / (row sum) as two fp16 terms in rows 0 and 1 of the weight operand (row 1 is swizzled by its index)

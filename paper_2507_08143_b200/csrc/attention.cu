@@ -4,15 +4,19 @@
 // the last, shorter chunk is a softmax over its own keys, pooling is a centred window with zero
 // padding.
 //
-// One CTA per (chunk, layer, KV head).  Warp 0 loads the chunk's keys once and streams the query
-// heads' rows in halves of 128 through a two-slot ring (TMA, 128-byte swizzle).  One thread of
-// warp 1 issues, per half, S = Q_half K^T (tcgen05.mma, 128 x 256 fp32 in tensor memory).  Warps
-// 2-9 share the 128 query rows (a pair of warps per 32 rows, 128 keys each): row maximum, e = exp(scale (s - max)) written as fp16 into shared
-// memory in the layout of an MN-major B operand, and the reciprocal of the row sum (two fp16 terms)
-// into rows 0 and 1 of a small K-major operand w.  A second MMA, E^T w (keys x 2: the half's normalised column sums),
-// lands in 32 columns of the half's own S accumulator once the softmax warps are done with S; four warps
-// add it to two registers per thread and write the chunk's result at the end.  S has two accumulators, so
-// that the products of the next half run beside the softmax of the current one.
+// Work item = one chunk of one layer and KV head; persistent CTAs (one per SM) walk the items.  Warp 0
+// loads an item's keys once and streams the query heads' rows in halves of 128 through a two-slot ring
+// (TMA, 128-byte swizzle).  One thread of warp 1 issues, per half, S = Q_half K^T (tcgen05.mma,
+// 128 x 256 fp32) into one of two accumulators in tensor memory, so that the products of the next half
+// run beside the softmax of the current one.  Warps 2-9 share the 128 query rows (a pair of warps per
+// 32 rows, 128 keys each): row maximum, e = 2^(scale log2e (s - max)) written as fp16 into shared memory
+// in the layout of an MN-major operand, and the reciprocal of the row sum (two fp16 terms) into rows 0
+// and 1 of a small K-major operand w.  A second MMA, E^T w (keys x 2: the half's normalised column
+// sums), lands in 32 columns of the half's own S accumulator once the softmax warps are done with S; each
+// warp adds the sums of its 128 keys to a register per thread and writes them at the end of the item.
+// The softmax warps are bound by instruction issue and latency (two warps per scheduler), not by the
+// exponential unit: hence packed fp32x2 arithmetic, three-input maxima, tensor-memory loads one
+// step ahead, and the first exponentials of a half computed before the wait for the E buffer.
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -113,7 +117,7 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         mbar_init(&s.k_full, 1);
         mbar_init(&s.k_empty, 1);
         for (int i = 0; i < 2; ++i) { mbar_init(&s.q_full[i], 1); mbar_init(&s.q_empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&s.s_full[i], 1); mbar_init(&s.c_full[i], 1); mbar_init(&s.drained[i], 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&s.s_full[i], 1); mbar_init(&s.c_full[i], 1); mbar_init(&s.drained[i], 8); }
         mbar_init(&s.p_ready, 32 * kSoftmaxWarps);
         s.abort = 0;
         s.abort_mma = 0;
@@ -217,20 +221,17 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         const int ch = (warp - 2) >> 2;                      // which 128 of the 256 keys
         const int row = q * 32 + lane;                       // query row within the half = TMEM lane
         const uint32_t quad_addr = tmem + ((uint32_t)(q * 32) << 16);
-        float col0 = 0.f, col1 = 0.f;                        // ch == 0: column sums of keys `row` and 128 + `row`
-        auto take_column_sums = [&](int g) {                 // TMEM lane = key within its half of the chunk
-            uint32_t c[2], d[2];
-            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(g & 1) * 256, c);
-            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(g & 1) * 256 + 16, d);
+        float col = 0.f;                                     // column sum of key ch * 128 + `row` (TMEM lane = key here)
+        auto take_column_sums = [&](int g) {                 // each warp takes the key half that it also exponentiates
+            uint32_t c[2];
+            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(g & 1) * 256 + ch * 16, c);
             tmem_ld_wait();
-            col0 += __uint_as_float(c[0]) + __uint_as_float(c[1]);       // hi and lo weights
-            col1 += __uint_as_float(d[0]) + __uint_as_float(d[1]);
+            col += __uint_as_float(c[0]) + __uint_as_float(c[1]);        // hi and lo weights
         };
         auto write_result = [&](const AttnItem& a) {         // an item's column sums are complete
             float* dst = out + (size_t)a.lh * p.total_tokens + a.tok_begin;
-            if (row < a.n_tok) dst[row] = col0;
-            if (kHalf + row < a.n_tok) dst[kHalf + row] = col1;
-            col0 = 0.f; col1 = 0.f;
+            if (ch * kHalf + row < a.n_tok) dst[ch * kHalf + row] = col;
+            col = 0.f;
         };
         const int n_halves = my_items * n_iter;
         AttnItem cur = attn_item(p, blockIdx.x), prev = cur;
@@ -313,14 +314,12 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                 // and its column sums are waiting in its accumulator
                 ok = mbar_wait(&s.c_full[(g - 1) & 1], ((g - 1) >> 1) & 1) && !*(volatile int*)&s.abort_mma;
                 if (!ok) break;
-                if (ch == 0) {
-                    tc_fence_after_sync();
-                    take_column_sums(g - 1);
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&s.drained[(g - 1) & 1]);
-                    if (it == 0) write_result(prev);         // that was the last half of the previous item
-                }
+                tc_fence_after_sync();
+                take_column_sums(g - 1);
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s.drained[(g - 1) & 1]);
+                if (it == 0) write_result(prev);             // that was the last half of the previous item
             }
             store(0);
             tmem_ld_wait_for(rb);
@@ -356,7 +355,7 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             mbar_arrive(&s.p_ready);
         }
         if (!ok) s.abort = 1;
-        if (ch == 0 && n_halves > 0) {                       // the last half's column sums, then the last item's result
+        if (n_halves > 0) {                       // the last half's column sums, then the last item's result
             const int last = n_halves - 1;
             const bool okd = ok && mbar_wait(&s.c_full[last & 1], (last >> 1) & 1) && !*(volatile int*)&s.abort_mma;
             tc_fence_after_sync();

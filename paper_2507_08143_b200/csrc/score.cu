@@ -25,13 +25,18 @@ constexpr int kThreads = 192;
 // leaves no shared memory for that.
 template <int MP> struct OutTiles { static constexpr int value = MP <= 48 ? 8 : 1; };
 constexpr int kBufs = 4;                  // accumulators in rotation
-template <int MP> struct BufCols { static constexpr uint32_t value = MP <= 64 ? 64 : 128; };   // tensor-memory columns each
+// Up to 64 sketch columns the two bf16 terms of W are one operand of 2 MP rows (hi on top of lo): one MMA per
+// k-step reads the key tile once and leaves k W_hi in columns [0, MP) and k W_lo in [MP, 2 MP) of the accumulator.
+template <int MP> struct Fused { static constexpr bool value = MP <= 64; };
+template <int MP> struct BufCols {                        // tensor-memory columns per accumulator (a power of two)
+    static constexpr uint32_t value = MP <= 16 ? 32 : (MP <= 32 ? 64 : 128);
+};
 
 template <int MP>
 struct __align__(1024) ScoreSmem {
     static constexpr int kStages = Stages<MP>::value;
     unsigned char tiles[kStages][kTileBytes];
-    unsigned char w[2][2][MP * 128];      // [term][channel half][MP rows x 64 channels]
+    unsigned char w[2][2][MP * 128];      // fused: [channel half][term][MP rows x 64 channels]; else [term][channel half][...]
     uint64_t full[kStages];
     uint64_t empty[kStages];
     uint64_t w_full;
@@ -87,7 +92,8 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
             for (int term = 0; term < 2; ++term)
 #pragma unroll
                 for (int half = 0; half < 2; ++half)
-                    tma_load_2d(s.w[term][half], &wmap, &s.w_full, half * 64, (unit * 2 + term) * MP);
+                    tma_load_2d(Fused<MP>::value ? s.w[half][term] : s.w[term][half], &wmap, &s.w_full, half * 64,
+                                (unit * 2 + term) * MP);
             for (int t = 0; t < n_tiles; ++t) {
                 const int stage = t % kStages, round = t / kStages;
                 if (round > 0 && !mbar_wait(&s.empty[stage], (round - 1) & 1)) { s.abort = 1; break; }
@@ -99,7 +105,7 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
             }
         }
     } else if (warp == 1) {
-        constexpr uint32_t idesc = umma_idesc_bf16(128, MP, 0, 0);
+        constexpr uint32_t idesc = umma_idesc_bf16(128, Fused<MP>::value ? 2 * MP : MP, 0, 0);
         bool ok = mbar_wait(&s.w_full, 0);
         for (int t = 0; t < n_tiles && ok; ++t) {
             const int stage = t % kStages, round = t / kStages;
@@ -112,15 +118,25 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
             if (lane == 0) {
                 const uint32_t a_base = smem_u32(s.tiles[stage]);
                 const uint32_t d_addr = tmem + buf * kCols;
-#pragma unroll
-                for (int term = 0; term < 2; ++term)
+                if constexpr (Fused<MP>::value) {
 #pragma unroll
                     for (int ks = 0; ks < 8; ++ks) {
                         const int half = ks >> 2, off = (ks & 3) * 32;
                         const uint64_t a_desc = umma_desc_sw128(a_base + half * kBoxBytes + off, 16, 1024);
-                        const uint64_t b_desc = umma_desc_sw128(smem_u32(s.w[term][half]) + off, 16, 1024);
-                        umma_bf16(d_addr, a_desc, b_desc, idesc, (term > 0) || (ks > 0));
+                        const uint64_t b_desc = umma_desc_sw128(smem_u32(s.w[half][0]) + off, 16, 1024);
+                        umma_bf16(d_addr, a_desc, b_desc, idesc, ks > 0);
                     }
+                } else {
+#pragma unroll
+                    for (int term = 0; term < 2; ++term)
+#pragma unroll
+                        for (int ks = 0; ks < 8; ++ks) {
+                            const int half = ks >> 2, off = (ks & 3) * 32;
+                            const uint64_t a_desc = umma_desc_sw128(a_base + half * kBoxBytes + off, 16, 1024);
+                            const uint64_t b_desc = umma_desc_sw128(smem_u32(s.w[term][half]) + off, 16, 1024);
+                            umma_bf16(d_addr, a_desc, b_desc, idesc, (term > 0) || (ks > 0));
+                        }
+                }
                 umma_commit(&s.empty[stage]);
                 umma_commit(&s.d_full[buf]);
             }
@@ -145,15 +161,41 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
             const bool ok = mbar_wait(&s.d_full[buf], use & 1) && !*(volatile int*)&s.abort_mma;
             if (!ok) { s.abort = 1; break; }
             tc_fence_after_sync();
-            float acc = 0.f;
+            // all loads of a group are issued before the one wait: their latencies overlap
+            const uint32_t d_row = tmem + ((uint32_t)(q * 32) << 16) + buf * kCols;
+            float acc4[4] = {0.f, 0.f, 0.f, 0.f};
+            if constexpr (Fused<MP>::value) {
+                uint32_t hi[MP / 16][16], lo[MP / 16][16];
 #pragma unroll
-            for (int c0 = 0; c0 < MP; c0 += 16) {
-                uint32_t r[16];
-                tmem_ld_32x32b_x16(tmem + ((uint32_t)(q * 32) << 16) + buf * kCols + c0, r);
+                for (int c = 0; c < MP / 16; ++c) {
+                    tmem_ld_32x32b_x16(d_row + c * 16, hi[c]);
+                    tmem_ld_32x32b_x16(d_row + MP + c * 16, lo[c]);
+                }
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 16; ++i) { float v = __uint_as_float(r[i]); acc = fmaf(v, v, acc); }
+                for (int c = 0; c < MP / 16; ++c)
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float v = __uint_as_float(hi[c][i]) + __uint_as_float(lo[c][i]);
+                        acc4[i & 3] = fmaf(v, v, acc4[i & 3]);
+                    }
+            } else {
+#pragma unroll
+                for (int g0 = 0; g0 < MP; g0 += 64) {
+                    uint32_t r[4][16];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) tmem_ld_32x32b_x16(d_row + g0 + c * 16, r[c]);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const float v = __uint_as_float(r[c][i]);
+                            acc4[i & 3] = fmaf(v, v, acc4[i & 3]);
+                        }
+                }
             }
+            const float acc = (acc4[0] + acc4[1]) + (acc4[2] + acc4[3]);
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&s.d_empty[buf]);

@@ -14,7 +14,7 @@
  *     void*; NULL is the default stream) and the call returns without synchronising.
  *   - Keys/values are bf16 with the d channels of a token contiguous; the other three strides
  *     (layer, KV head, token) are given in ELEMENTS and must be multiples of 8 (16 bytes); base
- *     pointers must be 16-byte aligned.  d must be 128.  1 <= m <= 64.
+ *     pointers must be 16-byte aligned.  d must be 128.  1 <= m <= 128.
  *   - Sequences are packed back to back along the token axis: sequence b owns tokens
  *     [cu_seqlens[b], cu_seqlens[b+1]) of every (layer, head).  A "unit" is one
  *     (layer, head, sequence) triple; unit id = (layer * heads + head) * batch + b.

@@ -237,7 +237,7 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
         const uint32_t key = order_key(sc[i]);
         head_gt += key > thr; head_eq += key == thr;
     }
-    int cnt = 0;                                        // packed: above | at << 16
+    int cnt_gt = 0, cnt_eq = 0;                         // full-width counters: a stretch may hold more than 2^16 scores
     for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
         float4 q[kAhead];
 #pragma unroll
@@ -249,26 +249,29 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
         for (int u = 0; u < kAhead; ++u) {
             int g, e;
             flags(q[u], g, e);
-            if (v0 + u * 32 + lane < vend) cnt += __popc(g) | (__popc(e) << 16);
+            if (v0 + u * 32 + lane < vend) { cnt_gt += __popc(g); cnt_eq += __popc(e); }
         }
     }
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, d);
+    for (int d = 16; d > 0; d >>= 1) {
+        cnt_gt += __shfl_xor_sync(0xffffffffu, cnt_gt, d);
+        cnt_eq += __shfl_xor_sync(0xffffffffu, cnt_eq, d);
+    }
     __syncthreads();                                    // earlier users of the shared arrays are done
-    if (lane == 0) s.cnt[0][0][warp] = cnt;
+    if (lane == 0) { s.cnt[0][0][warp] = cnt_gt; s.cnt[1][0][warp] = cnt_eq; }
     __syncthreads();
     int base_gt, base_eq;
     {
-        const int c = s.cnt[0][0][lane];                // kWarps == 32: one packed count per lane
-        int incl = c;
+        const int c_gt = s.cnt[0][0][lane], c_eq = s.cnt[1][0][lane];       // kWarps == 32: one pair of counts per lane
+        int incl_gt = c_gt, incl_eq = c_eq;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
-            const int t = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += t;
+            const int t_gt = __shfl_up_sync(0xffffffffu, incl_gt, off);
+            const int t_eq = __shfl_up_sync(0xffffffffu, incl_eq, off);
+            if (lane >= off) { incl_gt += t_gt; incl_eq += t_eq; }
         }
-        const int excl = __shfl_sync(0xffffffffu, incl - c, warp);          // exclusive prefix of this warp
-        base_gt = head_gt + (excl & 0xffff);
-        base_eq = head_eq + (excl >> 16);
+        base_gt = head_gt + __shfl_sync(0xffffffffu, incl_gt - c_gt, warp);  // exclusive prefixes of this warp
+        base_eq = head_eq + __shfl_sync(0xffffffffu, incl_eq - c_eq, warp);
     }
 
     // ---- emission: head, stretches, tail ----------------------------------------------------------

@@ -98,3 +98,14 @@ def test_across_heads_pipeline_on_leverage_scores(B):
     counts = np.diff(offs_np, axis=2)
     assert counts.min() >= 0 and np.all(counts.sum(axis=2) == w.heads * np.array(keep)[None, :])
     print("tokens kept per head (layer 0, sequence 0):", counts[0, 0].tolist())
+
+
+def test_across_heads_long_sequence_large_budget(B):
+    # more than 2^16 kept indices in a head, stretches of more than 2^16 scores per warp
+    rng = np.random.default_rng(5)
+    n, kk = 600000, 250000
+    shape = B.Shape(1, 3, 128, 48, [n])
+    s = rng.standard_normal((1, 3, n)).astype(np.float32)
+    s[0, 0] += 1.0                                         # the first head takes most of the budget
+    s[0, 2] = np.round(s[0, 2], 1)
+    _select_and_check(B, shape, torch.from_numpy(s).cuda(), [kk])

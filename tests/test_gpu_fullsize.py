@@ -38,7 +38,7 @@ def _properties_all_units(w, shape, keep, scores, idx, k_out, v_out, kr, v):
 
 
 def _full(B, name, sample_units):
-    w = inputs.workload(name)
+    w = name if isinstance(name, inputs.Workload) else inputs.workload(name)
     need = 2 * w.layers * w.heads * w.total_tokens * w.d * 2 * 1.45 + (4 << 30)
     free, _ = torch.cuda.mem_get_info()
     if free < need:
@@ -79,3 +79,10 @@ def test_c4_full_ragged(B):
 
 def test_c3_full(B):
     _full(B, "c3", [(0, 0, 0), (63, 7, 0)])
+
+
+def test_one_million_token_sequence_beside_a_short_one(B):
+    # the longest context of the paper's Fig. 1 (2^20 tokens) packed with a 300-token sequence:
+    # 32 Gram blocks of 32768 tokens per unit, fp64 across them
+    w = inputs.Workload("1m", 1, 2, 128, [1 << 20, 300], [0.1, 0.5], p=0.7, seed=77)
+    _full(B, w, [(0, 0, 0), (0, 1, 1)])

@@ -140,6 +140,23 @@ def test_select_exact_with_ties_and_edges(B):
                 np.testing.assert_array_equal(got, orc.top_k_indices(seg, keep[b]), err_msg=f"{l},{h},{b}")
 
 
+@pytest.mark.parametrize("n,keep", [(131072, 120000), (200001, 70000), (1 << 20, 900000), (1 << 21, 3), (3000000, 2999999)])
+def test_select_long_sequences_and_large_keep_counts(B, n, keep):
+    # more than 2^16 kept indices per unit, and stretches of more than 2^16 scores per warp
+    rng = np.random.default_rng(n % 1000)
+    s = rng.standard_normal((1, 2, n)).astype(np.float32)
+    s[0, 1] = np.round(s[0, 1], 2)                       # heavy ties
+    shape = B.Shape(1, 2, 128, 48, [n])
+    sc = torch.from_numpy(s).cuda()
+    idx = torch.full((1, 2, keep), -1, dtype=torch.int32, device="cuda")
+    ws = B.alloc_workspace(shape)
+    B.select(shape, sc, [keep], idx, ws)
+    torch.cuda.synchronize()
+    idx = idx.cpu().numpy()
+    for h in range(2):
+        np.testing.assert_array_equal(idx[0, h], orc.top_k_indices(s[0, h].astype(np.float64), keep), err_msg=f"head {h}")
+
+
 def test_compact_bit_exact_and_skips_bad_indices(B):
     w = inputs.Workload("compact", 2, 2, 128, [700, 300], [0.5, 0.5], seed=51)
     _, kr, v = inputs.make_tensors(w, device="cpu", want_pre=False)

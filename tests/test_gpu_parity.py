@@ -55,6 +55,24 @@ def test_ragged_small_sequences(B):
     print(f"ragged-small: err {worst:.2e}")
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_random_ragged_batches(B, seed):
+    # random batches: lengths from 0 to a few Gram blocks, around tile and chunk borders, any retention ratio
+    rng = np.random.default_rng(1000 + seed)
+    special = [0, 1, 2, 47, 48, 49, 127, 128, 129, 255, 256, 257, 511, 513, 1023, 1025, 2047, 2049, 4097]
+    batch = int(rng.integers(1, 7))
+    seqlens = [int(rng.choice(special)) if rng.random() < 0.6 else int(rng.integers(1, 40000)) for _ in range(batch)]
+    if sum(seqlens) == 0:
+        seqlens[0] = 300
+    ratios = [float(rng.choice([0.01, 0.1, 0.32, 0.5, 0.9, 1.0])) for _ in range(batch)]
+    m = int(rng.choice([5, 16, 48, 48, 48, 64]))
+    w = inputs.Workload(f"random-{seed}", int(rng.integers(1, 3)), int(rng.integers(1, 4)), 128, seqlens, ratios,
+                        p=float(rng.choice([0.5, 0.7, 1.0])), seed=500 + seed, m=m)
+    mode = "paper" if seed % 2 == 0 else "aliased"
+    worst, band, outs = _run_workload(B, w, mode=mode, device="cpu")
+    print(f"{w.name}: lens {seqlens} ratios {ratios} m {m} {mode}: err {worst:.2e}, band {band}")
+
+
 @pytest.mark.parametrize("m", [8, 16, 20, 32, 64])
 def test_other_sketch_dimensions(B, m):
     w = inputs.Workload(f"m{m}", 1, 2, 128, [700, 1300], [0.25, 0.4], p=0.7, seed=20 + m, m=m)
@@ -86,6 +104,24 @@ def test_token_major_layout(B):
     keep = _keep(B, w)
     outs = H.run_compress(B, shape, kp, kr, v, phi, keep)
     H.compare_all_units(shape, keep, outs, kp, kr, v, phi, what="token-major")
+
+
+def test_padded_rows_and_interleaved_kv_layout(B):
+    # keys and values of a token side by side in one buffer (a fused K|V projection output), rows
+    # padded to 264 elements: token stride 264, K at offset 0, V at offset 128
+    w = inputs.Workload("padded", 2, 2, 128, [1300, 257, 64], [0.3, 0.5, 0.25], p=0.7, seed=33)
+    kp, kr, v = inputs.make_tensors(w, device="cpu")
+    T = sum(w.seqlens)
+    buf = torch.zeros(w.layers, w.heads, T, 264, dtype=torch.bfloat16, device="cuda")
+    buf[..., :128] = kr.cuda()
+    buf[..., 128:256] = v.cuda()
+    k_view, v_view = buf[..., :128], buf[..., 128:256]
+    assert k_view.stride(2) == 264 and v_view.data_ptr() - k_view.data_ptr() == 256
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    phi = inputs.make_sketch_matrix(w.d, w.m, 6)
+    keep = _keep(B, w)
+    outs = H.run_compress(B, shape, k_view, k_view, v_view, phi, keep)
+    H.compare_all_units(shape, keep, outs, k_view, k_view, v_view, phi, what="padded")
 
 
 def test_staged_calls_match_fused(B):

@@ -114,3 +114,14 @@ def test_attention_llama_shape_long(B):
     shape, q, k, out = _attention(B, w, G, 7, scale, q=q, k=k)
     worst = _check(w, shape, q, k, out, G, 7, scale, units=[(0, 0, 0), (0, 7, 0)])
     print(f"attention llama shape n=8192: worst relative error {worst:.2e}")
+
+
+def test_attention_many_items_per_cta(B):
+    # 864 work items on 148 persistent CTAs: every CTA walks full and ragged chunks of several heads in turn
+    w = inputs.Workload("attn-many", 3, 4, 128, [5000, 257, 33, 12345], [0.5] * 4, p=0.7, seed=83)
+    scale = 1.0 / math.sqrt(128)
+    shape, q, k, out = _attention(B, w, 2, 1, scale)
+    assert not torch.isnan(out).any()
+    worst = _check(w, shape, q, k, out, 2, 1, scale,
+                   units=[(l, h, b) for l in (0, 2) for h in (0, 3) for b in range(4)])
+    print(f"attention, many items per CTA: worst rel err {worst:.2e}")

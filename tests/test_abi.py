@@ -121,3 +121,29 @@ def test_argument_errors_are_reported_before_any_launch():
                                 ctypes.c_void_p(1 << 23), 1 << 20, None)
     assert rc == -1
     assert "workspace" in B.error_string(-3) and B.error_string(0) == "ok"
+
+
+def test_variant_and_nll_argument_errors_are_reported_before_any_launch():
+    ok = B.Shape(1, 2, 128, 48, [1024])
+    wide = B.Shape(1, 2, 128, 128, [1024])
+    dev = lambda a: ctypes.c_void_p(a)
+
+    def variant(shape, fact, floor):
+        return B.LIB.compactor_score_variant(ctypes.byref(shape.c), _mat(), dev(1 << 21), fact, floor, None, 0.3,
+                                             dev(1 << 22), None, dev(1 << 23), 1 << 30, None)
+    assert variant(ok, 7, 1e-6) == -1                                    # unknown factorisation
+    assert variant(ok, B.FACTOR_EIG, 0.0) == -1 and variant(ok, B.FACTOR_EIG, float("nan")) == -1
+    assert variant(wide, B.FACTOR_EIG, 1e-6) == -2                       # the eigen route stops at 64 columns
+    assert B.workspace_bytes(wide) > B.workspace_bytes(ok)
+
+    cu = (ctypes.c_int32 * 2)(0, 4)
+
+    def nll(**kw):
+        return B.LIB.compactor_nll(dev(kw.get("x", 1 << 20)), kw.get("dt", 0), kw.get("rows", 4), kw.get("vocab", 32),
+                                   kw.get("stride", 32), dev(1 << 21), 1, kw.get("cu", cu), dev(1 << 22),
+                                   dev(kw.get("out", 1 << 23)), None)
+    assert nll(dt=5) == -1 and nll(vocab=0) == -1 and nll(rows=-1) == -1
+    assert nll(stride=16) == -1                                          # rows overlap
+    assert nll(stride=36) == -1                                          # 72 bytes: not a multiple of 16
+    assert nll(x=(1 << 20) + 2) == -1 and nll(x=0) == -1 and nll(out=0) == -1
+    assert nll(cu=(ctypes.c_int32 * 2)(0, 5)) == -1 and nll(cu=(ctypes.c_int32 * 2)(2, 4)) == -1

@@ -151,7 +151,7 @@ int compactor_nll(const void* logits, int32_t logits_dtype, int64_t rows, int32_
 /*
  * Bytes of device workspace that compactor_score and compactor_compress need for this shape.
  * compactor_select and compactor_compact only use a small table at its start and accept any
- * workspace of at least 12*(batch+1) bytes rounded up to 256.  The workspace must be 256-byte
+ * workspace of at least 16*(batch+1) bytes rounded up to 256.  The workspace must be 256-byte
  * aligned; its contents need not be preserved between calls.  Returns 0 for an invalid shape.
  */
 size_t compactor_workspace_bytes(const compactor_shape* shape);
@@ -257,7 +257,7 @@ int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_sc
  *   attn_out device fp32 [layers][heads][total_tokens].
  * The last, shorter chunk of a sequence is a softmax over its own keys.  Exponentials are
  * rounded to fp16 before they are summed over the query rows on the tensor cores (fp32
- * accumulation).  Workspace: compactor_workspace_bytes() suffices (12*(batch+1) bytes rounded up
+ * accumulation).  Workspace: compactor_workspace_bytes() suffices (16*(batch+1) bytes rounded up
  * to 256, plus 4 bytes per output element when pool > 1).
  */
 int compactor_attention_scores(const compactor_shape* shape, compactor_mat q, compactor_mat k,
@@ -294,8 +294,8 @@ int compactor_compact_across_heads(const compactor_shape* shape, compactor_mat k
  * no workspace argument: the scratch is a fixed array of compactor_builtin_scratch_bytes()
  * (32 MiB) inside the library, resident on every device the process uses from the first use of
  * the library on that device until the process exits.  The call allocates and frees nothing.
- *   - Size limit: the scratch must hold 12*(batch+1) bytes of tables, about 160 KiB per unit
- *     (at m = 48) and 128 KiB per Gram block (blocks are lengthened up to 32768 tokens to make it
+ *   - Size limit: the scratch must hold 16*(batch+1) bytes of tables, about 160 KiB per unit
+ *     (at m = 48) and 128 KiB per Gram block (blocks are lengthened up to 65536 tokens to make it
  *     fit, i.e. down to 4 bytes per token per (layer, head)).  A larger problem is refused with
  *     COMPACTOR_E_TOO_LARGE before anything is enqueued; split it by layers or use
  *     compactor_score.

@@ -20,7 +20,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
 struct HostPlan {
     Plan plan;
-    std::vector<int> tables;       // cu_seqlens | cu_keep | cu_chunks, each batch+1
+    std::vector<int> tables;       // cu_seqlens | cu_keep | cu_chunks | cu_schunks, each batch+1
     size_t off_tables, off_w, off_gpart, off_partials, off_scores, total_bytes;
     int units;
 };
@@ -73,16 +73,32 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     long long tc = count_chunks(chunk);
     if (tc > 0x7fffffffLL) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
     p.total_chunks = (int)tc;
+    // The scoring sweep writes no partial sums and sets up faster; its blocks are chosen for balance: the
+    // hardware hands out CTAs as SMs free up, so the sweep ends about half a block after the average SM.
+    int schunk = kMaxChunk;
+    best = 1e300;
+    for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
+        const double ctas = (double)count_chunks(c) * s->layers * s->heads;
+        const double per_cta_us = 2.0 + c * 256.0 / 44e3;
+        const double cost = (ctas / kSmCount < 1.0 ? 1.0 : ctas / kSmCount) * per_cta_us + 0.5 * per_cta_us;
+        if (cost < best * 0.999) { best = cost; schunk = c; }
+    }
+    p.schunk = schunk;
+    tc = count_chunks(schunk);
+    if (tc > 0x7fffffffLL) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    p.total_schunks = (int)tc;
 
     const int nb1 = s->batch + 1;
-    hp->tables.assign((size_t)3 * nb1, 0);
+    hp->tables.assign((size_t)4 * nb1, 0);
     int* cs = hp->tables.data();
     int* cc = cs + 2 * nb1;
+    int* csc = cs + 3 * nb1;
     for (int b = 0; b <= s->batch; ++b) cs[b] = s->cu_seqlens[b];
     for (int b = 0; b < s->batch; ++b) cc[b + 1] = cc[b] + (cs[b + 1] - cs[b] + chunk - 1) / chunk;
+    for (int b = 0; b < s->batch; ++b) csc[b + 1] = csc[b] + (cs[b + 1] - cs[b] + schunk - 1) / schunk;
 
     size_t off = 0;
-    hp->off_tables = off;   off += align_up(sizeof(int) * 3 * nb1);
+    hp->off_tables = off;   off += align_up(sizeof(int) * 4 * nb1);
     hp->off_w = off;        off += align_up(sizeof(__nv_bfloat16) * w_elems_per_unit(p.mp) * hp->units);
     hp->off_gpart = off;    off += align_up(sizeof(double) * kFactorSlices * p.mp * p.mp * hp->units);
     hp->off_partials = off; off += align_up(sizeof(double) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
@@ -125,10 +141,11 @@ cudaError_t upload_tables(HostPlan* hp, void* ws, cudaStream_t stream) {
     const int nb1 = hp->plan.batch + 1;
     int* dev = reinterpret_cast<int*>(static_cast<char*>(ws) + hp->off_tables);
     // The source is pageable host memory: the runtime stages it before this call returns.
-    cudaError_t e = cudaMemcpyAsync(dev, hp->tables.data(), sizeof(int) * 3 * nb1, cudaMemcpyHostToDevice, stream);
+    cudaError_t e = cudaMemcpyAsync(dev, hp->tables.data(), sizeof(int) * 4 * nb1, cudaMemcpyHostToDevice, stream);
     hp->plan.cu_seqlens = dev;
     hp->plan.cu_keep = dev + nb1;
     hp->plan.cu_chunks = dev + 2 * nb1;
+    hp->plan.cu_schunks = dev + 3 * nb1;
     return e;
 }
 

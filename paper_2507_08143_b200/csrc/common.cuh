@@ -10,13 +10,13 @@ namespace compactor {
 
 constexpr int kD = 128;            // head dimension the kernels are written for
 constexpr int kMaxM = 128;          // largest sketch dimension
-constexpr int kMaxChunk = 32768;   // most tokens per block (one CTA of the two streaming kernels)
+constexpr int kMaxChunk = 65536;   // most tokens per block (one CTA of a streaming kernel)
 constexpr int kMinChunk = 256;
 constexpr int kGramFlushTokens = 512;    // most tokens whose Gram matrix is summed in fp32 (tensor-core accumulators) before going to fp64
 constexpr int kGramElems = kD * kD;
 constexpr int kFactorSlices = 8;   // CTAs per unit that share the fp64 projection of the Gram matrix
 
-// Device-side view of one call: shapes plus the three prefix-sum tables that live at the start
+// Device-side view of one call: shapes plus the four prefix-sum tables that live at the start
 // of the workspace.  Passed to kernels by value.
 struct Plan {
     int layers, heads, batch;
@@ -29,6 +29,9 @@ struct Plan {
     const int* cu_seqlens; // device [batch+1]
     const int* cu_keep;    // device [batch+1]
     const int* cu_chunks;  // device [batch+1]
+    int schunk;            // tokens per block of the scoring sweep (no partial sums there: shorter blocks balance better)
+    int total_schunks;     // its blocks per (layer, head): sum_b ceil(n_b / schunk)
+    const int* cu_schunks; // device [batch+1]
 };
 
 struct Mat {               // compactor_mat with a typed pointer

@@ -61,9 +61,9 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
     const int chunk_id = blockIdx.x;
     const int lh = blockIdx.y;
     const int layer = lh / p.heads, head = lh % p.heads;
-    const int b = find_segment(p.cu_chunks, p.batch, chunk_id);
-    const int tok_begin = p.cu_seqlens[b] + (chunk_id - p.cu_chunks[b]) * p.chunk;
-    const int tok_end = min(tok_begin + p.chunk, p.cu_seqlens[b + 1]);
+    const int b = find_segment(p.cu_schunks, p.batch, chunk_id);
+    const int tok_begin = p.cu_seqlens[b] + (chunk_id - p.cu_schunks[b]) * p.schunk;
+    const int tok_end = min(tok_begin + p.schunk, p.cu_seqlens[b + 1]);
     const int n_tok = tok_end - tok_begin;
     const int n_tiles = (n_tok + kTile - 1) / kTile;
     const int unit = lh * p.batch + b;
@@ -221,7 +221,7 @@ cudaError_t launch_score_mp(const Plan& p, const CUtensorMap& kmap, const CUtens
     const int smem = (int)sizeof(ScoreSmem<MP>) + 1024;
     cudaError_t e = cudaFuncSetAttribute(score_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    dim3 grid(p.total_chunks, p.layers * p.heads);
+    dim3 grid(p.total_schunks, p.layers * p.heads);
     score_kernel<MP><<<grid, kThreads, smem, stream>>>(p, kmap, wmap, scores, status);
     return cudaGetLastError();
 }
@@ -230,7 +230,7 @@ cudaError_t launch_score_mp(const Plan& p, const CUtensorMap& kmap, const CUtens
 
 cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
                          cudaStream_t stream) {
-    if (p.total_chunks == 0) return cudaSuccess;
+    if (p.total_schunks == 0) return cudaSuccess;
     CUtensorMap kmap, wmap;
     const long long units = (long long)p.layers * p.heads * p.batch;
     if (!make_kv_tensor_map(&kmap, k.ptr, p.layers, p.heads, p.total_tokens, k.stride_layer, k.stride_head,

@@ -47,7 +47,7 @@ def test_builtin_scratch_matches_workspace_entry_point_twice():
 
 def test_builtin_scratch_rejects_oversized_problem():
     from paper_2507_08143_b200 import binding as B
-    shape = B.Shape(8, 8, 128, 48, [131072])            # needs about 128 MiB of Gram blocks
+    shape = B.Shape(64, 8, 128, 48, [131072])           # needs 128 MiB of Gram blocks even at the longest block length
     k = torch.empty(8, dtype=torch.bfloat16, device="cuda")
     fake = B.CompactorMat(k.data_ptr(), 128, 128, 128)   # never dereferenced: the size check comes first
     out = torch.empty(8, dtype=torch.float32, device="cuda")

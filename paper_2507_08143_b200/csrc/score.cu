@@ -1,12 +1,14 @@
 // Scoring pass (Algorithm 1, lines 5-6, fused): o_i = || k_i W ||^2 with W = Phi L^-T from the
 // factor kernel, so that U~ = K^ V~ Sigma~^-1 is never stored.  W arrives as two bf16 terms
-// (hi + lo); both are multiplied with the bf16 keys on the tensor cores and summed in fp32.
+// (hi + lo); both are multiplied with the bf16 keys on the tensor cores and added in fp32.
 //
 // One CTA per block of tokens of one unit, one CTA per SM.  Warp 0 streams 128-token tiles of K
 // (and W once) through a six-stage ring with TMA; one thread of warp 1 issues tcgen05.mma (A = key
-// tile, K-major; B = W^T, K-major; D = 128 tokens x MP fp32 in tensor memory, four accumulators
-// in rotation); warps 2-5 read D back, square, sum along the row and store one fp32 score per
-// token.
+// tile, K-major; B = the rows of W_hi on top of the rows of W_lo, K-major: one MMA per k-step, so
+// the key tile is fetched from shared memory once; D = 128 tokens x 2 MP fp32 in tensor memory,
+// four accumulators in rotation); warps 2-5 read D back, add the two halves, square, sum along the
+// row and park the scores of eight tiles in shared memory, from where they leave in 4 KB bursts.
+// Sketches wider than 64 columns keep the two terms as separate MMAs into one accumulator.
 #include "common.cuh"
 #include "sm100.cuh"
 

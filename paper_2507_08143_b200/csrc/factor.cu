@@ -369,6 +369,21 @@ eig_kernel(Plan p, const double* __restrict__ g_partials, const float* __restric
     __syncthreads();
     const bool bad = (s.flags & COMPACTOR_STATUS_NONFINITE) != 0;
 
+    // G is scaled by a power of two (exactly) so that its largest diagonal entry lies in [1/2, 1): the rotation
+    // angles can then be worked out in fp32 without overflow; the eigenvalues are scaled back at the end.
+    int scale_exp = 0;
+    if (!bad) {
+        double dmax = 0.0;
+        for (int i = 0; i < m; ++i) dmax = fmax(dmax, fabs(s.a[i * LD + i]));      // the same in every thread
+        if (dmax > 0.0) (void)frexp(dmax, &scale_exp);
+        __syncthreads();
+        for (int e = tid; e < MP * MP; e += kEigThreads) {
+            const int i = e / MP, j = e % MP;
+            s.a[i * LD + j] = ldexp(s.a[i * LD + j], -scale_exp);
+        }
+        __syncthreads();
+    }
+
     for (int sweep = 0; sweep < kEigMaxSweeps && !bad; ++sweep) {
         // off-diagonal mass against the whole: the same value in every thread, so all leave together
         double off = 0.0, all = 0.0;
@@ -400,35 +415,49 @@ eig_kernel(Plan p, const double* __restrict__ g_partials, const float* __restric
                 const int pp = min(a0, a1), qq = max(a0, a1);
                 const double apq = s.a[pp * LD + qq], app = s.a[pp * LD + pp], aqq = s.a[qq * LD + qq];
                 double c = 1.0, sn = 0.0;
-                if (fabs(apq) > 1e-300 && fabs(apq) > 1e-19 * sqrt(fabs(app) * fabs(aqq))) {
-                    const double theta = (aqq - app) / (2.0 * apq);
-                    const double t = copysign(1.0, theta) / (fabs(theta) + sqrt(fma(theta, theta, 1.0)));
-                    c = rsqrt(fma(t, t, 1.0));
-                    sn = t * c;
+                if (fabs(apq) > 1e-300) {
+                    // tan of the rotation angle to fp32 accuracy (a rotation by a slightly different angle still
+                    // is an exact similarity; it leaves 1e-7 of the pivot instead of nothing), then cos and
+                    // sin to fp64 accuracy from it, so that the rotation stays orthogonal: the cosine by two
+                    // Newton steps on a single-precision reciprocal square root
+                    const float theta = (float)(aqq - app) / (2.0f * (float)apq);    // inf when apq underflows: t = 0
+                    const float tf = copysignf(1.0f, theta) / (fabsf(theta) + sqrtf(fmaf(theta, theta, 1.0f)));
+                    const double t = (double)tf;
+                    const double x = fma(t, t, 1.0);                                 // in [1, 2]
+                    double r = (double)rsqrtf((float)x);
+                    r = r * fma(-0.5 * x, r * r, 1.5);
+                    r = r * fma(-0.5 * x, r * r, 1.5);
+                    c = r;
+                    sn = t * r;
                 }
                 s.rot_c[tid] = c; s.rot_s[tid] = sn; s.rot_p[tid] = pp; s.rot_q[tid] = qq;
             }
             __syncthreads();
-            // columns: A <- A J and V <- V J
-            for (int e = tid; e < 2 * n * half; e += kEigThreads) {
-                const int which = e / (n * half), r = e % (n * half);
-                const int i = r / half, k = r % half;
-                const int pp = s.rot_p[k], qq = s.rot_q[k];
-                const double c = s.rot_c[k], sn = s.rot_s[k];
-                double* mat = which ? s.v : s.a;
-                const double x = mat[i * LD + pp], y = mat[i * LD + qq];
-                mat[i * LD + pp] = fma(c, x, -sn * y);
-                mat[i * LD + qq] = fma(sn, x, c * y);
+            // columns: A <- A J and V <- V J.  A lane owns one index pair (there are at most 32), a warp takes
+            // every fourth row: no index arithmetic beyond additions, and the rotation stays in registers.
+            if (lane < half) {
+                const int pp = s.rot_p[lane], qq = s.rot_q[lane];
+                const double c = s.rot_c[lane], sn = s.rot_s[lane];
+                for (int i = warp; i < n; i += kEigThreads / 32) {
+                    double* ra = s.a + i * LD;
+                    double* rv = s.v + i * LD;
+                    const double x = ra[pp], y = ra[qq], u = rv[pp], w = rv[qq];
+                    ra[pp] = fma(c, x, -sn * y);
+                    ra[qq] = fma(sn, x, c * y);
+                    rv[pp] = fma(c, u, -sn * w);
+                    rv[qq] = fma(sn, u, c * w);
+                }
             }
             __syncthreads();
-            // rows: A <- J^T A
-            for (int e = tid; e < n * half; e += kEigThreads) {
-                const int k = e / n, i = e % n;
+            // rows: A <- J^T A.  A warp takes every fourth pair, its lanes the columns.
+            for (int k = warp; k < half; k += kEigThreads / 32) {
                 const int pp = s.rot_p[k], qq = s.rot_q[k];
                 const double c = s.rot_c[k], sn = s.rot_s[k];
-                const double x = s.a[pp * LD + i], y = s.a[qq * LD + i];
-                s.a[pp * LD + i] = fma(c, x, -sn * y);
-                s.a[qq * LD + i] = fma(sn, x, c * y);
+                for (int i = lane; i < n; i += 32) {
+                    const double x = s.a[pp * LD + i], y = s.a[qq * LD + i];
+                    s.a[pp * LD + i] = fma(c, x, -sn * y);
+                    s.a[qq * LD + i] = fma(sn, x, c * y);
+                }
             }
             __syncthreads();
         }
@@ -437,7 +466,7 @@ eig_kernel(Plan p, const double* __restrict__ g_partials, const float* __restric
     if (tid < MP) {
         double inv = 0.0;
         if (tid < m && !bad) {
-            const double lam = s.a[tid * LD + tid];
+            const double lam = ldexp(s.a[tid * LD + tid], scale_exp);
             if (lam < floor) atomicOr(&s.flags, COMPACTOR_STATUS_RANK);
             inv = rsqrt(fmax(lam, floor));
         }

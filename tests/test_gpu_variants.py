@@ -197,3 +197,26 @@ def test_eig_route_rejects_wide_sketches(B):
     with pytest.raises(B.CompactorError) as e:
         B.score_variant(shape, kr.cuda(), torch.eye(128).cuda(), out, ws, B.FACTOR_EIG, 1e-6)
     assert e.value.code == -2
+
+
+@pytest.mark.parametrize("shift", [-24, 20])
+def test_scores_do_not_depend_on_the_scale_of_the_keys(B, shift):
+    # K -> 2^shift K is exact in bf16 and in every sum of the Cholesky route: the scores are bit-identical.
+    # The eigen route with an inactive floor agrees to rounding (its rotation angles are rounded differently).
+    w = inputs.Workload("scale", 1, 2, 128, [3000, 500], [0.3, 0.3], p=0.7, seed=61)
+    _, kr, _ = inputs.make_tensors(w, device="cpu", want_pre=False)
+    scaled = (kr.float() * 2.0 ** shift).bfloat16()
+    assert torch.equal(scaled.float() * 2.0 ** -shift, kr.float())              # the scaling was exact
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    phi = inputs.make_sketch_matrix(w.d, w.m, w.seed).cuda()
+    ws = torch.empty(B.workspace_bytes(shape), dtype=torch.uint8, device="cuda")
+    out = [torch.empty((1, 2, 3500), dtype=torch.float32, device="cuda") for _ in range(4)]
+    B.score(shape, kr.cuda(), phi, out[0], ws)
+    B.score(shape, scaled.cuda(), phi, out[1], ws)
+    floor = 1e-6 * 4.0 ** min(shift, 0)                                          # far below either spectrum
+    B.score_variant(shape, kr.cuda(), phi, out[2], ws, B.FACTOR_EIG, floor)
+    B.score_variant(shape, scaled.cuda(), phi, out[3], ws, B.FACTOR_EIG, floor)
+    torch.cuda.synchronize()
+    assert torch.equal(out[0], out[1])
+    np.testing.assert_allclose(out[3].cpu().numpy(), out[2].cpu().numpy(), rtol=2e-5)
+    np.testing.assert_allclose(out[2].cpu().numpy(), out[0].cpu().numpy(), rtol=2e-4)

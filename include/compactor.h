@@ -11,7 +11,10 @@
  *     ordinary host memory, read before the call returns.  The library never allocates or frees
  *     device memory: every buffer, including the workspace, belongs to the caller.
  *   - Device work is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
- *     void*; NULL is the default stream) and the call returns without synchronising.
+ *     void*; NULL is the default stream) and the call returns without synchronising.  With up to
+ *     239 sequences per call everything enqueued is a kernel or a memset (the prefix tables travel
+ *     as a kernel argument), so the call can be recorded into a CUDA graph and replayed on new
+ *     contents of the same buffers; larger batches copy their tables from host memory instead.
  *   - Keys/values are bf16 with the d channels of a token contiguous; the other three strides
  *     (layer, KV head, token) are given in ELEMENTS and must be multiples of 8 (16 bytes); base
  *     pointers must be 16-byte aligned.  d must be 128.  1 <= m <= 128.

@@ -136,12 +136,30 @@ Mat to_mat(const compactor_mat& m) {
     return r;
 }
 
-// Copies the tables to the head of the workspace and points the plan at them.
+// Tables of up to kInlineTableInts entries travel to the device as a kernel argument: no copy from
+// host memory is enqueued, so the call can be recorded into a CUDA graph and replayed.
+constexpr int kInlineTableInts = 960;
+struct InlineTables { int n; int v[kInlineTableInts]; };
+__global__ void write_tables_kernel(const __grid_constant__ InlineTables t, int* __restrict__ dst) {
+    for (int i = threadIdx.x; i < t.n; i += blockDim.x) dst[i] = t.v[i];
+}
+
+// Puts the tables at the head of the workspace and points the plan at them.
 cudaError_t upload_tables(HostPlan* hp, void* ws, cudaStream_t stream) {
     const int nb1 = hp->plan.batch + 1;
     int* dev = reinterpret_cast<int*>(static_cast<char*>(ws) + hp->off_tables);
-    // The source is pageable host memory: the runtime stages it before this call returns.
-    cudaError_t e = cudaMemcpyAsync(dev, hp->tables.data(), sizeof(int) * 4 * nb1, cudaMemcpyHostToDevice, stream);
+    cudaError_t e;
+    if (4 * nb1 <= kInlineTableInts) {
+        InlineTables t;
+        t.n = 4 * nb1;
+        memcpy(t.v, hp->tables.data(), sizeof(int) * 4 * nb1);
+        write_tables_kernel<<<1, 256, 0, stream>>>(t, dev);
+        e = cudaGetLastError();
+    } else {
+        // Larger batches: a copy from pageable host memory, which the runtime stages before this call
+        // returns (such a call cannot be recorded into a graph).
+        e = cudaMemcpyAsync(dev, hp->tables.data(), sizeof(int) * 4 * nb1, cudaMemcpyHostToDevice, stream);
+    }
     hp->plan.cu_seqlens = dev;
     hp->plan.cu_keep = dev + nb1;
     hp->plan.cu_chunks = dev + 2 * nb1;

@@ -135,7 +135,8 @@ __device__ uint32_t radix_select(SelectSmem& s, int want, int* ties, Visit visit
 // to the top `want`.  `sample` / `n_sample` are some of the values, used to guess their range.
 template <class Visit>
 __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __restrict__ sample, int n_sample,
-                                   int want_total, int* ties) {
+                                   int want_total, int* ties, bool* all_finite_out = nullptr) {
+    if (all_finite_out != nullptr) *all_finite_out = false;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     // ---- value range from a sample ------------------------------------------------------------
     {
@@ -192,6 +193,7 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
         const int members = s.hist[tbin];
         __syncthreads();
         if (!any_nonfinite && members <= kCand) {
+            if (all_finite_out != nullptr) *all_finite_out = true;       // every value has been seen and is finite
             visit([&](float v) {
                 if (bin_of(v) == tbin) s.cand[atomicAdd(&s.n_cand, 1)] = order_key(v);
             });
@@ -214,6 +216,9 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
 // scores above and at the threshold, one block-wide scan turns the counts into output offsets, and
 // then each warp emits its stretch on its own (a shuffle scan of per-lane counts per 128 scores).
 // The pass is bound by instruction issue, hence four scores per load and per scan.
+// kPlain: every score is known to be finite, so that comparing the floats themselves orders them as the
+// keys do (and -0 == +0 either way); that saves the key mapping, which is most of the work per score.
+template <bool kPlain>
 __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n, uint32_t thr, int ties,
                              int* __restrict__ out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -225,10 +230,16 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
     const int vbegin = min(n_vec, warp * per_warp), vend = min(n_vec, vbegin + per_warp);
     constexpr int kAhead = 4;                                             // vector steps loaded together
 
+    const float thr_f = __uint_as_float((thr & 0x80000000u) ? (thr & 0x7fffffffu) : ~thr);   // the float behind the key
     auto flags = [&](const float4& q, int& g, int& e) {                   // 4-bit masks: above / at the threshold
-        const uint32_t k0 = order_key(q.x), k1 = order_key(q.y), k2 = order_key(q.z), k3 = order_key(q.w);
-        g = (k0 > thr) | ((k1 > thr) << 1) | ((k2 > thr) << 2) | ((k3 > thr) << 3);
-        e = (k0 == thr) | ((k1 == thr) << 1) | ((k2 == thr) << 2) | ((k3 == thr) << 3);
+        if (kPlain) {
+            g = (q.x > thr_f) | ((q.y > thr_f) << 1) | ((q.z > thr_f) << 2) | ((q.w > thr_f) << 3);
+            e = (q.x == thr_f) | ((q.y == thr_f) << 1) | ((q.z == thr_f) << 2) | ((q.w == thr_f) << 3);
+        } else {
+            const uint32_t k0 = order_key(q.x), k1 = order_key(q.y), k2 = order_key(q.z), k3 = order_key(q.w);
+            g = (k0 > thr) | ((k1 > thr) << 1) | ((k2 > thr) << 2) | ((k3 > thr) << 3);
+            e = (k0 == thr) | ((k1 == thr) << 1) | ((k2 == thr) << 2) | ((k3 == thr) << 3);
+        }
     };
 
     // ---- counts: head (warp 0), the warp's stretch, tail (last warp) ----------------------------
@@ -343,8 +354,10 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
         return;
     }
     int ties = 0;
-    const uint32_t thr = find_threshold(s, [&](auto f) { for_each_score(sc, n, f); }, sc, n, kk, &ties);
-    emit_ordered(s, sc, n, thr, ties, out);
+    bool all_finite = false;
+    const uint32_t thr = find_threshold(s, [&](auto f) { for_each_score(sc, n, f); }, sc, n, kk, &ties, &all_finite);
+    if (all_finite) emit_ordered<true>(s, sc, n, thr, ties, out);
+    else emit_ordered<false>(s, sc, n, thr, ties, out);
 }
 
 // ---- selection across the heads of a layer (Section 3.4's alternative) -------------------------
@@ -432,7 +445,7 @@ across_emit_kernel(Plan p, const float* __restrict__ scores, const uint32_t* __r
         for (int i = threadIdx.x; i < n; i += kThreads) out[i] = i;
         return;
     }
-    emit_ordered(s, sc, n, thr_in[lb], ties_in[lb * p.heads + head], out);
+    emit_ordered<false>(s, sc, n, thr_in[lb], ties_in[lb * p.heads + head], out);
 }
 
 // Eq. 6: s = z(a) + lambda z(o), population standard deviation, per unit.  Overwrites the

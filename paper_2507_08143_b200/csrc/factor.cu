@@ -122,30 +122,59 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
                         const int e = tid + q * kProjThreads;
                         acc[q] += __ldcs(cur.part + (size_t)pp * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
                     }
+                __syncthreads();                              // the previous item's products are done with c and t
+#pragma unroll
+                for (int q = 0; q < kPer; ++q) s.c[tid + q * kProjThreads] = acc[q];
             } else {
-                // short sequence: fp64 Gram straight from the keys
+                // short sequence: fp64 Gram straight from the keys, C[:, rows] = K^T K[:, rows], as fp64 mma.m8n8k4
+                // over four tokens at a time (a warp owns four 8 x 8 tiles of the 128 x 16 slice)
                 const int layer = cur.lh / p.heads, head = cur.lh % p.heads;
                 const __nv_bfloat16* kbase = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
                                              (long long)p.cu_seqlens[cur.b] * kmat.stride_token;
-                for (int t0 = 0; t0 < cur.n_tok; t0 += kStageTokens) {
-                    const int nt = min(kStageTokens, cur.n_tok - t0);
-                    __syncthreads();
-                    for (int i = tid; i < nt * kD; i += kProjThreads)
-                        s.keys[i] = (double)__bfloat162float(kbase[(long long)(t0 + i / kD) * kmat.stride_token + (i % kD)]);
-                    __syncthreads();
-                    for (int t = 0; t < nt; ++t) {
-                        const double* krow = s.keys + t * kD;
+                constexpr int kTilesPerWarp = (kD / 8) * (kRows / 8) / (kProjThreads / 32);
+                double d[kTilesPerWarp][2];
 #pragma unroll
-                        for (int q = 0; q < kPer; ++q) {
-                            const int e = tid + q * kProjThreads;
-                            acc[q] = fma(krow[e / kRows], krow[row0 + (e % kRows)], acc[q]);
+                for (int j = 0; j < kTilesPerWarp; ++j) d[j][0] = d[j][1] = 0.0;
+                // the keys of the next stage are on their way while the current stage is multiplied
+                constexpr int kLoads = kStageTokens * kD / kProjThreads;
+                float nxt[kLoads];
+                auto fetch = [&](int t0) {                    // missing tokens of the last stage are zeros
+#pragma unroll
+                    for (int u = 0; u < kLoads; ++u) {
+                        const int i = tid + u * kProjThreads, t = t0 + i / kD;
+                        nxt[u] = t < cur.n_tok ? __bfloat162float(kbase[(long long)t * kmat.stride_token + (i % kD)]) : 0.f;
+                    }
+                };
+                fetch(0);
+                for (int t0 = 0; t0 < cur.n_tok; t0 += kStageTokens) {
+                    __syncthreads();
+#pragma unroll
+                    for (int u = 0; u < kLoads; ++u) s.keys[tid + u * kProjThreads] = (double)nxt[u];
+                    __syncthreads();
+                    if (t0 + kStageTokens < cur.n_tok) fetch(t0 + kStageTokens);
+#pragma unroll
+                    for (int ks = 0; ks < kStageTokens / 4; ++ks) {
+                        const double* krow = s.keys + (ks * 4 + fk) * kD;          // token ks*4 + fk of the stage
+#pragma unroll
+                        for (int j = 0; j < kTilesPerWarp; ++j) {
+                            const int tile = warp + j * (kProjThreads / 32);
+                            const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
+                            const double a = krow[mt * 8 + fr];                     // A[channel][token]
+                            const double bv = krow[row0 + nt8 * 8 + fr];            // B[token][channel of the slice]
+                            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                                         : "+d"(d[j][0]), "+d"(d[j][1]) : "d"(a), "d"(bv));
                         }
                     }
                 }
-            }
-            __syncthreads();                                  // the previous item's products are done with c and t
+                __syncthreads();                              // the previous item's products are done with c and t
 #pragma unroll
-            for (int q = 0; q < kPer; ++q) s.c[tid + q * kProjThreads] = acc[q];
+                for (int j = 0; j < kTilesPerWarp; ++j) {
+                    const int tile = warp + j * (kProjThreads / 32);
+                    const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
+                    s.c[(mt * 8 + fr) * kRows + nt8 * 8 + 2 * fk] = d[j][0];
+                    s.c[(mt * 8 + fr) * kRows + nt8 * 8 + 2 * fk + 1] = d[j][1];
+                }
+            }
         }
         __syncthreads();
 

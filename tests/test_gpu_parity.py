@@ -285,3 +285,23 @@ def test_bounded_wait_gives_up_and_context_survives(B):
     x = torch.ones(8, device="cuda")
     assert float(x.sum()) == 8.0                       # the context is still usable
     assert B.wait_selftest() == 4
+
+
+def test_repeated_calls_are_bit_identical(B):
+    # no atomics on floating-point data and fixed summation orders everywhere: the same inputs give the same bits
+    w = inputs.Workload("repeat", 2, 3, 128, [5000, 300, 1400], [0.3, 0.5, 0.9], p=0.7, seed=44)
+    _, kr, v = [None if t is None else t.cuda() for t in inputs.make_tensors(w, device="cpu", want_pre=False)]
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    phi = inputs.make_sketch_matrix(w.d, w.m, w.seed)
+    keep = _keep(B, w)
+    q = inputs.make_queries(w, 2, device="cpu").cuda()
+    ws = B.alloc_workspace(shape)
+    runs = []
+    for _ in range(3):
+        attn = torch.empty(w.layers, w.heads, shape.total_tokens, dtype=torch.float32, device="cuda")
+        B.attention_scores(shape, q, kr, 2, attn, ws, scale=128 ** -0.5, pool=3)
+        outs = H.run_compress(B, shape, kr, kr, v, phi, keep, attn=attn)
+        runs.append((attn,) + tuple(outs))
+    for other in runs[1:]:
+        for a, b in zip(runs[0], other):
+            assert torch.equal(a, b)

@@ -30,7 +30,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the dominant kernels per head-token, from ncu captures of a smaller case of
 # the same kernels (see profiles/); bytes read + written per token of one (layer, head).
-NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN = {"gram": 257.1, "score": 260.7, "compact": 316.1}   # compact: at 32 % kept
+NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN = {}
 
 
 def parse_args():
@@ -124,16 +124,13 @@ def algorithmic_bytes(w, keep, mode):
     return per_lh * w.layers * w.heads
 
 
-def stage_bytes(w, keep, mode, chunk_tokens=32768):
+def stage_bytes(w, keep, mode):
     """Minimal bytes of each kernel run on its own (per step)."""
     row = w.d * 2
     lh = w.layers * w.heads
     tok = sum(w.seqlens); kept = sum(keep)
-    n_part = sum((n + chunk_tokens - 1) // chunk_tokens for n in w.seqlens)
     return {
-        "gram": lh * (tok * row + n_part * 131072),
-        "factor": lh * n_part * 131072,
-        "score": lh * tok * (row + 4),
+        "sweep": lh * tok * (row + 4),          # the keys once from HBM (their second read is meant to hit L2) + scores
         "blend": 0,
         "select": lh * (tok * 4 + kept * 4),
         "compact": lh * kept * (4 * row + 4),
@@ -416,7 +413,7 @@ def main():
                    "keep": keep if w.batch <= 4 else total_keep, "units_per_gpu": w.units,
                    "l2": "inputs (GBs per step) far exceed the 126 MB L2; no flush needed"},
         "head_tokens_per_s": value * L * Hh,
-        "gpu_launches": 7 * args.steps,
+        "gpu_launches": 4 * args.steps,
         "stage_ms": {k: round(t, 4) for k, t in stage_ms.items()},
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",

@@ -87,8 +87,8 @@ EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch
 FACTOR_CHOLESKY = 0
 FACTOR_EIG = 1
 
-N_STAGE_EVENTS = 7
-STAGE_NAMES = ["gram", "factor", "score", "blend", "select", "compact"]
+N_STAGE_EVENTS = 5
+STAGE_NAMES = ["sweep", "blend", "select", "compact"]
 
 
 def version() -> int:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcompactor.so")
-SOURCES = ["api.cu", "tensormap.cu", "gram.cu", "factor.cu", "score.cu", "select.cu", "compact.cu", "attention.cu", "nll.cu"]
+SOURCES = ["api.cu", "tensormap.cu", "sweep.cu", "gram.cu", "factor.cu", "score.cu", "select.cu", "compact.cu", "attention.cu", "nll.cu"]
 
 
 def _stale() -> bool:

@@ -1,6 +1,7 @@
 // Host entry points of the C ABI declared in compactor.h: argument checking, workspace layout
 // and kernel sequencing.  No device memory is allocated here.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -14,16 +15,66 @@ using namespace compactor;
 namespace {
 
 constexpr size_t kAlign = 256;
-constexpr int kSmCount = 148;   // B200; only used to pick the Gram block length
+constexpr int kFallbackSmCount = 148;     // B200, if the device cannot be asked
+constexpr int kFusedMaxMp = 48;           // widest padded sketch the fused sweep holds in shared memory
+constexpr int kPieceTokens = 1024;        // piece length of the fused sweep, doubled for very long sequences
+constexpr int kMaxPiecesPerUnit = 160;
+constexpr int kMaxCtas = 256;             // upper bound on the CTAs of the fused sweep (one per SM)
+constexpr size_t kL2WindowBytes = (size_t)64 << 20;   // keys that may wait in L2 between their two reads
 
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+// Number of SMs of the current device (asked once per device).
+int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return kFallbackSmCount;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = kFallbackSmCount;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+// The fused persistent sweep is switched on with COMPACTOR_FUSED_SWEEP=1 (it does not yet beat the
+// separate kernels; see sweep.cu).
+bool fused_sweep_enabled() {
+    const char* e = getenv("COMPACTOR_FUSED_SWEEP");
+    return e != nullptr && e[0] == '1';
+}
 
 struct HostPlan {
     Plan plan;
     std::vector<int> tables;       // cu_seqlens | cu_keep | cu_chunks | cu_schunks, each batch+1
     size_t off_tables, off_w, off_gpart, off_partials, off_scores, total_bytes;
     int units;
+    // fused sweep (Cholesky route, padded sketch of at most kFusedMaxMp columns)
+    bool fused;
+    int slices, window, n_slots, max_pieces;
+    long long total_pieces;
+    size_t off_sched, sched_bytes, off_tbuf;
 };
+
+// Workspace layout of the fused sweep for the plan's current window.
+void layout_fused(HostPlan* hp) {
+    const Plan& p = hp->plan;
+    const int nb1 = p.batch + 1;
+    // claims may run past the window by one piece per CTA
+    const long long want = (long long)hp->window + kMaxCtas;
+    const long long slots = hp->total_pieces < want ? hp->total_pieces : want;
+    hp->n_slots = (int)(slots < 1 ? 1 : slots);
+    size_t off = 0;
+    hp->off_tables = off;   off += align_up(sizeof(int) * 4 * nb1);
+    hp->off_sched = off;    hp->sched_bytes = sizeof(SweepSched) + sizeof(int) * 5 * (size_t)hp->units;
+                            off += align_up(hp->sched_bytes);
+    hp->off_w = off;        off += align_up(sizeof(__nv_bfloat16) * w_elems_per_unit(p.mp) * hp->units);
+    hp->off_tbuf = off;     off += align_up(sizeof(double) * kD * p.mp * (size_t)hp->units);
+    hp->off_partials = off; off += align_up(sizeof(float) * kGramElems * (size_t)hp->n_slots);
+    hp->off_gpart = hp->off_partials;
+    hp->off_scores = off;   off += align_up(sizeof(float) * (size_t)p.total_tokens * p.layers * p.heads);
+    hp->total_bytes = off;
+}
 
 bool shape_ok(const compactor_shape* s, int* err) {
     if (s == nullptr || s->cu_seqlens == nullptr) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
@@ -38,7 +89,8 @@ bool shape_ok(const compactor_shape* s, int* err) {
 }
 
 // Fills everything that depends on the shape alone (keep counts are added by the caller).
-bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
+// `allow_fused`: lay the workspace out for the fused sweep when the sketch is narrow enough.
+bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fused = true) {
     if (!shape_ok(s, err)) return false;
     Plan& p = hp->plan;
     memset(&p, 0, sizeof(p));
@@ -46,6 +98,59 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     p.m = s->m; p.mp = s->m <= 64 ? (s->m + 15) / 16 * 16 : 128;
     p.total_tokens = s->cu_seqlens[s->batch];
     hp->units = s->layers * s->heads * s->batch;
+    hp->fused = allow_fused && p.mp <= kFusedMaxMp && fused_sweep_enabled();
+    hp->slices = 0; hp->window = 0; hp->n_slots = 0; hp->max_pieces = 0; hp->total_pieces = 0;
+    hp->off_sched = 0; hp->sched_bytes = 0; hp->off_tbuf = 0;
+
+    if (hp->fused) {
+        // Pieces of 1024 tokens keep the keys that wait between their two reads within L2; sequences beyond
+        // 160 pieces get longer ones (their keys outlive L2 anyway) so that the ring of partials stays small.
+        long long n_max = 0;
+        for (int b = 0; b < s->batch; ++b) {
+            const long long n = s->cu_seqlens[b + 1] - s->cu_seqlens[b];
+            if (n > n_max) n_max = n;
+        }
+        int piece = kPieceTokens;
+        if (const char* e = getenv("COMPACTOR_PIECE_TOKENS")) {         // tuning aid: 1024, 2048, 4096, ...
+            const long v = strtol(e, nullptr, 10);
+            if (v >= kPieceTokens && v <= kMaxChunk && (v & (v - 1)) == 0) piece = (int)v;
+        }
+        while ((n_max + piece - 1) / piece > kMaxPiecesPerUnit && piece < kMaxChunk) piece *= 2;
+        const int nb1 = s->batch + 1;
+        hp->tables.assign((size_t)4 * nb1, 0);
+        int* cs = hp->tables.data();
+        int* cc = cs + 2 * nb1;
+        long long tc = 0;
+        for (int b = 0; b <= s->batch; ++b) cs[b] = s->cu_seqlens[b];
+        for (int b = 0; b < s->batch; ++b) {
+            tc += (cs[b + 1] - cs[b] + piece - 1) / piece;
+            if (tc > 0x7fffffffLL) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+            cc[b + 1] = (int)tc;
+        }
+        // row slices of a unit's projection: more of them the more partials there are to add up
+        int* csl = cs + 3 * nb1;
+        for (int b = 0; b < s->batch; ++b) {
+            const int pieces = cc[b + 1] - cc[b];
+            const int sl = pieces >= 96 ? 32 : pieces >= 48 ? 16 : pieces >= 24 ? 8 : pieces >= 12 ? 4 : pieces >= 4 ? 2 : 1;
+            csl[b + 1] = csl[b] + sl;
+        }
+        hp->total_pieces = tc * s->layers * s->heads;
+        if (hp->total_pieces > 0x7fffffffLL) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+        p.chunk = p.schunk = piece;
+        p.total_chunks = (int)tc;
+        p.total_schunks = csl[s->batch];
+        hp->max_pieces = (int)((n_max + piece - 1) / piece);
+        hp->slices = p.total_schunks;
+        size_t window_bytes = kL2WindowBytes;
+        if (const char* e = getenv("COMPACTOR_L2_WINDOW_MIB")) {        // tuning aid
+            const long v = strtol(e, nullptr, 10);
+            if (v > 0 && v < 65536) window_bytes = (size_t)v << 20;
+        }
+        const long long budget = (long long)(window_bytes / ((size_t)piece * kD * sizeof(__nv_bfloat16)));
+        hp->window = (int)(budget > hp->max_pieces + 1 ? budget : hp->max_pieces + 1);
+        layout_fused(hp);
+        return true;
+    }
 
     // Block length (tokens per CTA of the two sweeps, one fp64 Gram partial per block): the power
     // of two times 256 that minimises a small cost model - waves of CTAs over the SMs, a fixed
@@ -63,7 +168,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     double best = 1e300;
     for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
         const double ctas = (double)count_chunks(c) * s->layers * s->heads;
-        const double waves = ceil(ctas / kSmCount);
+        const double waves = ceil(ctas / kFallbackSmCount);
         const double per_cta_us = 4.0 + c * 256.0 / 44e3;             // 44 GB/s = 44e3 B/us per SM
         const double partial_us = ctas * 2.0 * 131072.0 / 6.4e6;      // written once, read once at 6.4 TB/s
         const double cost = waves * per_cta_us + partial_us;
@@ -80,7 +185,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err) {
     for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
         const double ctas = (double)count_chunks(c) * s->layers * s->heads;
         const double per_cta_us = 2.0 + c * 256.0 / 44e3;
-        const double cost = (ctas / kSmCount < 1.0 ? 1.0 : ctas / kSmCount) * per_cta_us + 0.5 * per_cta_us;
+        const double cost = (ctas / kFallbackSmCount < 1.0 ? 1.0 : ctas / kFallbackSmCount) * per_cta_us + 0.5 * per_cta_us;
         if (cost < best * 0.999) { best = cost; schunk = c; }
     }
     p.schunk = schunk;
@@ -179,26 +284,59 @@ struct Marks {
     }
 };
 
+#ifdef COMPACTOR_SWEEP_PROFILE
+long long* g_sweep_profile = nullptr;     // instrumented builds only: per-CTA cycle counters
+#endif
+
 int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn, float lambda,
                 float* scores, int32_t* status, char* ws, cudaStream_t stream, const Marks& mk = Marks(),
                 int factorization = COMPACTOR_FACTOR_CHOLESKY, double eig_floor = 0.0) {
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(ws + hp.off_w);
-    double* partials = reinterpret_cast<double*>(ws + hp.off_partials);
     if (status != nullptr) CK(cudaMemsetAsync(status, 0, sizeof(int32_t) * hp.units, stream));
-    CK(mk.mark(0, stream));
-    CK(launch_gram(hp.plan, k, partials, status, stream));
-    CK(mk.mark(1, stream));
-    CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, status,
-                     factorization, eig_floor, stream));
-    CK(mk.mark(2, stream));
-    CK(launch_score(hp.plan, k, w, scores, status, stream));
-    CK(mk.mark(3, stream));
+    if (hp.fused) {
+        // one persistent kernel: Gram pieces, factorisation and scoring pieces from a common work queue
+        if (factorization != COMPACTOR_FACTOR_CHOLESKY) return COMPACTOR_E_INVALID_ARGUMENT;
+        CK(cudaMemsetAsync(ws + hp.off_sched, 0, hp.sched_bytes, stream));
+        SweepArgs a;
+        memset(&a, 0, sizeof(a));
+        a.p = hp.plan; a.k = k;
+        a.units = hp.units; a.total_pieces = (int)hp.total_pieces;
+        a.total_ftasks = hp.plan.total_schunks * hp.plan.layers * hp.plan.heads;
+        a.window = hp.window; a.n_slots = hp.n_slots;
+        a.sched = reinterpret_cast<SweepSched*>(ws + hp.off_sched);
+        a.gram_done = reinterpret_cast<int*>(ws + hp.off_sched + sizeof(SweepSched));
+        a.slices_claimed = a.gram_done + hp.units;
+        a.slices_done = a.slices_claimed + hp.units;
+        a.score_claimed = a.slices_done + hp.units;
+        a.w_ready = a.score_claimed + hp.units;
+        a.partials = reinterpret_cast<float*>(ws + hp.off_partials);
+        a.t_buf = reinterpret_cast<double*>(ws + hp.off_tbuf);
+        a.w = w; a.phi = phi; a.scores = scores; a.status = status;
+#ifdef COMPACTOR_SWEEP_PROFILE
+        a.prof = g_sweep_profile;
+#endif
+        CK(mk.mark(0, stream));
+        CK(launch_sweep(a, sm_count() < kMaxCtas ? sm_count() : kMaxCtas, stream));
+        CK(mk.mark(1, stream));
+    } else {
+        double* partials = reinterpret_cast<double*>(ws + hp.off_partials);
+        CK(mk.mark(0, stream));
+        CK(launch_gram(hp.plan, k, partials, status, stream));
+        CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, status,
+                         factorization, eig_floor, stream));
+        CK(launch_score(hp.plan, k, w, scores, status, stream));
+        CK(mk.mark(1, stream));
+    }
     if (attn != nullptr) CK(launch_blend(hp.plan, attn, lambda, scores, stream));
-    CK(mk.mark(4, stream));
+    CK(mk.mark(2, stream));
     return COMPACTOR_OK;
 }
 
 }  // namespace
+
+#ifdef COMPACTOR_SWEEP_PROFILE
+extern "C" void compactor_debug_set_profile_buffer(long long* device_counters) { g_sweep_profile = device_counters; }
+#endif
 
 extern "C" {
 
@@ -208,7 +346,7 @@ const char* compactor_error_string(int code) {
     switch (code) {
         case COMPACTOR_OK: return "ok";
         case COMPACTOR_E_INVALID_ARGUMENT: return "invalid argument";
-        case COMPACTOR_E_UNSUPPORTED: return "unsupported shape (d must be 128, 1 <= m <= 64)";
+        case COMPACTOR_E_UNSUPPORTED: return "unsupported shape (d must be 128, 1 <= m <= 128)";
         case COMPACTOR_E_WORKSPACE: return "workspace too small";
         case COMPACTOR_E_CUDA: return "CUDA runtime error";
         case COMPACTOR_E_TOO_LARGE: return "problem needs more scratch than the built-in 32 MiB array holds";
@@ -254,9 +392,12 @@ int compactor_calibrated_ratio(double nll, double alpha, double beta, double tau
 }
 
 size_t compactor_workspace_bytes(const compactor_shape* shape) {
+    // enough for either route: the fused sweep and the separate kernels of the variants
     HostPlan hp; int err = 0;
-    if (!make_plan(shape, &hp, &err)) return 0;
-    return hp.total_bytes;
+    if (!make_plan(shape, &hp, &err, false)) return 0;
+    const size_t separate = hp.total_bytes;
+    if (!make_plan(shape, &hp, &err, true)) return 0;
+    return hp.total_bytes > separate ? hp.total_bytes : separate;
 }
 
 int compactor_score(const compactor_shape* shape, compactor_mat k_score, const float* phi,
@@ -285,7 +426,7 @@ int compactor_score_variant(const compactor_shape* shape, compactor_mat k_score,
     if (factorization != COMPACTOR_FACTOR_EIG) return COMPACTOR_E_INVALID_ARGUMENT;
     if (!(eig_floor > 0.0) || !std::isfinite(eig_floor)) return COMPACTOR_E_INVALID_ARGUMENT;
     HostPlan hp; int err = 0;
-    if (!make_plan(shape, &hp, &err)) return err;
+    if (!make_plan(shape, &hp, &err, false)) return err;
     if (hp.plan.mp > 64) return COMPACTOR_E_UNSUPPORTED;
     if (!mat_ok(k_score) || phi == nullptr || scores_out == nullptr || workspace == nullptr)
         return COMPACTOR_E_INVALID_ARGUMENT;
@@ -354,11 +495,11 @@ static int compress_impl(const compactor_shape* shape, compactor_mat k_score, co
     int rc = run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores, status, ws, st, mk);
     if (rc != COMPACTOR_OK) return rc;
     if (hp.plan.total_keep > 0) CK(launch_select(hp.plan, scores, idx_out, st));
-    CK(mk.mark(5, st));
+    CK(mk.mark(3, st));
     if (hp.plan.total_keep > 0)
         CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out,
                           static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
-    CK(mk.mark(6, st));
+    CK(mk.mark(4, st));
     return COMPACTOR_OK;
 }
 
@@ -446,8 +587,16 @@ int compactor_score_builtin_scratch(const compactor_shape* shape, compactor_mat 
     HostPlan hp; int err = 0;
     if (!make_plan(shape, &hp, &err)) return err;
     if (!mat_ok(k_score) || phi == nullptr || scores_out == nullptr) return COMPACTOR_E_INVALID_ARGUMENT;
-    // Everything before the scores region must fit; longer Gram blocks need less scratch.
-    while (hp.off_scores > kBuiltinScratchBytes && hp.plan.chunk < kMaxChunk) replan_chunk(shape, &hp, hp.plan.chunk * 2);
+    // Everything before the scores region must fit.  The fused sweep gets by with a shorter ring of Gram
+    // partials (fewer pieces between the two reads of the keys); the separate kernels with longer Gram blocks.
+    if (hp.fused) {
+        while (hp.off_scores > kBuiltinScratchBytes && hp.window > hp.max_pieces + 1) {
+            hp.window = hp.window / 2 > hp.max_pieces + 1 ? hp.window / 2 : hp.max_pieces + 1;
+            layout_fused(&hp);
+        }
+    } else {
+        while (hp.off_scores > kBuiltinScratchBytes && hp.plan.chunk < kMaxChunk) replan_chunk(shape, &hp, hp.plan.chunk * 2);
+    }
     if (hp.off_scores > kBuiltinScratchBytes) return COMPACTOR_E_TOO_LARGE;
     if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
     void* scratch = nullptr;
@@ -487,7 +636,7 @@ extern "C" int compactor_attention_scores(const compactor_shape* shape, compacto
                                           int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,
                                           float* attn_out, void* workspace, size_t workspace_bytes, void* stream) {
     HostPlan hp; int err = 0;
-    if (!make_plan(shape, &hp, &err)) return err;
+    if (!make_plan(shape, &hp, &err, false)) return err;
     if (chunk != 256) return COMPACTOR_E_UNSUPPORTED;
     if (!mat_ok(q) || !mat_ok(k) || attn_out == nullptr || workspace == nullptr || q_per_kv < 1 ||
         (long long)shape->heads * q_per_kv > 65535 || !(scale > 0.f) || !isfinite(scale) || pool < 1 || (pool & 1) == 0)

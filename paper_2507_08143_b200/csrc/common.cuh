@@ -39,6 +39,40 @@ struct Mat {               // compactor_mat with a typed pointer
     long long stride_layer, stride_head, stride_token;
 };
 
+// Shared state of the fused sweep's work queue (global memory, zeroed before every launch).  Both
+// 64-bit words are only ever changed by compare-and-swap.
+struct SweepSched {
+    unsigned long long fstate;   // high half: leading units whose slices are all claimed; low half: leading units whose Gram pieces are all in
+    unsigned long long sstate;   // high half: leading units whose scoring pieces are all claimed; low half: leading units whose W is written
+    unsigned int gram_next;      // Gram pieces claimed
+    unsigned int abort;          // a bounded wait ran out somewhere: everybody leaves
+    unsigned int pad[10];
+};
+
+// Arguments of the fused sweep.  `p.chunk` is the piece length and `p.total_chunks` / `p.cu_chunks`
+// count pieces; `p.total_schunks` / `p.cu_schunks` count the row slices of the factor tasks.
+struct SweepArgs {
+    Plan p;
+    Mat k;
+    int units, total_pieces;
+    int total_ftasks;            // factor tasks: (layer, head) x sum over sequences of their row slices (p.cu_schunks, p.total_schunks)
+    int window;                  // Gram pieces may run this far ahead of the scoring front
+    int n_slots;                 // partial slots (>= window + CTAs); piece i uses slot i % n_slots
+    SweepSched* sched;
+    int* gram_done;              // [units] finished Gram pieces
+    int* slices_claimed;         // [units] claimed slice tasks (may overshoot)
+    int* slices_done;            // [units] finished slice tasks
+    int* score_claimed;          // [units] claimed scoring pieces (may overshoot)
+    int* w_ready;                // [units] 1 once W is written
+    float* partials;             // [n_slots][128][128] fp32
+    double* t_buf;               // [units][128][mp] fp64: T = C Phi
+    __nv_bfloat16* w;            // [units][2][mp][128]
+    const float* phi;            // [128][m] fp32
+    float* scores;
+    int* status;
+    long long* prof;             // per-CTA cycle counters of an instrumented build, else null
+};
+
 // Largest b with table[b] <= x, for a non-decreasing table of nb+1 entries with table[0] = 0.
 __device__ __forceinline__ int find_segment(const int* __restrict__ table, int nb, int x) {
     int lo = 0, hi = nb;          // invariant: table[lo] <= x < table[hi] (table[nb] > x by construction)
@@ -56,6 +90,7 @@ cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, c
                           __nv_bfloat16* w, int* status, int factorization, double eig_floor, cudaStream_t stream);
 cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
                          cudaStream_t stream);
+cudaError_t launch_sweep(const SweepArgs& a, int sm_count, cudaStream_t stream);
 cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* scores, cudaStream_t stream);
 cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStream_t stream);
 cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int* idx,

@@ -11,10 +11,10 @@
  *     ordinary host memory, read before the call returns.  The library never allocates or frees
  *     device memory: every buffer, including the workspace, belongs to the caller.
  *   - Device work is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
- *     void*; NULL is the default stream) and the call returns without synchronising.  With up to
- *     239 sequences per call everything enqueued is a kernel or a memset (the prefix tables travel
- *     as a kernel argument), so the call can be recorded into a CUDA graph and replayed on new
- *     contents of the same buffers; larger batches copy their tables from host memory instead.
+ *     void*; NULL is the default stream) and the call returns without synchronising.  Everything
+ *     enqueued is a kernel or a memset (the prefix tables travel as kernel arguments, 239
+ *     sequences per small launch), so the call can be recorded into a CUDA graph and replayed on
+ *     new contents of the same buffers.
  *   - Keys/values are bf16 with the d channels of a token contiguous; the other three strides
  *     (layer, KV head, token) are given in ELEMENTS and must be multiples of 8 (16 bytes); base
  *     pointers must be 16-byte aligned.  d must be 128.  1 <= m <= 128.
@@ -234,11 +234,11 @@ int compactor_compress(const compactor_shape* shape, compactor_mat k_score, comp
  * compactor_compress with stage markers, for measurement (the paper reports one wall-clock
  * number per context length, Fig. 1; this splits ours by stage).  stage_events is a HOST array of
  * n_events cudaEvent_t handles created by the caller (NULL entries are skipped).  They are
- * recorded on the stream: [0] before the first kernel, [1] after the Gram pass, [2] after the
- * factorisation, [3] after the scoring pass, [4] after the blend (recorded even when there is
- * none), [5] after selection, [6] after compaction.  Results are identical to compactor_compress.
+ * recorded on the stream: [0] before the scoring sweep (Gram pass, factorisation, scoring pass),
+ * [1] after it, [2] after the blend (recorded even when there is none), [3] after selection,
+ * [4] after compaction.  Results are identical to compactor_compress.
  */
-#define COMPACTOR_N_STAGE_EVENTS 7
+#define COMPACTOR_N_STAGE_EVENTS 5
 int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
                                 compactor_mat v_cache, const float* phi, const float* attn_scores,
                                 float lambda, const int32_t* keep_counts,
@@ -266,6 +266,17 @@ int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_sc
 int compactor_attention_scores(const compactor_shape* shape, compactor_mat q, compactor_mat k,
                                int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,
                                float* attn_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * compactor_attention_scores (Eq. 5) with the per-unit status word of the other device calls:
+ * `status` (device int32 [layers*heads*batch], may be NULL) is cleared when the call starts and
+ * receives COMPACTOR_STATUS_TIMEOUT for every unit of a CTA one of whose bounded device-side waits
+ * ran out (the attention term of such a unit is unspecified).  Everything else as above.
+ */
+int compactor_attention_scores_status(const compactor_shape* shape, compactor_mat q, compactor_mat k,
+                                      int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,
+                                      float* attn_out, int32_t* status, void* workspace, size_t workspace_bytes,
+                                      void* stream);
 
 /*
  * Selection across the heads of a layer (Section 3.4 allows the top scores to be taken over all
@@ -299,7 +310,7 @@ int compactor_compact_across_heads(const compactor_shape* shape, compactor_mat k
  * the library on that device until the process exits.  The call allocates and frees nothing.
  *   - Size limit: the scratch must hold 16*(batch+1) bytes of tables, about 160 KiB per unit
  *     (at m = 48) and 128 KiB per Gram block (blocks are lengthened up to 65536 tokens to make it
- *     fit, i.e. down to 4 bytes per token per (layer, head)).  A larger problem is refused with
+ *     fit, i.e. down to 2 bytes per token per (layer, head)).  A larger problem is refused with
  *     COMPACTOR_E_TOO_LARGE before anything is enqueued; split it by layers or use
  *     compactor_score.
  *   - The first call on each device looks up the array's device address; make that first call

@@ -61,6 +61,8 @@ def _load() -> ctypes.CDLL:
     lib.compactor_compress_profiled.argtypes = lib.compactor_compress.argtypes + [POINTER(c_void_p), c_int32]
     lib.compactor_attention_scores.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_int32, c_int32,
                                                c_float, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_attention_scores_status.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_int32, c_int32,
+                                                      c_float, c_int32, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.compactor_across_heads_workspace_bytes.restype = c_size_t
     lib.compactor_across_heads_workspace_bytes.argtypes = [POINTER(CompactorShape)]
     lib.compactor_select_across_heads.argtypes = [POINTER(CompactorShape), c_void_p, POINTER(c_int32), c_void_p, c_void_p,
@@ -80,7 +82,7 @@ LIB_PATH = _build.LIB
 EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch", "compactor_make_sketch_srht", "compactor_keep_count",
            "compactor_calibrated_ratio", "compactor_fit_calibration", "compactor_workspace_bytes", "compactor_score", "compactor_select",
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
-           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores", "compactor_wait_selftest",
+           "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores", "compactor_attention_scores_status", "compactor_wait_selftest",
            "compactor_across_heads_workspace_bytes", "compactor_select_across_heads", "compactor_compact_across_heads",
            "compactor_score_variant", "compactor_nll"]
 
@@ -268,10 +270,16 @@ def score_builtin_scratch(shape: Shape, k_score: torch.Tensor, phi: torch.Tensor
 
 
 def attention_scores(shape: Shape, q: torch.Tensor, k: torch.Tensor, q_per_kv: int, attn_out: torch.Tensor,
-                     workspace: torch.Tensor, scale: float, pool: int = 1, chunk: int = 256) -> None:
+                     workspace: torch.Tensor, scale: float, pool: int = 1, chunk: int = 256,
+                     status: Optional[torch.Tensor] = None) -> None:
     """Eq. 5: chunked non-causal attention column sums of `q` [layers, heads*q_per_kv, tokens, d] against `k`."""
-    _check(LIB.compactor_attention_scores(byref(shape.c), mat(q), mat(k), q_per_kv, chunk, scale, pool, _ptr(attn_out),
-                                          _ptr(workspace), workspace.numel(), _stream()), "compactor_attention_scores")
+    if status is None:
+        _check(LIB.compactor_attention_scores(byref(shape.c), mat(q), mat(k), q_per_kv, chunk, scale, pool, _ptr(attn_out),
+                                              _ptr(workspace), workspace.numel(), _stream()), "compactor_attention_scores")
+    else:
+        _check(LIB.compactor_attention_scores_status(byref(shape.c), mat(q), mat(k), q_per_kv, chunk, scale, pool,
+                                                     _ptr(attn_out), _ptr(status), _ptr(workspace), workspace.numel(),
+                                                     _stream()), "compactor_attention_scores_status")
 
 
 def across_heads_workspace_bytes(shape: Shape) -> int:

@@ -241,8 +241,9 @@ Mat to_mat(const compactor_mat& m) {
     return r;
 }
 
-// Tables of up to kInlineTableInts entries travel to the device as a kernel argument: no copy from
-// host memory is enqueued, so the call can be recorded into a CUDA graph and replayed.
+// The tables travel to the device as kernel arguments, kInlineTableInts entries per launch: no copy from
+// host memory is enqueued, so the call never makes the runtime wait for the stream and can be recorded
+// into a CUDA graph and replayed, whatever the batch size.
 constexpr int kInlineTableInts = 960;
 struct InlineTables { int n; int v[kInlineTableInts]; };
 __global__ void write_tables_kernel(const __grid_constant__ InlineTables t, int* __restrict__ dst) {
@@ -253,23 +254,20 @@ __global__ void write_tables_kernel(const __grid_constant__ InlineTables t, int*
 cudaError_t upload_tables(HostPlan* hp, void* ws, cudaStream_t stream) {
     const int nb1 = hp->plan.batch + 1;
     int* dev = reinterpret_cast<int*>(static_cast<char*>(ws) + hp->off_tables);
-    cudaError_t e;
-    if (4 * nb1 <= kInlineTableInts) {
+    const long long total = 4LL * nb1;
+    for (long long done = 0; done < total; done += kInlineTableInts) {
         InlineTables t;
-        t.n = 4 * nb1;
-        memcpy(t.v, hp->tables.data(), sizeof(int) * 4 * nb1);
-        write_tables_kernel<<<1, 256, 0, stream>>>(t, dev);
-        e = cudaGetLastError();
-    } else {
-        // Larger batches: a copy from pageable host memory, which the runtime stages before this call
-        // returns (such a call cannot be recorded into a graph).
-        e = cudaMemcpyAsync(dev, hp->tables.data(), sizeof(int) * 4 * nb1, cudaMemcpyHostToDevice, stream);
+        t.n = (int)(total - done < kInlineTableInts ? total - done : kInlineTableInts);
+        memcpy(t.v, hp->tables.data() + done, sizeof(int) * t.n);
+        write_tables_kernel<<<1, 256, 0, stream>>>(t, dev + done);
+        const cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
     }
     hp->plan.cu_seqlens = dev;
     hp->plan.cu_keep = dev + nb1;
     hp->plan.cu_chunks = dev + 2 * nb1;
     hp->plan.cu_schunks = dev + 3 * nb1;
-    return e;
+    return cudaSuccess;
 }
 
 #define CK(expr) do { cudaError_t e__ = (expr); if (e__ != cudaSuccess) return COMPACTOR_E_CUDA; } while (0)
@@ -632,9 +630,10 @@ extern "C" int compactor_nll(const void* logits, int32_t logits_dtype, int64_t r
 
 // ---------------------------------------------------------------------------------------------
 // Attention term (Eq. 5).
-extern "C" int compactor_attention_scores(const compactor_shape* shape, compactor_mat q, compactor_mat k,
-                                          int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,
-                                          float* attn_out, void* workspace, size_t workspace_bytes, void* stream) {
+extern "C" int compactor_attention_scores_status(const compactor_shape* shape, compactor_mat q, compactor_mat k,
+                                                 int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,
+                                                 float* attn_out, int32_t* status, void* workspace,
+                                                 size_t workspace_bytes, void* stream) {
     HostPlan hp; int err = 0;
     if (!make_plan(shape, &hp, &err, false)) return err;
     if (chunk != 256) return COMPACTOR_E_UNSUPPORTED;
@@ -647,10 +646,18 @@ extern "C" int compactor_attention_scores(const compactor_shape* shape, compacto
     if (workspace_bytes < hp.off_w + raw_bytes) return COMPACTOR_E_WORKSPACE;
     if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (status != nullptr) CK(cudaMemsetAsync(status, 0, sizeof(int32_t) * hp.units, st));
     CK(upload_tables(&hp, workspace, st));
     float* raw = reinterpret_cast<float*>(static_cast<char*>(workspace) + hp.off_w);
-    CK(launch_attention(hp.plan, to_mat(q), to_mat(k), q_per_kv, scale, pool, raw, attn_out, st));
+    CK(launch_attention(hp.plan, to_mat(q), to_mat(k), q_per_kv, scale, pool, raw, attn_out, status, st));
     return COMPACTOR_OK;
+}
+
+extern "C" int compactor_attention_scores(const compactor_shape* shape, compactor_mat q, compactor_mat k,
+                                          int32_t q_per_kv, int32_t chunk, float scale, int32_t pool,
+                                          float* attn_out, void* workspace, size_t workspace_bytes, void* stream) {
+    return compactor_attention_scores_status(shape, q, k, q_per_kv, chunk, scale, pool, attn_out, nullptr, workspace,
+                                             workspace_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -88,13 +88,14 @@ __device__ __forceinline__ void softmax_pair_sync(int q) {     // the two warps 
 }
 
 // Where a work item (one chunk of one layer and KV head) lies.
-struct AttnItem { int layer, head, lh, tok_begin, n_tok; };
+struct AttnItem { int layer, head, lh, b, tok_begin, n_tok; };
 __device__ __forceinline__ AttnItem attn_item(const Plan& p, int item) {
     AttnItem a;
     a.lh = item / p.total_chunks;
     const int chunk_id = item % p.total_chunks;
     a.layer = a.lh / p.heads; a.head = a.lh % p.heads;
     const int b = find_segment(p.cu_chunks, p.batch, chunk_id);
+    a.b = b;
     a.tok_begin = p.cu_seqlens[b] + (chunk_id - p.cu_chunks[b]) * kChunk;
     a.n_tok = min(kChunk, p.cu_seqlens[b + 1] - a.tok_begin);
     return a;
@@ -104,7 +105,7 @@ __device__ __forceinline__ AttnItem attn_item(const Plan& p, int item) {
 // up once.  Halves are numbered through all of a CTA's items (g), which fixes every barrier's phase.
 __global__ void __launch_bounds__(kThreads, 1)
 attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
-                 int q_per_kv, float scale_log2e, int n_items, float* __restrict__ out) {
+                 int q_per_kv, float scale_log2e, int n_items, float* __restrict__ out, int* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
     AttnSmem& s = *reinterpret_cast<AttnSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
     const int n_iter = 2 * q_per_kv;                   // halves of 128 query rows per item (even)
@@ -235,15 +236,19 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         };
         const int n_halves = my_items * n_iter;
         AttnItem cur = attn_item(p, blockIdx.x), prev = cur;
-        bool ok = true;
-        for (int g = 0; g < n_halves && ok; ++g) {
+        // A wait that gives up raises the abort flag; from then on no softmax thread waits any more, and all of them
+        // keep the same control flow (so nobody is left alone at a named barrier); the results are then garbage
+        // and the unit is flagged.
+        auto wait_ft = [&](uint64_t* bar, uint32_t parity) {
+            if (*(volatile int*)&s.abort || *(volatile int*)&s.abort_mma) return;
+            if (!mbar_wait(bar, parity)) s.abort = 1;
+        };
+        for (int g = 0; g < n_halves; ++g) {
             const int r = g / n_iter, it = g - r * n_iter;
             if (it == 0 && r > 0) { prev = cur; cur = attn_item(p, blockIdx.x + r * gridDim.x); }
             const int n_tok = cur.n_tok;
             const bool full = n_tok == kChunk;               // only the last chunk of a sequence needs masks
-            // the two warps of a pair take the same decisions here (they meet at a named barrier below)
-            ok = mbar_wait(&s.s_full[g & 1], (g >> 1) & 1) && !*(volatile int*)&s.abort_mma;
-            if (!ok) break;
+            wait_ft(&s.s_full[g & 1], (g >> 1) & 1);
             tc_fence_after_sync();
             const uint32_t lane_addr = quad_addr + (uint32_t)(g & 1) * 256 + ch * 128;
             const bool row_valid = (it & 1) * kHalf + row < n_tok;
@@ -312,8 +317,7 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             if (g > 0) {
                 // E and the weights of the previous half have been multiplied: they may be overwritten,
                 // and its column sums are waiting in its accumulator
-                ok = mbar_wait(&s.c_full[(g - 1) & 1], ((g - 1) >> 1) & 1) && !*(volatile int*)&s.abort_mma;
-                if (!ok) break;
+                wait_ft(&s.c_full[(g - 1) & 1], ((g - 1) >> 1) & 1);
                 tc_fence_after_sync();
                 take_column_sums(g - 1);
                 tc_fence_before_sync();
@@ -354,20 +358,24 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             tc_fence_before_sync();
             mbar_arrive(&s.p_ready);
         }
-        if (!ok) s.abort = 1;
         if (n_halves > 0) {                       // the last half's column sums, then the last item's result
             const int last = n_halves - 1;
-            const bool okd = ok && mbar_wait(&s.c_full[last & 1], (last >> 1) & 1) && !*(volatile int*)&s.abort_mma;
+            wait_ft(&s.c_full[last & 1], (last >> 1) & 1);
             tc_fence_after_sync();
-            if (okd) {
-                take_column_sums(last);
-                write_result(cur);
-            }
+            take_column_sums(last);
+            write_result(cur);
         }
     }
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem, kTmemCols);
+    if (threadIdx.x == 0 && (s.abort || s.abort_mma) && status != nullptr && my_items > 0) {
+        // a bounded wait ran out: flag every unit this CTA worked on
+        for (int r = 0; r < my_items; ++r) {
+            const AttnItem it = attn_item(p, blockIdx.x + r * gridDim.x);
+            atomicOr(&status[it.lh * p.batch + it.b], COMPACTOR_STATUS_TIMEOUT);
+        }
+    }
 }
 
 // Centred mean over `pool` tokens inside each sequence, zero beyond its ends.
@@ -387,7 +395,7 @@ __global__ void pool_kernel(Plan p, const float* __restrict__ raw, float* __rest
 }  // namespace
 
 cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_per_kv, float scale, int pool,
-                             float* raw, float* out, cudaStream_t stream) {
+                             float* raw, float* out, int* status, cudaStream_t stream) {
     if (p.total_chunks == 0) return cudaSuccess;
     CUtensorMap qmap, kmap;
     if (!make_kv_tensor_map(&qmap, q.ptr, p.layers, p.heads * q_per_kv, p.total_tokens, q.stride_layer, q.stride_head,
@@ -405,7 +413,7 @@ cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_pe
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     const int grid = (int)(n_items < n_sm ? n_items : n_sm);          // one CTA per SM (shared memory)
     attention_kernel<<<grid, kThreads, smem, stream>>>(p, qmap, kmap, q_per_kv, scale * 1.4426950408889634f,
-                                                       (int)n_items, dst);
+                                                       (int)n_items, dst, status);
     e = cudaGetLastError();
     if (e != cudaSuccess || pool <= 1) return e;
     pool_kernel<<<dim3((p.total_tokens + 255) / 256, p.layers * p.heads), 256, 0, stream>>>(p, raw, out, pool);

@@ -105,7 +105,7 @@ cudaError_t launch_select_across(const Plan& p, const float* scores, int* idx, i
 cudaError_t launch_compact_across(const Plan& p, const Mat& k, const Mat& v, const int* idx, const int* head_offsets,
                                   __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream);
 cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_per_kv, float scale, int pool,
-                             float* raw, float* out, cudaStream_t stream);
+                             float* raw, float* out, int* status, cudaStream_t stream);
 
 // Bytes of W (two bf16 terms, [term][mp][128]) per unit.
 __host__ __device__ inline size_t w_elems_per_unit(int mp) { return (size_t)2 * mp * kD; }

@@ -159,9 +159,10 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
         const int et = threadIdx.x - 64;                     // 0..127 among the epilogue threads
         for (int t = 0; t < n_tiles; ++t) {
             const int buf = t % kBufs, use = t / kBufs;
-            // all 128 epilogue threads take the same decision (they meet at a named barrier below)
-            const bool ok = mbar_wait(&s.d_full[buf], use & 1) && !*(volatile int*)&s.abort_mma;
-            if (!ok) { s.abort = 1; break; }
+            // A wait that gives up raises the abort flag; after that no epilogue thread waits any more, and all of
+            // them keep walking the tiles (so that nobody is left alone at the named barrier below): the scores
+            // of the unit are then garbage and the unit is flagged.
+            if (!*(volatile int*)&s.abort && !*(volatile int*)&s.abort_mma && !mbar_wait(&s.d_full[buf], use & 1)) s.abort = 1;
             tc_fence_after_sync();
             // all loads of a group are issued before the one wait: their latencies overlap
             const uint32_t d_row = tmem + ((uint32_t)(q * 32) << 16) + buf * kCols;

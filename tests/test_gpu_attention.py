@@ -30,8 +30,10 @@ def _attention(B, w, q_per_kv, pool, scale, q=None, k=None):
     shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
     out = torch.full((w.layers, w.heads, shape.total_tokens), float("nan"), dtype=torch.float32, device="cuda")
     ws = B.alloc_workspace(shape)
-    B.attention_scores(shape, q, k, q_per_kv, out, ws, scale=scale, pool=pool)
+    status = torch.full((w.layers * w.heads * w.batch,), -1, dtype=torch.int32, device="cuda")
+    B.attention_scores(shape, q, k, q_per_kv, out, ws, scale=scale, pool=pool, status=status)
     torch.cuda.synchronize()
+    assert int(status.abs().max()) == 0, "no bounded wait may run out in a healthy run (status is cleared by the call)"
     return shape, q, k, out
 
 

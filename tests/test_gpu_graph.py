@@ -1,5 +1,5 @@
 """The fused call recorded into a CUDA graph and replayed: every step is a kernel or a memset on the
-caller's stream (the prefix tables of up to 239 sequences travel as a kernel argument), so a replay
+caller's stream (the prefix tables travel as kernel arguments, 239 sequences per launch), so a replay
 with new contents in the same buffers gives what a direct call gives."""
 import pytest
 import torch
@@ -50,3 +50,42 @@ def test_compress_replayed_from_a_cuda_graph_matches_direct_calls():
         for a, b in zip(g_out, d_out):
             assert torch.equal(a, b), f"replay differs from a direct call (seed {seed})"
         assert int(g_out[1].min()) >= 0
+
+
+def test_batch_of_several_hundred_sequences_under_capture():
+    # more sequences than one table launch carries: still nothing but kernels and memsets, so capture works,
+    # and the units come out as in separate one-sequence calls
+    from paper_2507_08143_b200 import binding as B
+    import numpy as np
+    rng = np.random.default_rng(5)
+    seqlens = [int(x) for x in rng.integers(1, 700, size=523)]
+    w = inputs.Workload("many", 1, 2, 128, seqlens, [0.4] * len(seqlens), p=0.7, seed=81)
+    _, kr, v = [None if t is None else t.cuda() for t in inputs.make_tensors(w, device="cpu", want_pre=False)]
+    shape = B.Shape(1, 2, 128, 48, seqlens)
+    keep = [B.keep_count(n, 0.4) for n in seqlens]
+    phi = inputs.make_sketch_matrix(128, 48, 1).cuda()
+    T, KK = shape.total_tokens, sum(keep)
+    scores = torch.full((1, 2, T), -1.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((1, 2, KK), -1, dtype=torch.int32, device="cuda")
+    ko = torch.zeros(1, 2, KK, 128, dtype=torch.bfloat16, device="cuda"); vo = torch.zeros_like(ko)
+    ws = B.alloc_workspace(shape)
+    B.compress(shape, kr, kr, v, phi, keep, idx, ko, vo, ws, scores_out=scores)
+    torch.cuda.synchronize()
+    direct = (scores.clone(), idx.clone(), ko.clone(), vo.clone())
+    for t in (scores, idx, ko, vo):
+        t.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        B.compress(shape, kr, kr, v, phi, keep, idx, ko, vo, ws, scores_out=scores)
+    graph.replay()
+    torch.cuda.synchronize()
+    for a, b in zip((scores, idx, ko, vo), direct):
+        assert torch.equal(a, b)
+    cu, ck = shape.cu_seqlens, np.concatenate([[0], np.cumsum(keep)])
+    for b in (0, 239, 240, 522):                      # either side of the first table launch, and the last sequence
+        one = B.Shape(1, 2, 128, 48, [seqlens[b]])
+        s1 = torch.empty(1, 2, seqlens[b], dtype=torch.float32, device="cuda")
+        B.score(one, kr[:, :, cu[b]:cu[b + 1]], phi, s1, B.alloc_workspace(one))
+        torch.cuda.synchronize()
+        # the two calls may cut the Gram sums into different blocks: equal up to fp32 rounding of those sums
+        assert torch.allclose(s1, scores[:, :, cu[b]:cu[b + 1]], rtol=1e-4, atol=0), f"sequence {b}"

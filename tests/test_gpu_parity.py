@@ -249,6 +249,38 @@ def test_fewer_rows_than_sketch_columns(B):
     scores, idx, ko, vo, status = H.run_compress(B, shape, kr, kr, v, phi, keep)
     s = scores.cpu().numpy()
     np.testing.assert_allclose(s[:, :, :45], 1.0, rtol=2e-3)
+    # the 48-token sequence has exactly as many rows as the sketch has columns: K^ is square, and as long as
+    # it is well conditioned (it is for this seed: the oracle says so too) every score is 1 as well
+    worst, _ = H.compare_all_units(shape, keep, (scores, idx, ko, vo, status), kr, kr, v, phi, what="short")
+    np.testing.assert_allclose(s[:, :, 45:], 1.0, rtol=2e-3)
+    st = status.cpu().numpy().reshape(2, 3)
+    assert np.all(st[:, :2] & 2) and not np.any(st & ~2)       # n < m: rank deficient by construction, nothing else flagged
+
+
+@pytest.mark.parametrize("n", [47, 48, 49])
+def test_sequence_lengths_around_the_sketch_dimension(B, n):
+    # n = m - 1: one direction of the sketch is empty (scores 1, rank flag); n = m: square K^; n = m + 1: the first
+    # length with scores below 1.  All against the oracle, status bits included.
+    w = inputs.Workload(f"n{n}", 1, 2, 128, [n, 300], [0.5, 0.5], p=0.7, seed=300 + n)
+    kp, kr, v = [t.cuda() for t in inputs.make_tensors(w, device="cpu")]
+    shape = B.Shape(1, 2, 128, 48, w.seqlens)
+    phi = inputs.make_sketch_matrix(128, 48, 3)
+    keep = _keep(B, w)
+    outs = H.run_compress(B, shape, kr, kr, v, phi, keep)
+    worst, _ = H.compare_all_units(shape, keep, outs, kr, kr, v, phi, what=w.name)
+    st = outs[4].cpu().numpy().reshape(2, 2)
+    s = outs[0].cpu().numpy()[:, :, :n]
+    if n < 48:
+        assert np.all(st[:, 0] == 2)
+        np.testing.assert_allclose(s, 1.0, rtol=1e-3)
+    else:
+        assert np.all(st[:, 0] == 0), st
+        if n == 48:
+            np.testing.assert_allclose(s, 1.0, rtol=1e-3)
+        else:
+            assert s.min() < 0.999 and abs(float(s[0, 0].sum()) - 48.0) < 0.05
+    assert np.all(st[:, 1] == 0)
+    print(f"n={n}: max rel score err {worst:.2e}")
 
 
 def test_nonfinite_input_sets_status_and_returns(B):

@@ -30,7 +30,8 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of the dominant kernels per head-token, from ncu captures of a smaller case of
 # the same kernels (see profiles/); bytes read + written per token of one (layer, head).
-NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN = {}
+# keyed by (workload, kernel); only a capture of that workload at its own retention ratio counts
+NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN = {("c3", "gram"): 257.1, ("c3", "score"): 260.7, ("c3", "compact"): 316.1}
 
 
 def parse_args():
@@ -45,7 +46,9 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (debugging)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--cpu-units", type=int, default=16, help="units in the CPU-baseline sample")
+    ap.add_argument("--cpu-units", type=int, default=None,
+                    help="units in the CPU-baseline sample (default 16; 4 per step for --impl reference)")
+    ap.add_argument("--no-extra", action="store_true", help="skip the other workloads, the attention term and the NLL pass")
     ap.add_argument("--fig1-n", type=int, default=None, help="with --fig1: only this context length")
     ap.add_argument("--nll", action="store_true",
                     help="time the NLL reduction of Section 3.5 on 8192 x 128256 bf16 logits instead of the headline")
@@ -130,7 +133,9 @@ def stage_bytes(w, keep, mode):
     lh = w.layers * w.heads
     tok = sum(w.seqlens); kept = sum(keep)
     return {
-        "sweep": lh * tok * (row + 4),          # the keys once from HBM (their second read is meant to hit L2) + scores
+        "gram": lh * tok * row,                 # the keys once (the few fp64 partial sums are not credited)
+        "factor": 0,
+        "score": lh * tok * (row + 4),
         "blend": 0,
         "select": lh * (tok * 4 + kept * 4),
         "compact": lh * kept * (4 * row + 4),
@@ -138,7 +143,10 @@ def stage_bytes(w, keep, mode):
 
 
 def run_reference(args):
-    """The oracle, as it stands, on the host cores: a bounded sample of the workload's units."""
+    """The oracle, as it stands, on the host cores: a bounded sample of the workload's units per step
+    (--cpu-units, default 4: about half a second per step at the headline workload)."""
+    if args.cpu_units is None:
+        args.cpu_units = 4
     import numpy as np
     import torch
     from paper_2507_08143_b200 import inputs
@@ -149,7 +157,7 @@ def run_reference(args):
     w = inputs.workload(args.workload, layers=args.layers)
     phi = inputs.make_sketch_matrix(w.d, w.m, w.seed).numpy()
     keep = [orc.keep_count(n, r) for n, r in zip(w.seqlens, w.ratios)]
-    sample = max(1, min(args.cpu_units, 4))
+    sample = max(1, args.cpu_units)
     units = [(0, h % w.heads, b % w.batch) for h, b in zip(range(sample), range(sample))]
     data = []
     for (l, h, b) in units:
@@ -162,7 +170,7 @@ def run_reference(args):
         for ks, kr, v, kk, n in data:
             orc.compress_unit(ks, kr, v, phi, kk)
 
-    for _ in range(min(args.warmup, 1)):
+    for _ in range(args.warmup):
         step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
@@ -175,7 +183,7 @@ def run_reference(args):
     desc = f"{len(data)} units of {w.name} per step ({head_tokens} head-tokens), scaled to {w.layers}x{w.heads} units per token"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "mode": args.mode, "layers": w.layers, "kv_heads": w.heads, "d": w.d,
                    "m": w.m, "seqlens": w.seqlens if w.batch <= 4 else f"{w.batch} sequences"},
@@ -186,6 +194,8 @@ def run_reference(args):
 
 def cpu_baseline(args, w, keep, phi):
     import torch
+    if args.cpu_units is None:
+        args.cpu_units = 16
     from paper_2507_08143_b200 import inputs
     from oracle import compactor_oracle as orc
     sample = max(1, args.cpu_units)
@@ -309,6 +319,107 @@ def run_nll(args):
                               "mean_nll": float(out.cpu()[0])}}))
 
 
+def time_workload(B, inputs, torch, name, mode, steps, warmup):
+    """One workload through the fused call: ms per step, stage times, fraction of the HBM roofline."""
+    w = inputs.workload(name)
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    keep = [B.keep_count(n, r) for n, r in zip(w.seqlens, w.ratios)]
+    phi_d = inputs.make_sketch_matrix(w.d, w.m, w.seed).cuda()
+    kp, kr, v = inputs.make_tensors(w, device="cuda", want_pre=(mode == "paper"))
+    k_score = kp if mode == "paper" else kr
+    total_keep = sum(keep)
+    idx = torch.empty(w.layers, w.heads, total_keep, dtype=torch.int32, device="cuda")
+    k_out = torch.empty(w.layers, w.heads, total_keep, w.d, dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+    status = torch.zeros(w.units, dtype=torch.int32, device="cuda")
+    ws = B.alloc_workspace(shape)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")           # larger than L2
+    small = w.layers * w.heads * w.total_tokens * w.d * 2 < (512 << 20)          # inputs near the L2 size: flush between steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(B.N_STAGE_EVENTS)] for _ in range(steps)]
+    for es in ev:
+        for e in es:
+            e.record()
+    for _ in range(max(warmup, 3)):
+        B.compress(shape, k_score, kr, v, phi_d, keep, idx, k_out, v_out, ws, status=status)
+    torch.cuda.synchronize()
+    for es in ev:
+        if small:
+            flush.zero_()
+        B.compress_profiled(shape, k_score, kr, v, phi_d, keep, idx, k_out, v_out, ws, es, status=status)
+    torch.cuda.synchronize()
+    assert int(status.max().item()) == 0
+    ms = statistics.median(es[0].elapsed_time(es[-1]) for es in ev)
+    stage_ms = {nm: statistics.median(es[j].elapsed_time(es[j + 1]) for es in ev) for j, nm in enumerate(B.STAGE_NAMES)}
+    peak, _ = measured_peak()
+    b_alg = algorithmic_bytes(w, keep, mode)
+    gbs = b_alg / (ms * 1e-3) / 1e9
+    del kp, kr, v, idx, k_out, v_out, ws, flush
+    torch.cuda.empty_cache()
+    return {"workload": w.name, "mode": mode, "units": w.units, "tokens": w.total_tokens, "ms_per_step": round(ms, 4),
+            "tokens_per_s": round(w.total_tokens / (ms * 1e-3)), "stage_ms": {k: round(t, 4) for k, t in stage_ms.items()},
+            "path_roofline": {"algorithmic_bytes_per_step": b_alg, "achieved": round(gbs, 1), "frac": round(gbs / peak, 4)},
+            "l2": "flushed before every step" if small else "inputs exceed L2"}
+
+
+def extra_measurements(args, B, inputs, torch):
+    """The other benchmark workloads, the attention term, the full method and the NLL pass: a few timed
+    steps each (medians of CUDA-event times), reported beside the headline."""
+    out = {"other_workloads": {}}
+    steps = 5
+    for key, name, mode in (("c1", "c1", "aliased"), ("c2", "c2", "aliased"), ("c4", "c4", "aliased"), ("c3-paper", "c3", "paper")):
+        out["other_workloads"][key] = time_workload(B, inputs, torch, name, mode, steps, 3)
+    # the paper's Fig. 1 shape at n = 131072: one layer, 8 KV heads x 4 query heads, batch 1
+    n, G = 131072, 4
+    w = inputs.Workload("fig1-n131072", 1, 8, 128, [n], [0.3], p=0.7, n_out=4, theta=5e5, seed=100)
+    _, kr, v = inputs.make_tensors(w, device="cuda", want_pre=False)
+    q = inputs.make_queries(w, G, device="cuda")
+    shape = B.Shape(1, 8, 128, 48, [n])
+    keep = [B.keep_count(n, 0.3)]
+    phi = inputs.make_sketch_matrix(128, 48, 0).cuda()
+    attn = torch.empty(1, 8, n, dtype=torch.float32, device="cuda")
+    ws = B.alloc_workspace(shape)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def timed(fn, iters=7):
+        for _ in range(3):
+            fn()
+        ts = []
+        for _ in range(iters):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts)
+
+    t_attn = timed(lambda: B.attention_scores(shape, q, kr, G, attn, ws, scale=128 ** -0.5, pool=7))
+    flops = 2.0 * 8 * G * n * 256 * 128                                  # Q K^T of every 256-token chunk
+    out["attention"] = {"shape": "1 layer x 8 KV heads x 4 query heads, n = 131072, chunk 256, pool 7", "ms": round(t_attn, 4),
+                        "qk_tflops": round(flops / (t_attn * 1e-3) / 1e12, 1)}
+    opt = B.options(selection=B.SELECT_ACROSS_HEADS, lam=0.3, q_per_kv=G, scale=128 ** -0.5, pool=7)
+    idx = torch.empty(1, 8 * keep[0], dtype=torch.int32, device="cuda")
+    offs = torch.empty(1, 1, 9, dtype=torch.int32, device="cuda")
+    ko = torch.empty(1, 8 * keep[0], 128, dtype=torch.bfloat16, device="cuda"); vo = torch.empty_like(ko)
+    wsf = torch.empty(B.compress_full_workspace_bytes(shape, opt), dtype=torch.uint8, device="cuda")
+    t_full = timed(lambda: B.compress_full(shape, opt, q, kr, kr, v, phi, keep, idx, ko, vo, wsf, head_offsets_out=offs))
+    out["full_method"] = {"shape": "as above, keep 30 %, lambda 0.3, m 48, selection across heads; one compactor_compress_full call",
+                          "ms": round(t_full, 4),
+                          "paper_h100_full_score_ms": FIG1_PAPER_FULL_MS_H100[n],
+                          "note": "the paper's figure is the scoring time alone on an H100 80GB (context, not a target)"}
+    del kr, v, q, attn, ws, idx, ko, vo, wsf
+    torch.cuda.empty_cache()
+    rows, vocab = 8192, 128256
+    g = torch.Generator(device="cuda"); g.manual_seed(7)
+    logits = (torch.randn(rows, vocab, device="cuda", generator=g) * 4).to(torch.bfloat16)
+    targets = torch.randint(0, vocab, (rows,), device="cuda", generator=g, dtype=torch.int32)
+    row_nll = torch.empty(rows, dtype=torch.float32, device="cuda")
+    res = torch.empty(1, dtype=torch.float64, device="cuda")
+    t_nll = timed(lambda: B.nll(logits, targets, [rows], row_nll, res))
+    peak, _ = measured_peak()
+    gbs = rows * vocab * 2 / t_nll / 1e6
+    out["nll"] = {"rows": rows, "vocab": vocab, "dtype": "bf16", "ms": round(t_nll, 4), "GB/s": round(gbs, 1), "frac": round(gbs / peak, 4)}
+    return out
+
+
 def main():
     args = parse_args()
     if args.nll:
@@ -397,7 +508,7 @@ def main():
     dominant = max(stage_ms, key=stage_ms.get)
     peak, peak_kind = measured_peak()
     achieved = sb[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN.get(dominant)
+    traffic = NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN.get((args.workload, dominant)) if args.layers is None else None
     if traffic is not None:
         traffic = traffic * L * Hh * w.total_tokens
     b_alg = algorithmic_bytes(w, keep, args.mode)
@@ -413,7 +524,7 @@ def main():
                    "keep": keep if w.batch <= 4 else total_keep, "units_per_gpu": w.units,
                    "l2": "inputs (GBs per step) far exceed the 126 MB L2; no flush needed"},
         "head_tokens_per_s": value * L * Hh,
-        "gpu_launches": 4 * args.steps,
+        "gpu_launches": 7 * args.steps,       # table upload, Gram pass, projection, Cholesky, scoring pass, selection, compaction
         "stage_ms": {k: round(t, 4) for k, t in stage_ms.items()},
         "roofline": {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
@@ -427,6 +538,10 @@ def main():
         result["e2e"] = e2e(args, B, w, shape, keep, phi_d, k_score, kr, v, dist, world)
     if rank == 0 and world == 1 and not args.no_cpu:
         result["cpu_baseline"] = cpu_baseline(args, w, keep, phi)
+    if rank == 0 and world == 1 and not args.no_extra:
+        del kp, kr, v, k_score, idx, k_out, v_out, ws
+        torch.cuda.empty_cache()
+        result.update(extra_measurements(args, B, inputs, torch))
     if rank == 0:
         print(json.dumps(result))
     if dist is not None:

@@ -234,11 +234,11 @@ int compactor_compress(const compactor_shape* shape, compactor_mat k_score, comp
  * compactor_compress with stage markers, for measurement (the paper reports one wall-clock
  * number per context length, Fig. 1; this splits ours by stage).  stage_events is a HOST array of
  * n_events cudaEvent_t handles created by the caller (NULL entries are skipped).  They are
- * recorded on the stream: [0] before the scoring sweep (Gram pass, factorisation, scoring pass),
- * [1] after it, [2] after the blend (recorded even when there is none), [3] after selection,
- * [4] after compaction.  Results are identical to compactor_compress.
+ * recorded on the stream: [0] before the first kernel, [1] after the Gram pass, [2] after the
+ * factorisation, [3] after the scoring pass, [4] after the blend (recorded even when there is
+ * none), [5] after selection, [6] after compaction.  Results are identical to compactor_compress.
  */
-#define COMPACTOR_N_STAGE_EVENTS 5
+#define COMPACTOR_N_STAGE_EVENTS 7
 int compactor_compress_profiled(const compactor_shape* shape, compactor_mat k_score, compactor_mat k_cache,
                                 compactor_mat v_cache, const float* phi, const float* attn_scores,
                                 float lambda, const int32_t* keep_counts,
@@ -301,6 +301,51 @@ int compactor_compact_across_heads(const compactor_shape* shape, compactor_mat k
                                    const int32_t* idx, const int32_t* head_offsets,
                                    const int32_t* keep_counts, void* k_out, void* v_out,
                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The paper's whole method in one call: attention term (Eq. 5) -> leverage scores (Algorithm 1)
+ * -> blend (Eq. 6) -> selection within each head or across the heads of a layer (Section 3.4) ->
+ * gather.  The experiments of Section 4 use chunk 256, lambda 0.3, m 48 and selection across heads.
+ *   options      HOST struct:
+ *     selection      COMPACTOR_SELECT_PER_HEAD or COMPACTOR_SELECT_ACROSS_HEADS.
+ *     factorization  COMPACTOR_FACTOR_CHOLESKY or COMPACTOR_FACTOR_EIG (with eig_floor), as in
+ *                    compactor_score_variant.
+ *     lambda         weight of the leverage term in Eq. 6 (ignored without an attention term).
+ *     q_per_kv       query heads per KV head; 0 = no attention term: the score is the leverage
+ *                    score alone and q is ignored.
+ *     chunk, scale, pool   as in compactor_attention_scores (chunk must be 256).
+ *   q            queries, bf16 [layers][heads * q_per_kv][total_tokens][d] (ignored if q_per_kv = 0).
+ *   k_score      keys scored by Algorithm 1 (the paper: before positional encoding);
+ *   k_cache      keys the attention term is taken against and the rows are gathered from (may be
+ *                the same tensor as k_score);  v_cache likewise for the values.
+ *   scores_out   device fp32 [layers][heads][total_tokens] or NULL: the final (blended) score.
+ *   idx_out, k_out, v_out
+ *                per-head selection: the layouts of compactor_select / compactor_compact;
+ *                across heads: those of compactor_select_across_heads / compactor_compact_across_heads.
+ *   head_offsets_out  device int32 [layers][batch][heads + 1]; across heads only (else may be NULL).
+ *   status       device int32 [layers*heads*batch] or NULL; cleared once, then collects the flags of
+ *                the attention and the scoring kernels.
+ * Workspace: compactor_compress_full_workspace_bytes(shape, options), 256-byte aligned.  Errors as for
+ * the calls it is made of; everything is checked before anything is enqueued.
+ */
+#define COMPACTOR_SELECT_PER_HEAD      0
+#define COMPACTOR_SELECT_ACROSS_HEADS  1
+typedef struct compactor_options {
+    int32_t selection;
+    int32_t factorization;
+    double  eig_floor;
+    float   lambda;
+    int32_t q_per_kv;
+    int32_t chunk;
+    float   scale;
+    int32_t pool;
+} compactor_options;
+size_t compactor_compress_full_workspace_bytes(const compactor_shape* shape, const compactor_options* options);
+int compactor_compress_full(const compactor_shape* shape, const compactor_options* options, compactor_mat q,
+                            compactor_mat k_score, compactor_mat k_cache, compactor_mat v_cache,
+                            const float* phi, const int32_t* keep_counts, float* scores_out,
+                            int32_t* idx_out, int32_t* head_offsets_out, void* k_out, void* v_out,
+                            int32_t* status, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * compactor_score for callers that cannot allocate device memory (the paper has no counterpart;

@@ -24,6 +24,11 @@ class CompactorShape(Structure):
                 ("batch", c_int32), ("cu_seqlens", POINTER(c_int32))]
 
 
+class CompactorOptions(Structure):
+    _fields_ = [("selection", c_int32), ("factorization", c_int32), ("eig_floor", c_double), ("lam", c_float),
+                ("q_per_kv", c_int32), ("chunk", c_int32), ("scale", c_float), ("pool", c_int32)]
+
+
 class CompactorError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -69,6 +74,11 @@ def _load() -> ctypes.CDLL:
                                                   c_void_p, c_size_t, c_void_p]
     lib.compactor_compact_across_heads.argtypes = [POINTER(CompactorShape), CompactorMat, CompactorMat, c_void_p, c_void_p,
                                                    POINTER(c_int32), c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.compactor_compress_full_workspace_bytes.restype = c_size_t
+    lib.compactor_compress_full_workspace_bytes.argtypes = [POINTER(CompactorShape), POINTER(CompactorOptions)]
+    lib.compactor_compress_full.argtypes = [POINTER(CompactorShape), POINTER(CompactorOptions), CompactorMat, CompactorMat,
+                                            CompactorMat, CompactorMat, c_void_p, POINTER(c_int32), c_void_p, c_void_p,
+                                            c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
     lib.compactor_wait_selftest.argtypes = [c_void_p, c_void_p]
     lib.compactor_builtin_scratch_bytes.restype = c_size_t
     lib.compactor_score_builtin_scratch.argtypes = [POINTER(CompactorShape), CompactorMat, c_void_p, c_void_p, c_float,
@@ -84,13 +94,15 @@ EXPORTS = ["compactor_version", "compactor_error_string", "compactor_make_sketch
            "compactor_compact", "compactor_compress", "compactor_compress_profiled",
            "compactor_builtin_scratch_bytes", "compactor_score_builtin_scratch", "compactor_attention_scores", "compactor_attention_scores_status", "compactor_wait_selftest",
            "compactor_across_heads_workspace_bytes", "compactor_select_across_heads", "compactor_compact_across_heads",
-           "compactor_score_variant", "compactor_nll"]
+           "compactor_score_variant", "compactor_nll", "compactor_compress_full_workspace_bytes", "compactor_compress_full"]
 
 FACTOR_CHOLESKY = 0
 FACTOR_EIG = 1
+SELECT_PER_HEAD = 0
+SELECT_ACROSS_HEADS = 1
 
-N_STAGE_EVENTS = 5
-STAGE_NAMES = ["sweep", "blend", "select", "compact"]
+N_STAGE_EVENTS = 7
+STAGE_NAMES = ["gram", "factor", "score", "blend", "select", "compact"]
 
 
 def version() -> int:
@@ -299,6 +311,28 @@ def compact_across_heads(shape: Shape, k_cache: torch.Tensor, v_cache: torch.Ten
     _check(LIB.compactor_compact_across_heads(byref(shape.c), mat(k_cache), mat(v_cache), _ptr(idx), _ptr(head_offsets),
                                               _keep_array(keep_counts), _ptr(k_out), _ptr(v_out), _ptr(workspace),
                                               workspace.numel(), _stream()), "compactor_compact_across_heads")
+
+
+def options(selection: int = SELECT_PER_HEAD, factorization: int = FACTOR_CHOLESKY, eig_floor: float = 1e-6,
+            lam: float = 0.3, q_per_kv: int = 0, chunk: int = 256, scale: float = 128 ** -0.5, pool: int = 1) -> CompactorOptions:
+    return CompactorOptions(selection, factorization, eig_floor, lam, q_per_kv, chunk, scale, pool)
+
+
+def compress_full_workspace_bytes(shape: Shape, opt: CompactorOptions) -> int:
+    return int(LIB.compactor_compress_full_workspace_bytes(byref(shape.c), byref(opt)))
+
+
+def compress_full(shape: Shape, opt: CompactorOptions, q: Optional[torch.Tensor], k_score: torch.Tensor,
+                  k_cache: torch.Tensor, v_cache: torch.Tensor, phi: torch.Tensor, keep_counts: Sequence[int],
+                  idx_out: torch.Tensor, k_out: torch.Tensor, v_out: torch.Tensor, workspace: torch.Tensor,
+                  head_offsets_out: Optional[torch.Tensor] = None, scores_out: Optional[torch.Tensor] = None,
+                  status: Optional[torch.Tensor] = None) -> None:
+    """The paper's whole method in one call (attention term, leverage scores, blend, selection, gather)."""
+    qm = mat(q) if q is not None else CompactorMat(None, 0, 0, 0)
+    _check(LIB.compactor_compress_full(byref(shape.c), byref(opt), qm, mat(k_score), mat(k_cache), mat(v_cache), _ptr(phi),
+                                       _keep_array(keep_counts), _ptr(scores_out), _ptr(idx_out), _ptr(head_offsets_out),
+                                       _ptr(k_out), _ptr(v_out), _ptr(status), _ptr(workspace), workspace.numel(),
+                                       _stream()), "compactor_compress_full")
 
 
 def wait_selftest() -> int:

@@ -288,9 +288,9 @@ long long* g_sweep_profile = nullptr;     // instrumented builds only: per-CTA c
 
 int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn, float lambda,
                 float* scores, int32_t* status, char* ws, cudaStream_t stream, const Marks& mk = Marks(),
-                int factorization = COMPACTOR_FACTOR_CHOLESKY, double eig_floor = 0.0) {
+                int factorization = COMPACTOR_FACTOR_CHOLESKY, double eig_floor = 0.0, bool clear_status = true) {
     __nv_bfloat16* w = reinterpret_cast<__nv_bfloat16*>(ws + hp.off_w);
-    if (status != nullptr) CK(cudaMemsetAsync(status, 0, sizeof(int32_t) * hp.units, stream));
+    if (status != nullptr && clear_status) CK(cudaMemsetAsync(status, 0, sizeof(int32_t) * hp.units, stream));
     if (hp.fused) {
         // one persistent kernel: Gram pieces, factorisation and scoring pieces from a common work queue
         if (factorization != COMPACTOR_FACTOR_CHOLESKY) return COMPACTOR_E_INVALID_ARGUMENT;
@@ -315,18 +315,22 @@ int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn,
 #endif
         CK(mk.mark(0, stream));
         CK(launch_sweep(a, sm_count() < kMaxCtas ? sm_count() : kMaxCtas, stream));
-        CK(mk.mark(1, stream));
+        CK(mk.mark(1, stream));                 // the one kernel does all three steps: the whole time shows as the first
+        CK(mk.mark(2, stream));
+        CK(mk.mark(3, stream));
     } else {
         double* partials = reinterpret_cast<double*>(ws + hp.off_partials);
         CK(mk.mark(0, stream));
         CK(launch_gram(hp.plan, k, partials, status, stream));
+        CK(mk.mark(1, stream));
         CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, status,
                          factorization, eig_floor, stream));
+        CK(mk.mark(2, stream));
         CK(launch_score(hp.plan, k, w, scores, status, stream));
-        CK(mk.mark(1, stream));
+        CK(mk.mark(3, stream));
     }
     if (attn != nullptr) CK(launch_blend(hp.plan, attn, lambda, scores, stream));
-    CK(mk.mark(2, stream));
+    CK(mk.mark(4, stream));
     return COMPACTOR_OK;
 }
 
@@ -493,11 +497,11 @@ static int compress_impl(const compactor_shape* shape, compactor_mat k_score, co
     int rc = run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores, status, ws, st, mk);
     if (rc != COMPACTOR_OK) return rc;
     if (hp.plan.total_keep > 0) CK(launch_select(hp.plan, scores, idx_out, st));
-    CK(mk.mark(3, st));
+    CK(mk.mark(5, st));
     if (hp.plan.total_keep > 0)
         CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out,
                           static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
-    CK(mk.mark(4, st));
+    CK(mk.mark(6, st));
     return COMPACTOR_OK;
 }
 
@@ -706,6 +710,115 @@ extern "C" int compactor_compact_across_heads(const compactor_shape* shape, comp
     CK(upload_tables(&hp, workspace, st));
     CK(launch_compact_across(hp.plan, to_mat(k_cache), to_mat(v_cache), idx, head_offsets,
                              static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
+    return COMPACTOR_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The paper's whole method in one call (Sections 3.3, 3.4 and the set-up of Section 4).
+namespace {
+
+struct FullLayout {
+    size_t off_attn, off_attn_ws, off_across, total;
+    size_t main_bytes, attn_ws_bytes;
+};
+
+bool full_layout(const compactor_shape* shape, const compactor_options* opt, FullLayout* fl, int* err) {
+    if (opt == nullptr) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    HostPlan hp;
+    if (!make_plan(shape, &hp, err, false)) return false;
+    if (opt->selection != COMPACTOR_SELECT_PER_HEAD && opt->selection != COMPACTOR_SELECT_ACROSS_HEADS) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    if (opt->factorization != COMPACTOR_FACTOR_CHOLESKY && opt->factorization != COMPACTOR_FACTOR_EIG) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    if (opt->q_per_kv < 0) { *err = COMPACTOR_E_INVALID_ARGUMENT; return false; }
+    const size_t plane = sizeof(float) * (size_t)hp.plan.total_tokens * shape->layers * shape->heads;
+    fl->main_bytes = compactor_workspace_bytes(shape);
+    size_t off = align_up(fl->main_bytes);
+    fl->off_attn = off;
+    if (opt->q_per_kv > 0) off += align_up(plane);
+    fl->off_attn_ws = off;
+    fl->attn_ws_bytes = 0;
+    if (opt->q_per_kv > 0) {
+        fl->attn_ws_bytes = align_up(hp.off_w + (opt->pool > 1 ? plane : 0));
+        off += fl->attn_ws_bytes;
+    }
+    fl->off_across = off;
+    if (opt->selection == COMPACTOR_SELECT_ACROSS_HEADS)
+        off += align_up(sizeof(int32_t) * (size_t)shape->layers * shape->batch * (shape->heads + 1));
+    fl->total = off;
+    return true;
+}
+
+}  // namespace
+
+extern "C" size_t compactor_compress_full_workspace_bytes(const compactor_shape* shape, const compactor_options* options) {
+    FullLayout fl; int err = 0;
+    if (!full_layout(shape, options, &fl, &err)) return 0;
+    return fl.total;
+}
+
+extern "C" int compactor_compress_full(const compactor_shape* shape, const compactor_options* options, compactor_mat q,
+                                       compactor_mat k_score, compactor_mat k_cache, compactor_mat v_cache,
+                                       const float* phi, const int32_t* keep_counts, float* scores_out,
+                                       int32_t* idx_out, int32_t* head_offsets_out, void* k_out, void* v_out,
+                                       int32_t* status, void* workspace, size_t workspace_bytes, void* stream) {
+    FullLayout fl; int err = 0;
+    if (!full_layout(shape, options, &fl, &err)) return err;
+    const bool across = options->selection == COMPACTOR_SELECT_ACROSS_HEADS;
+    const bool with_attn = options->q_per_kv > 0;
+    const bool eig = options->factorization == COMPACTOR_FACTOR_EIG;
+    HostPlan hp;
+    if (!make_plan(shape, &hp, &err, !eig)) return err;
+    if (eig && (hp.plan.mp > 64 || !(options->eig_floor > 0.0) || !std::isfinite(options->eig_floor)))
+        return hp.plan.mp > 64 ? COMPACTOR_E_UNSUPPORTED : COMPACTOR_E_INVALID_ARGUMENT;
+    if (!mat_ok(k_score) || !mat_ok(k_cache) || !mat_ok(v_cache) || phi == nullptr || idx_out == nullptr ||
+        k_out == nullptr || v_out == nullptr || workspace == nullptr || !set_keep(shape, keep_counts, &hp))
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if ((((uintptr_t)k_out | (uintptr_t)v_out) & 15) != 0 || ((uintptr_t)workspace & 255) != 0)
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (across && (head_offsets_out == nullptr || (long long)shape->heads * hp.plan.total_keep > 0x7fffffffLL))
+        return COMPACTOR_E_INVALID_ARGUMENT;
+    if (across && shape->heads > 64) return COMPACTOR_E_UNSUPPORTED;
+    if (with_attn) {
+        if (options->chunk != 256) return COMPACTOR_E_UNSUPPORTED;
+        if (!mat_ok(q) || (long long)shape->heads * options->q_per_kv > 65535 || !(options->scale > 0.f) ||
+            !isfinite(options->scale) || options->pool < 1 || (options->pool & 1) == 0)
+            return COMPACTOR_E_INVALID_ARGUMENT;
+    }
+    if (workspace_bytes < fl.total) return COMPACTOR_E_WORKSPACE;
+    if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* ws = static_cast<char*>(workspace);
+    if (status != nullptr) CK(cudaMemsetAsync(status, 0, sizeof(int32_t) * hp.units, st));
+    float* attn = nullptr;
+    if (with_attn) {
+        // Eq. 5 on the cache's keys (the ones attention sees), into a plane of the workspace
+        HostPlan ap;
+        if (!make_plan(shape, &ap, &err, false)) return err;
+        replan_chunk(shape, &ap, options->chunk);
+        char* aws = ws + fl.off_attn_ws;
+        CK(upload_tables(&ap, aws, st));
+        attn = reinterpret_cast<float*>(ws + fl.off_attn);
+        CK(launch_attention(ap.plan, to_mat(q), to_mat(k_cache), options->q_per_kv, options->scale, options->pool,
+                            reinterpret_cast<float*>(aws + ap.off_w), attn, status, st));
+    }
+    float* scores = scores_out != nullptr ? scores_out : reinterpret_cast<float*>(ws + hp.off_scores);
+    CK(upload_tables(&hp, ws, st));
+    const int rc = run_scoring(hp, to_mat(k_score), phi, attn, options->lambda, scores, status, ws, st, Marks(),
+                               options->factorization, options->eig_floor, false);
+    if (rc != COMPACTOR_OK) return rc;
+    if (!across) {
+        if (hp.plan.total_keep > 0) {
+            CK(launch_select(hp.plan, scores, idx_out, st));
+            CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out,
+                              static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
+        }
+    } else {
+        uint32_t* thr = reinterpret_cast<uint32_t*>(ws + fl.off_across);
+        int* ties = reinterpret_cast<int*>(thr) + (size_t)shape->layers * shape->batch;
+        CK(launch_select_across(hp.plan, scores, idx_out, head_offsets_out, thr, ties, st));
+        if (hp.plan.total_keep > 0)
+            CK(launch_compact_across(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out, head_offsets_out,
+                                     static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
+    }
     return COMPACTOR_OK;
 }
 

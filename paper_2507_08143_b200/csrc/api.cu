@@ -51,7 +51,7 @@ struct HostPlan {
     int units;
     // fused sweep (Cholesky route, padded sketch of at most kFusedMaxMp columns)
     bool fused;
-    int slices, window, n_slots, max_pieces;
+    int slices, window, n_slots, max_pieces, resident16;
     long long total_pieces;
     size_t off_sched, sched_bytes, off_tbuf;
 };
@@ -146,7 +146,13 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
             const long v = strtol(e, nullptr, 10);
             if (v > 0 && v < 65536) window_bytes = (size_t)v << 20;
         }
-        const long long budget = (long long)(window_bytes / ((size_t)piece * kD * sizeof(__nv_bfloat16)));
+        hp->resident16 = 16;
+        if (const char* e = getenv("COMPACTOR_RESIDENT_16THS")) {       // tuning aid
+            const long v = strtol(e, nullptr, 10);
+            if (v >= 1 && v <= 16) hp->resident16 = (int)v;
+        }
+        // the window counts all pieces; only resident16 / 16 of them occupy L2 while they wait
+        const long long budget = (long long)(window_bytes / ((size_t)piece * kD * sizeof(__nv_bfloat16))) * 16 / hp->resident16;
         hp->window = (int)(budget > hp->max_pieces + 1 ? budget : hp->max_pieces + 1);
         layout_fused(hp);
         return true;
@@ -300,7 +306,7 @@ int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn,
         a.p = hp.plan; a.k = k;
         a.units = hp.units; a.total_pieces = (int)hp.total_pieces;
         a.total_ftasks = hp.plan.total_schunks * hp.plan.layers * hp.plan.heads;
-        a.window = hp.window; a.n_slots = hp.n_slots;
+        a.window = hp.window; a.n_slots = hp.n_slots; a.resident16 = hp.resident16;
         a.sched = reinterpret_cast<SweepSched*>(ws + hp.off_sched);
         a.gram_done = reinterpret_cast<int*>(ws + hp.off_sched + sizeof(SweepSched));
         a.slices_claimed = a.gram_done + hp.units;

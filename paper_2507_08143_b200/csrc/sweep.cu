@@ -14,11 +14,11 @@
 //                 G = Phi^T T, the Cholesky factor G = L L^T (pivots below 2^-20 of their
 //                 diagonal entry dropped: pseudo-inverse reading) and W = Phi L^-T.
 //
-// Scheduling.  One CTA per SM.  Warp 0 claims sweep pieces from global counters (a scoring piece
+// Scheduling.  One CTA per SM.  Warp 10 claims sweep pieces from global counters (a scoring piece
 // whose W is ready first, else the next Gram piece, which may run at most `window` pieces ahead of
-// the scoring front: that bounds the keys waiting in L2), streams their tiles through a ring of
-// shared memory with TMA and hands the piece to warp 1 (tcgen05.mma issue) and warps 2-9 (epilogue)
-// through a small queue.  Between pieces, and whenever they are idle, warps 2-9 claim factor tasks.
+// the scoring front: that bounds the keys waiting in L2) and hands them, through a small queue, to
+// warp 0 (which streams their tiles through a ring of shared memory with TMA), warp 1 (tcgen05.mma
+// issue) and warps 2-9 (epilogue).  Between pieces, and whenever they are idle, warps 2-9 claim factor tasks.
 // Claims are fetch-adds on per-unit counters (they never fail, so any number of CTAs can claim at once);
 // two 64-bit words hold, each, the prefix of units that are ready and the prefix that is used up, and
 // move by compare-and-swap once per unit.  Results do not depend on who runs what: every sum has a
@@ -42,8 +42,9 @@ constexpr int kStages = 4;
 constexpr int kFlushTiles = kGramFlushTokens / kTile;
 constexpr int kWorkerWarps = 8;
 constexpr int kWorkers = 32 * kWorkerWarps;
-constexpr int kThreads = 64 + kWorkers;    // warp 0: scheduler + TMA, warp 1: MMA, warps 2-9: epilogue and factor tasks
-constexpr int kQueue = 4;                  // pieces handed over inside a CTA
+constexpr int kThreads = 64 + kWorkers + 32;   // warp 0: TMA loads, warp 1: MMA, warps 2-9: epilogue and factor tasks, warp 10: scheduler
+constexpr int kSchedWarp = 2 + kWorkerWarps;
+constexpr int kQueue = 3;                  // pieces handed over inside a CTA (the scheduler claims at most this far ahead)
 constexpr uint32_t kTmemCols = 512;        // two Gram accumulators (128 columns each) + two scoring accumulators
 constexpr uint32_t kScoreCol0 = 256;
 constexpr int kOutTiles = 4;               // tiles whose scores leave together
@@ -162,12 +163,17 @@ __device__ void advance_w_prefix(const SweepArgs& a) {
 // 1 / sqrt(x) for a positive, finite, normal x: single-precision seed on x scaled by an even power of two
 // into [1, 4), one Newton step in double precision (relative error of the order of 1e-13: the factor it
 // scales stays consistent, L L^T = G to that accuracy, far below what the scores resolve), scaled back.
-// The chain of 48 dependent pivots is what the factorisation's latency consists of.
+// The chain of 48 dependent pivots is what the factorisation's latency consists of, so the conversions
+// between the two formats are done on the bit patterns (integer instructions have a fraction of the
+// latency of the conversion instructions).
 __device__ __forceinline__ double fast_rsqrt(double x) {
-    const int hi = __double2hiint(x);
+    const int hi = __double2hiint(x), lo = __double2loint(x);
     const int eh = (((hi >> 20) & 0x7ff) - 1023) >> 1;
-    const double xs = __hiloint2double(hi - ((2 * eh) << 20), __double2loint(x));
-    double y = (double)rsqrtf((float)xs);
+    const int hs = hi - ((2 * eh) << 20);                                   // x * 2^(-2 eh), in [1, 4)
+    const double xs = __hiloint2double(hs, lo);
+    const float xf = __int_as_float(((hs - ((1023 - 127) << 20)) << 3) | (int)((unsigned)lo >> 29));   // xs truncated to fp32
+    const int yb = __float_as_int(rsqrtf(xf));                              // in (0.5, 1]
+    double y = __hiloint2double((int)((unsigned)yb >> 3) + ((1023 - 127) << 20), yb << 29);
     const double h = 0.5 * xs;
     y = y * fma(-h * y, y, 1.5);
     return __hiloint2double(__double2hiint(y) - (eh << 20), __double2loint(y));
@@ -187,39 +193,41 @@ __device__ __noinline__ bool factor_panel(double* g, const double* diag0, double
 #pragma unroll
     for (int r = 0; r < kPanel; ++r)
 #pragma unroll
-        for (int c = 0; c <= r; ++c) dd[r][c] = (j0 + r < j1) ? g[(j0 + c) * LD + j0 + r] : 0.0;
+        for (int c = 0; c <= r; ++c) {               // loads are unconditional (they then travel together); masked afterwards
+            const double v = g[(j0 + c) * LD + j0 + r];
+            dd[r][c] = (j0 + r < j1) ? v : 0.0;
+        }
     const int r0 = lane, r1 = lane + 32;
     double a0[kPanel], a1[kPanel];
 #pragma unroll
     for (int c = 0; c < kPanel; ++c) {
-        a0[c] = (r0 < m && j0 + c < j1) ? g[(j0 + c) * LD + r0] : 0.0;
-        a1[c] = (r1 < m && j0 + c < j1) ? g[(j0 + c) * LD + r1] : 0.0;
+        const double v0 = g[(j0 + c) * LD + min(r0, LD - 1)], v1 = g[(j0 + c) * LD + min(r1, LD - 1)];
+        a0[c] = (r0 < m && j0 + c < j1) ? v0 : 0.0;
+        a1[c] = (r1 < m && j0 + c < j1) ? v1 : 0.0;
     }
+    // One straight line of code (no branches): the pivot chain, the solves of the lane's rows and the inverse of the
+    // diagonal block are independent chains of double-precision operations, and the compiler interleaves them.
+    // Columns past j1 (a short last panel) have a zero pivot: they are "dropped" (zero column) without being counted.
     double inv[kPanel];
     bool dropped = false;
 #pragma unroll
     for (int c = 0; c < kPanel; ++c) {
-        inv[c] = 0.0;
-        if (j0 + c < j1) {
-            const double piv = dd[c][c], d0 = diag0[j0 + c];
-            const bool keep = piv > kPivotFloor * d0 && d0 > 0.0;
-            if (keep) inv[c] = fast_rsqrt(piv); else dropped = true;
-            dd[c][c] = piv * inv[c];
+        const double piv = dd[c][c], d0 = diag0[min(j0 + c, LD - 1)];
+        const bool keep = piv > kPivotFloor * d0 && d0 > 0.0;
+        inv[c] = keep ? fast_rsqrt(keep ? piv : 1.0) : 0.0;
+        dropped = dropped || (!keep && j0 + c < j1);
+        dd[c][c] = piv * inv[c];
 #pragma unroll
-            for (int r = c + 1; r < kPanel; ++r) dd[r][c] *= inv[c];
+        for (int r = c + 1; r < kPanel; ++r) dd[r][c] *= inv[c];
 #pragma unroll
-            for (int r = c + 1; r < kPanel; ++r)
+        for (int r = c + 1; r < kPanel; ++r)
 #pragma unroll
-                for (int c2 = c + 1; c2 <= r; ++c2) dd[r][c2] = fma(-dd[r][c], dd[c2][c], dd[r][c2]);
-        }
-    }
-    // the lane's rows: l[c] = (a[c] - sum_{c' < c} l[c'] L_JJ[c][c']) / L_JJ[c][c]
-#pragma unroll
-    for (int c = 0; c < kPanel; ++c) {
+            for (int c2 = c + 1; c2 <= r; ++c2) dd[r][c2] = fma(-dd[r][c], dd[c2][c], dd[r][c2]);
+        // the lane's rows: l[c] = (a[c] - sum_{c' < c} l[c'] L_JJ[c][c']) / L_JJ[c][c], right-looking
         a0[c] *= inv[c];
         a1[c] *= inv[c];
 #pragma unroll
-        for (int c2 = c + 1; c2 < kPanel; ++c2) {          // independent updates: short dependency chains
+        for (int c2 = c + 1; c2 < kPanel; ++c2) {
             a0[c2] = fma(-a0[c], dd[c2][c], a0[c2]);
             a1[c2] = fma(-a1[c], dd[c2][c], a1[c2]);
         }
@@ -231,26 +239,25 @@ __device__ __noinline__ bool factor_panel(double* g, const double* diag0, double
             if (r1 < m && r1 >= j0 + c) g[(j0 + c) * LD + r1] = a1[c];
         }
     }
-    // X = L_JJ^-1 by forward substitution, column k: x[k] = inv[k], x[n] = -inv[n] sum_{t=k}^{n-1} L_JJ[n][t] x[t]
-    if (lane < kPanel) {
+    // X = L_JJ^-1 by forward substitution (every lane computes it, lane k stores column k):
+    // x[k] = inv[k], x[n] = -inv[n] sum_{t=k}^{n-1} L_JJ[n][t] x[t], right-looking
 #pragma unroll
-        for (int k = 0; k < kPanel; ++k) {
-            double x[kPanel];                             // x[n] first collects -sum_t L[n][t] x[t], then is scaled
+    for (int k = 0; k < kPanel; ++k) {
+        double x[kPanel];
 #pragma unroll
-            for (int n = k + 1; n < kPanel; ++n) x[n] = 0.0;
-            x[k] = inv[k];
+        for (int n = k + 1; n < kPanel; ++n) x[n] = 0.0;
+        x[k] = inv[k];
 #pragma unroll
-            for (int t = k; t < kPanel; ++t) {
-                if (t > k) x[t] *= inv[t];
+        for (int t = k; t < kPanel; ++t) {
+            if (t > k) x[t] *= inv[t];
 #pragma unroll
-                for (int n = t + 1; n < kPanel; ++n) x[n] = fma(-dd[n][t], x[t], x[n]);
-            }
-            if (lane == k) {
-                if (j0 + k < j1) inv_diag[j0 + k] = inv[k];
+            for (int n = t + 1; n < kPanel; ++n) x[n] = fma(-dd[n][t], x[t], x[n]);
+        }
+        if (lane == k) {
+            if (j0 + k < j1) inv_diag[j0 + k] = inv[k];
 #pragma unroll
-                for (int n = k + 1; n < kPanel; ++n)
-                    if (j0 + n < j1) g[(j0 + n) * LD + j0 + k] = x[n];
-            }
+            for (int n = k + 1; n < kPanel; ++n)
+                if (j0 + n < j1) g[(j0 + n) * LD + j0 + k] = x[n];
         }
     }
     return dropped;
@@ -289,7 +296,8 @@ __device__ __noinline__ void solve_w_tiles(const float* phi, const double* g, co
 #pragma unroll
         for (int sk = 0; sk < 2; ++sk) {
             const int k = 4 * sk + fk, n = fr;                                        // B[k][n] = X[n][k]
-            const double b = k < n ? g[(J * 8 + n) * LD + J * 8 + k] : (k == n ? inv_diag[J * 8 + n] : 0.0);
+            const double xg = g[(J * 8 + n) * LD + J * 8 + k], xd = inv_diag[J * 8 + n];    // both loaded, one chosen
+            const double b = k < n ? xg : (k == n ? xd : 0.0);
             const int src = (lane & ~3) | (2 * sk + (fk >> 1));
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) {
@@ -337,7 +345,7 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
             mbar_init(&s.sacc_full[i], 1); mbar_init(&s.sacc_empty[i], kWorkerWarps / 2);
             mbar_init(&s.w_full[i], 1);    mbar_init(&s.w_empty[i], 1);
         }
-        for (int i = 0; i < kQueue; ++i) { mbar_init(&s.tq_full[i], 1); mbar_init(&s.tq_empty[i], 1 + kWorkerWarps); }
+        for (int i = 0; i < kQueue; ++i) { mbar_init(&s.tq_full[i], 1); mbar_init(&s.tq_empty[i], 2 + kWorkerWarps); }
         s.abort = 0;
         fence_barrier_init();
     }
@@ -358,15 +366,13 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
     };
     int last_unit = 0;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ scheduler + TMA producer
+    if (warp == kSchedWarp) {
+        // ------------------------------------------------------------ scheduler: claims pieces, ahead of the loads
         if (lane == 0) {
-            uint64_t pol_first;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
-            int tq_count = 0, tile_count = 0, score_count = 0;
+            int tq_count = 0;
             for (;;) {
                 Task t;
-                t.type = kTaskExit; t.piece = 0; t.lh = 0; t.b = 0; t.tok_begin = 0; t.n_tok = 0; t.unit = last_unit; t.pad = 0;
+                t.type = kTaskExit; t.piece = 0; t.lh = 0; t.b = 0; t.tok_begin = 0; t.n_tok = 0; t.unit = 0; t.pad = 0;
                 const long long t0 = clock64();
                 for (;;) {
                     PROF_INC(1);
@@ -409,6 +415,20 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                 mbar_arrive(&s.tq_full[slot]);
                 ++tq_count;
                 if (t.type == kTaskExit) break;
+            }
+        }
+    } else if (warp == 0) {
+        // ------------------------------------------------------------ TMA loads of the claimed pieces
+        if (lane == 0) {
+            uint64_t pol_first;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_first));
+            int tq_count = 0, tile_count = 0, score_count = 0;
+            for (;;) {
+                const int slot = tq_count % kQueue;
+                wait(&s.tq_full[slot], (tq_count / kQueue) & 1);
+                const Task t = s.tq[slot];
+                ++tq_count;
+                if (t.type == kTaskExit) { mbar_arrive(&s.tq_empty[slot]); break; }
                 last_unit = t.unit;
                 const int layer = t.lh / p.heads, head = t.lh - layer * p.heads;
                 if (t.type == kTaskScore) {
@@ -425,6 +445,10 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                     }
                     ++score_count;
                 }
+                // Keys that are to wait in L2 for their second read are loaded with the default priority; the second
+                // read itself, and the first read of the pieces that are not meant to stay, leave first.
+                const int in_unit = t.piece - unit_piece_start(p, t.unit);
+                const bool stays = t.type == kTaskGram && ((in_unit * 5) & 15) < a.resident16;
                 const int n_tiles = (t.n_tok + kTile - 1) / kTile;
                 PROF_T(tp2);
                 for (int j = 0; j < n_tiles; ++j) {
@@ -434,7 +458,7 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                     if (*(volatile int*)&s.abort) continue;
                     mbar_arrive_expect_tx(&s.full[stage], kTileBytes);
                     const int tok = t.tok_begin + j * kTile;
-                    if (t.type == kTaskScore) {
+                    if (!stays) {
                         tma_load_4d_hint(s.tiles[stage], &kmap, &s.full[stage], 0, tok, head, layer, pol_first);
                         tma_load_4d_hint(s.tiles[stage] + kBoxBytes, &kmap, &s.full[stage], 64, tok, head, layer, pol_first);
                     } else {
@@ -443,6 +467,7 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                     }
                 }
                 PROF_ADD(t.type == kTaskGram ? 5 : 6, tp2);
+                mbar_arrive(&s.tq_empty[slot]);
             }
             // After a give-up some copies may still be on their way into this CTA's shared memory.
             if (*(volatile int*)&s.abort) {
@@ -463,7 +488,9 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
         int tq_count = 0, tile_count = 0, g_groups = 0, s_tiles = 0, score_count = 0;
         for (;;) {
             const int slot = tq_count % kQueue;
+            PROF_T(tm0);
             wait(&s.tq_full[slot], (tq_count / kQueue) & 1);
+            if (lane == 0) PROF_ADD(23, tm0);
             const Task t = s.tq[slot];
             ++tq_count;
             if (t.type == kTaskExit || *(volatile int*)&s.abort) {
@@ -478,8 +505,12 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                     const int stage = tile_count % kStages, round = tile_count / kStages;
                     ++tile_count;
                     const int gg = g_groups + j / kFlushTiles, in_group = j % kFlushTiles, buf = gg & 1;
+                    PROF_T(tm1);
                     if (in_group == 0 && gg >= 2) wait(&s.gacc_empty[buf], ((gg >> 1) - 1) & 1);
+                    if (lane == 0) PROF_ADD(24, tm1);
+                    PROF_T(tm2);
                     wait(&s.full[stage], round & 1);
+                    if (lane == 0) PROF_ADD(25, tm2);
                     tc_fence_after_sync();
                     const int valid = min(kTile, t.n_tok - j * kTile);
                     if (valid < kTile) {
@@ -510,14 +541,20 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                 g_groups += (n_tiles + kFlushTiles - 1) / kFlushTiles;
             } else {
                 const int wb = score_count & 1;
+                PROF_T(tm3);
                 wait(&s.w_full[wb], (score_count >> 1) & 1);
+                if (lane == 0) PROF_ADD(26, tm3);
                 for (int j = 0; j < n_tiles; ++j) {
                     const int stage = tile_count % kStages, round = tile_count / kStages;
                     ++tile_count;
                     const int buf = s_tiles & 1, use = s_tiles >> 1;
                     ++s_tiles;
+                    PROF_T(tm4);
                     wait(&s.full[stage], round & 1);
+                    if (lane == 0) PROF_ADD(27, tm4);
+                    PROF_T(tm5);
                     if (use > 0) wait(&s.sacc_empty[buf], (use - 1) & 1);
+                    if (lane == 0) PROF_ADD(28, tm5);
                     tc_fence_after_sync();
                     if (lane == 0) {
                         const uint32_t a_base = smem_u32(s.tiles[stage]);
@@ -540,7 +577,7 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
             __syncwarp();
             if (lane == 0) mbar_arrive(&s.tq_empty[slot]);
         }
-    } else {
+    } else if (warp >= 2 && warp < kSchedWarp) {
         // ------------------------------------------------------------ epilogue warps and factor tasks
         const int wtid = threadIdx.x - 64, wwarp = warp - 2;
         const int q = warp & 3;                          // TMEM lane quadrant this warp may read
@@ -888,16 +925,24 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                     }
                     workers_sync();
                     if (wtid == 0) PROF_ADD(18, tpan);
-                    const int nt = m - j1;                   // trailing block: rows and columns j1 .. m-1
-                    if (nt > 0) {
-                        for (int e = wtid; e < nt * nt; e += kWorkers) {
-                            const int c = e / nt, i = e - c * nt;      // consecutive threads: consecutive rows i of one column c
-                            if (c > i) continue;
-                            double v = g[(j1 + c) * LD + j1 + i];
+                    // trailing block, rows and columns j1 .. : A_ij -= L_i L_j^T by 8 x 8 tiles on fp64 mma (lower tiles only;
+                    // rows and columns past m hold zeros)
+                    const int nb = (MP - j1) / 8;
+                    if (j1 < m && nb > 0) {
+                        for (int tile = wwarp; tile < nb * (nb + 1) / 2; tile += kWorkerWarps) {
+                            int rem = tile, bi = 0;
+                            while (rem > bi) { rem -= bi + 1; ++bi; }
+                            const int bj = rem;
+                            double* cp = g + (j1 + 8 * bj + 2 * fk) * LD + j1 + 8 * bi + fr;      // fragment (row fr, columns 2 fk, + 1)
+                            double d[2] = {cp[0], cp[LD]};
 #pragma unroll
-                            for (int kk = 0; kk < kPanel; ++kk)
-                                if (j0 + kk < j1) v = fma(-g[(j0 + kk) * LD + j1 + i], g[(j0 + kk) * LD + j1 + c], v);
-                            g[(j1 + c) * LD + j1 + i] = v;
+                            for (int sk = 0; sk < 2; ++sk) {
+                                const double av = g[(j0 + 4 * sk + fk) * LD + j1 + 8 * bi + fr];   // L[j1 + 8 bi + fr][j0 + k]
+                                const double bv = g[(j0 + 4 * sk + fk) * LD + j1 + 8 * bj + fr];   // (L_j^T)[k][n] = L[j1 + 8 bj + n][j0 + k]
+                                mma_f64(d, -av, bv);
+                            }
+                            cp[0] = d[0];
+                            cp[LD] = d[1];
                         }
                         workers_sync();
                         if (wtid == 0) PROF_ADD(19, tpan);

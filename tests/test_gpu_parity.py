@@ -337,3 +337,20 @@ def test_repeated_calls_are_bit_identical(B):
     for other in runs[1:]:
         for a, b in zip(runs[0], other):
             assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("name", ["c0", "ragged"])
+def test_fused_sweep_kernel_gives_the_same_answers(B, name, monkeypatch):
+    # the one-kernel sweep (Gram pieces, factor tasks and scoring pieces from a common work queue) is switched on by an
+    # environment variable that the library reads at every call; it has to pass the same comparison with the oracle
+    monkeypatch.setenv("COMPACTOR_FUSED_SWEEP", "1")
+    if name == "c0":
+        w = inputs.workload("c0")
+    else:
+        w = inputs.Workload("fused-ragged", 2, 3, 128, [1000, 129, 0, 128, 127, 5300, 49, 300, 2049],
+                            [0.3, 0.5, 0.5, 0.2, 0.5, 0.3, 0.5, 1.0, 0.1], p=0.7, seed=12)
+    worst, band, outs = _run_workload(B, w, device="cpu")
+    st = outs[4].cpu().numpy().reshape(w.layers * w.heads, w.batch)
+    nonempty = [b for b, n in enumerate(w.seqlens) if n >= 48]
+    assert np.all(st[:, nonempty] == 0)
+    print(f"fused sweep, {w.name}: max rel score err {worst:.2e}")

@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--mode", default="aliased", choices=["aliased", "paper"],
                     help="aliased: score and gather the rotated keys; paper: score pre-rotation keys")
     ap.add_argument("--layers", type=int, default=None, help="override the layer count (debugging)")
+    ap.add_argument("--heads", type=int, default=None, help="override the KV-head count (slices of a few units for profiling)")
+    ap.add_argument("--flush-l2", action="store_true", help="write a 256 MiB buffer before every timed step (small slices)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-units", type=int, default=None,
@@ -446,6 +448,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     w = sharding.rank_workload(inputs.workload(args.workload, layers=args.layers), rank)
+    if args.heads is not None:
+        w.heads = args.heads
     shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
     keep = [B.keep_count(n, r) for n, r in zip(w.seqlens, w.ratios)]
     total_keep = sum(keep)
@@ -486,8 +490,11 @@ def main():
         time.sleep(0.3)
     t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if args.flush_l2 else None
     t_beg.record()
     for i in range(args.steps):
+        if flush is not None:
+            flush.zero_()
         step(events[i * B.N_STAGE_EVENTS:(i + 1) * B.N_STAGE_EVENTS])
     t_end.record()
     barrier()
@@ -508,7 +515,7 @@ def main():
     dominant = max(stage_ms, key=stage_ms.get)
     peak, peak_kind = measured_peak()
     achieved = sb[dominant] / (stage_ms[dominant] * 1e-3) / 1e9
-    traffic = NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN.get((args.workload, dominant)) if args.layers is None else None
+    traffic = NCU_TRAFFIC_BYTES_PER_HEAD_TOKEN.get((args.workload, dominant)) if args.layers is None and args.heads is None else None
     if traffic is not None:
         traffic = traffic * L * Hh * w.total_tokens
     b_alg = algorithmic_bytes(w, keep, args.mode)

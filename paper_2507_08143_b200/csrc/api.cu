@@ -39,10 +39,14 @@ int sm_count() {
 
 // The fused persistent sweep is switched on with COMPACTOR_FUSED_SWEEP=1 (it does not yet beat the
 // separate kernels; see sweep.cu).
-bool fused_sweep_enabled() {
+// 0: separate kernels; 1: one launch (Gram, factor and scoring pieces interleaved, keys meant to stay in L2);
+// 2: two launches of the same kernel (Gram pieces with the factor tasks hidden behind them, then scoring pieces).
+int fused_sweep_mode() {
     const char* e = getenv("COMPACTOR_FUSED_SWEEP");
-    return e != nullptr && e[0] == '1';
+    if (e == nullptr) return 0;
+    return e[0] == '1' ? 1 : (e[0] == '2' ? 2 : 0);
 }
+bool fused_sweep_enabled() { return fused_sweep_mode() != 0; }
 
 struct HostPlan {
     Plan plan;
@@ -152,7 +156,8 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
             if (v >= 1 && v <= 16) hp->resident16 = (int)v;
         }
         // the window counts all pieces; only resident16 / 16 of them occupy L2 while they wait
-        const long long budget = (long long)(window_bytes / ((size_t)piece * kD * sizeof(__nv_bfloat16))) * 16 / hp->resident16;
+        long long budget = (long long)(window_bytes / ((size_t)piece * kD * sizeof(__nv_bfloat16))) * 16 / hp->resident16;
+        if (fused_sweep_mode() == 2) budget = 1024;          // nothing waits in L2: the window only bounds the ring of partial sums
         hp->window = (int)(budget > hp->max_pieces + 1 ? budget : hp->max_pieces + 1);
         layout_fused(hp);
         return true;
@@ -319,11 +324,23 @@ int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn,
 #ifdef COMPACTOR_SWEEP_PROFILE
         a.prof = g_sweep_profile;
 #endif
+        const int ctas = sm_count() < kMaxCtas ? sm_count() : kMaxCtas;
         CK(mk.mark(0, stream));
-        CK(launch_sweep(a, sm_count() < kMaxCtas ? sm_count() : kMaxCtas, stream));
-        CK(mk.mark(1, stream));                 // the one kernel does all three steps: the whole time shows as the first
-        CK(mk.mark(2, stream));
-        CK(mk.mark(3, stream));
+        if (fused_sweep_mode() == 2) {
+            a.phase = 1;
+            CK(launch_sweep(a, ctas, stream));
+            CK(mk.mark(1, stream));             // Gram pieces with the factor tasks behind them
+            CK(mk.mark(2, stream));
+            a.phase = 2;
+            CK(launch_sweep(a, ctas, stream));
+            CK(mk.mark(3, stream));
+        } else {
+            a.phase = 0;
+            CK(launch_sweep(a, ctas, stream));
+            CK(mk.mark(1, stream));             // the one kernel does all three steps: the whole time shows as the first
+            CK(mk.mark(2, stream));
+            CK(mk.mark(3, stream));
+        }
     } else {
         double* partials = reinterpret_cast<double*>(ws + hp.off_partials);
         CK(mk.mark(0, stream));

@@ -58,6 +58,7 @@ struct SweepArgs {
     int total_ftasks;            // factor tasks: (layer, head) x sum over sequences of their row slices (p.cu_schunks, p.total_schunks)
     int window;                  // Gram pieces may run this far ahead of the scoring front
     int n_slots;                 // partial slots (>= window + CTAs); piece i uses slot i % n_slots
+    int phase;                   // 0: one launch does everything; 1: Gram pieces and factor tasks only; 2: scoring pieces only
     int resident16;              // sixteenths of a unit's pieces whose keys are meant to wait in L2 for the second read
     SweepSched* sched;
     int* gram_done;              // [units] finished Gram pieces

@@ -66,7 +66,7 @@ constexpr int kLdC = kD + 4;               // row stride (doubles) of the staged
 #endif
 
 enum { kTaskGram = 0, kTaskScore = 1, kTaskExit = 2 };
-enum { kActSweep = 0, kActFactor = 1 };
+enum { kActSweep = 0, kActFactor = 1, kActQuit = 2 };
 
 struct Task { int type, piece, lh, b, tok_begin, n_tok, unit, pad; };
 
@@ -379,9 +379,11 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                     if (*(volatile int*)&s.abort || *(volatile unsigned*)&a.sched->abort) break;
                     const unsigned long long ss = ld_acquire_u64(&a.sched->sstate);
                     const unsigned g = *(volatile unsigned*)&a.sched->gram_next;
-                    const int s_unit = (int)(ss >> 32), w_units = (int)(unsigned)ss;
+                    const int s_unit = (int)(ss >> 32);
+                    const int w_units = a.phase == 2 ? a.units : (int)(unsigned)ss;     // the scoring launch finds every W written
                     if (s_unit >= a.units) break;                      // every scoring piece has been claimed
-                    if (s_unit < w_units) {
+                    if (a.phase == 1 && (int)g >= total_pieces) break; // the Gram launch: every Gram piece has been claimed
+                    if (a.phase != 1 && s_unit < w_units) {
                         // a scoring piece of the first unit that still has some: claims are fetch-adds, they never fail
                         const int idx = atomicAdd(a.score_claimed + s_unit, 1);
                         if (idx < unit_pieces(p, s_unit)) {
@@ -396,7 +398,11 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                         atomicCAS(&a.sched->sstate, ss, ss + 1ull);
                         continue;
                     }
-                    if ((int)g < total_pieces && (int)g < unit_piece_start(p, s_unit) + a.window) {
+                    // Gram pieces may run `window` pieces ahead of the scoring front (of the units whose W is written, in
+                    // the launch that does no scoring): their partial sums live in a ring of slots
+                    const int front = a.phase == 1 ? w_units : s_unit;
+                    if (a.phase != 2 && (int)g < total_pieces &&
+                        (int)g < (front >= a.units ? total_pieces : unit_piece_start(p, front)) + a.window) {
                         const int idx = (int)atomicAdd(&a.sched->gram_next, 1u);
                         if (idx < total_pieces) { piece_to_task(p, idx, kTaskGram, &t); break; }
                         continue;
@@ -585,6 +591,7 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
         int tq_count = 0, g_groups = 0, s_tiles = 0, iter = 0;
         unsigned long long hint_fs = 0;
         bool have_hint = false;
+        bool draining = false;       // the Gram launch: no pieces left for this CTA, but factor tasks may still come
         for (;;) {
             // ---- the leader picks the next thing to do: a factor task that is ready, else the next piece of this CTA
             PROF_T(tw0);
@@ -595,7 +602,8 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                 const long long t0 = clock64();
                 for (;;) {
                     if (*(volatile int*)&s.abort) {
-                        // the producer stops claiming and hands over the exit task: wait for it (short, bounded)
+                        if (draining) { action = kActQuit; break; }
+                        // the scheduler stops claiming and hands over the exit task: wait for it (short, bounded)
                         if (mbar_try_wait(&s.tq_full[slot], qphase) || clock64() - t0 > kWaitLimitCycles) break;
                         continue;
                     }
@@ -614,7 +622,9 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
                         atomicCAS(&a.sched->fstate, fs, fs + (1ull << 32));     // all slices of that unit are taken: move on
                         continue;
                     }
-                    if (mbar_try_wait(&s.tq_full[slot], qphase)) break;
+                    if (draining) {
+                        if (f_unit >= a.units || *(volatile unsigned*)&a.sched->abort) { action = kActQuit; break; }
+                    } else if (mbar_try_wait(&s.tq_full[slot], qphase)) break;
                     if (!fresh) continue;                 // the hint was old: look again before sleeping
                     if (gunits < a.units &&
                         (int)ld_acquire_u32(reinterpret_cast<const unsigned*>(a.gram_done) + gunits) == unit_pieces(p, gunits)) {
@@ -635,11 +645,16 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
             if (wtid == 0) PROF_ADD(8, tw0);
             PROF_T(tw1);
 
+            if (action == kActQuit) break;
             if (action == kActSweep) {
                 const int slot = tq_count % kQueue;
                 const Task t = s.tq[slot];
                 ++tq_count;
-                if (t.type == kTaskExit) break;
+                if (t.type == kTaskExit) {
+                    if (a.phase != 1) break;
+                    draining = true;          // stay for the factor tasks of the units that are still being summed
+                    continue;
+                }
                 if (wtid == 0) { hint_fs = ld_relaxed_u64(&a.sched->fstate); have_hint = true; }
                 const int n_tiles = (t.n_tok + kTile - 1) / kTile;
                 if (t.type == kTaskGram) {

@@ -216,7 +216,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     size_t off = 0;
     hp->off_tables = off;   off += align_up(sizeof(int) * 4 * nb1);
     hp->off_w = off;        off += align_up(sizeof(__nv_bfloat16) * w_elems_per_unit(p.mp) * hp->units);
-    hp->off_gpart = off;    off += align_up(sizeof(double) * kFactorSlices * p.mp * p.mp * hp->units);
+    hp->off_gpart = off;    off += align_up(sizeof(double) * kD * p.mp * hp->units);             // T = C Phi per unit
     hp->off_partials = off; off += align_up(sizeof(double) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
     hp->off_scores = off;   off += align_up(sizeof(float) * (size_t)p.total_tokens * s->layers * s->heads);
     hp->total_bytes = off;
@@ -347,7 +347,7 @@ int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn,
         CK(launch_gram(hp.plan, k, partials, status, stream));
         CK(mk.mark(1, stream));
         CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, status,
-                         factorization, eig_floor, stream));
+                         factorization, eig_floor, sm_count(), stream));
         CK(mk.mark(2, stream));
         CK(launch_score(hp.plan, k, w, scores, status, stream));
         CK(mk.mark(3, stream));

@@ -14,7 +14,7 @@ constexpr int kMaxChunk = 65536;   // most tokens per block (one CTA of a stream
 constexpr int kMinChunk = 256;
 constexpr int kGramFlushTokens = 512;    // most tokens whose Gram matrix is summed in fp32 (tensor-core accumulators) before going to fp64
 constexpr int kGramElems = kD * kD;
-constexpr int kFactorSlices = 8;   // CTAs per unit that share the fp64 projection of the Gram matrix
+constexpr int kFactorSlices = 4;   // CTAs per unit that share the fp64 projection of the Gram matrix
 
 // Device-side view of one call: shapes plus the four prefix-sum tables that live at the start
 // of the workspace.  Passed to kernels by value.
@@ -88,8 +88,9 @@ __device__ __forceinline__ int find_segment(const int* __restrict__ table, int n
 // Kernel launchers (each defined next to its kernel).  All enqueue on `stream` and return the
 // launch status.
 cudaError_t launch_gram(const Plan& p, const Mat& k, double* partials, int* status, cudaStream_t stream);
-cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* g_partials,
-                          __nv_bfloat16* w, int* status, int factorization, double eig_floor, cudaStream_t stream);
+cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* t_buf,
+                          __nv_bfloat16* w, int* status, int factorization, double eig_floor, int sm_count,
+                          cudaStream_t stream);
 cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
                          cudaStream_t stream);
 cudaError_t launch_sweep(const SweepArgs& a, int sm_count, cudaStream_t stream);

@@ -1,27 +1,27 @@
 // Small factorisation (Algorithm 1, line 4, by the Cholesky route that Section 3.2 and
 // Appendix C allow), in two kernels, all fp64:
 //
-//   project_kernel   eight CTAs per unit, each owning 16 rows of C = sum of the unit's Gram
-//                    partials: T_r = C[rows,:] Phi and the partial projection
-//                    G_r = Phi[rows,:]^T T_r, so that G = Phi^T C Phi = sum_r G_r.  This is where
-//                    the fp64 FMAs are (1.1 M per unit); they run as fp64 mma.m8n8k4, spread over
-//                    the whole device.
-//   cholesky_kernel  one small CTA per unit (four fit on an SM, so all units of a large batch are
-//                    resident at once): G = sum_r G_r, G = L L^T in one warp (left-looking,
-//                    reciprocal square roots), then W = Phi L^-T with one thread per row of Phi
-//                    holding the row in registers, split into two bf16 terms.  The score of a key
-//                    row k_i is then || k_i W ||^2 (Algorithm 1, lines 5-6).
+//   project_kernel   four CTAs per unit, each owning 32 rows of C = sum of the unit's Gram
+//                    partials: T[rows,:] = C[rows,:] Phi on fp64 mma.m8n8k4 (this is where the
+//                    fp64 work is: 0.8 M multiply-adds per unit, spread over the whole device).
+//   cholesky_kernel  one small CTA per unit, several per SM: G = Phi^T T (fp64 mma), G = L L^T by
+//                    panels of eight columns (the 8 x 8 diagonal blocks are factored redundantly
+//                    by every lane of a warp, so no pivot has to travel), then W = Phi L^-T as a
+//                    blocked substitution on fp64 mma, split into two bf16 terms.  The score of a
+//                    key row k_i is then || k_i W ||^2 (Algorithm 1, lines 5-6).
 //
 // Rank handling: a pivot not larger than 2^-20 of its original diagonal entry (the fp32 noise
 // floor of the fp32 Gram runs) is treated as a direction of the null space and dropped;
 // with the remaining pivot set P, W = Phi[:, P] L_PP^-T, which equals the pseudo-inverse reading
 // o_i = k^_i G^+ k^_i^T whenever k^_i lies in the range of G.
 #include "common.cuh"
+#include "factor_math.cuh"
 
 namespace compactor {
 namespace {
 
-constexpr double kPivotFloor = 9.5367431640625e-07;   // 2^-20
+using namespace factor_math;
+
 // Sequences this short are near the sketch dimension, where G is close to singular and the fp32
 // rounding inside the Gram partials would dominate the scores; their Gram matrix is summed in
 // fp64 straight from the keys instead (the work is tiny).
@@ -34,43 +34,33 @@ constexpr int kProjThreads = 256;
 
 template <int MP>
 struct ProjectSmem {
-    static constexpr int kLd = MP + 8;     // row stride (doubles): four consecutive rows of 8 land in distinct banks
+    static constexpr int kLd = MP + 4;     // row stride (doubles): the four k-rows of a B fragment land in distinct banks
     double phi[kD * kLd];                  // Phi widened, [channel][column]
     double c[kD * kRows];                  // C[k][row0 + i] at [k * kRows + i]  (C is symmetric)
-    double t[kRows * kLd];                 // T_r
     double keys[kStageTokens * kD];
 };
 
 // Persistent: each CTA loads Phi once and then walks (unit, slice) items with a grid stride; the
 // global loads of the next item's partials are in flight while the current item is multiplied.
 template <int MP>
-__global__ void __launch_bounds__(kProjThreads)
+__global__ void __launch_bounds__(kProjThreads, 2)
 project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const float* __restrict__ phi,
-               double* __restrict__ g_partials, int n_items) {
+               double* __restrict__ t_buf, int n_items) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using Smem = ProjectSmem<MP>;
     Smem& s = *reinterpret_cast<Smem*>(smem_raw);
     constexpr int LD = Smem::kLd;
-    constexpr int kPer = kD * kRows / kProjThreads;     // 8 elements of the C slice per thread: e = tid + 256 q
-    constexpr int kInFlight = 4;                        // partials loaded ahead per item
+    constexpr int kPer = kD * kRows / kProjThreads;     // elements of the C slice per thread: e = tid + 256 q
+    constexpr int kInFlight = 2;                        // partials loaded ahead per item
+    constexpr int kWarps = kProjThreads / 32;
     const int m = p.m, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int fr = lane >> 2, fk = lane & 3;            // fragment coordinates: A[fr][fk], B[fk][fr], C[fr][2 fk, 2 fk + 1]
     constexpr int kNT = MP / 8;                         // 8-column tiles
 
-    {   // Phi, widened; all loads of a thread are issued before the first is used
-        constexpr int kPerThread = kD * MP / kProjThreads;
-        float v[kPerThread];
-#pragma unroll
-        for (int q = 0; q < kPerThread; ++q) {
-            const int i = tid + q * kProjThreads, row = i / MP, col = i % MP;
-            v[q] = (col < m) ? __ldg(phi + row * m + col) : 0.f;
-        }
-#pragma unroll
-        for (int q = 0; q < kPerThread; ++q) {
-            const int i = tid + q * kProjThreads;
-            s.phi[(i / MP) * LD + (i % MP)] = (double)v[q];
-        }
+    for (int i = tid; i < kD * MP; i += kProjThreads) {   // Phi, widened
+        const int row = i / MP, col = i - row * MP;
+        s.phi[row * LD + col] = (col < m) ? (double)__ldg(phi + row * m + col) : 0.0;
     }
 
     // Item bookkeeping and the look-ahead loads.
@@ -87,18 +77,29 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
     };
     double pre[kInFlight][kPer];
     auto prefetch = [&](const Item& it) {
+        const bool any = it.n_part > 0 && it.n_tok > kExactGramTokens;      // the same for the whole CTA
 #pragma unroll
         for (int u = 0; u < kInFlight; ++u)
 #pragma unroll
             for (int q = 0; q < kPer; ++q) {
                 const int e = tid + q * kProjThreads;
                 pre[u][q] = 0.0;
-                if (u < it.n_part && it.n_tok > kExactGramTokens) {
-                    // volatile: keeps the load here, ahead of the matrix products, instead of at its first use
-                    const double* src = it.part + (size_t)u * kGramElems + (e / kRows) * kD + it.slice * kRows + (e % kRows);
+                if (any) {
+                    // The loads are unconditional (partials past the last one re-read the last and are masked below).
+                    // volatile: keeps the load here, ahead of the matrix products, instead of at its first use.
+                    const int uu = u < it.n_part ? u : it.n_part - 1;
+                    const double* src = it.part + (size_t)uu * kGramElems + (e / kRows) * kD + it.slice * kRows + (e % kRows);
                     asm volatile("ld.global.cs.f64 %0, [%1];" : "=d"(pre[u][q]) : "l"(src));
                 }
             }
+        if (any) {
+#pragma unroll
+            for (int u = 0; u < kInFlight; ++u)
+                if (u >= it.n_part) {
+#pragma unroll
+                    for (int q = 0; q < kPer; ++q) pre[u][q] = 0.0;
+                }
+        }
     };
 
     int item = blockIdx.x;
@@ -106,7 +107,7 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
     if (item < n_items) { cur = decode(item); prefetch(cur); }
     for (; item < n_items; item += gridDim.x) {
         const int row0 = cur.slice * kRows;
-        // ---- the item's 16 columns of C (= 16 rows, by symmetry), summed over the partials ------
+        // ---- the item's 32 columns of C (= 32 rows, by symmetry), summed over the partials ------
         {
             double acc[kPer];
 #pragma unroll
@@ -122,16 +123,16 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
                         const int e = tid + q * kProjThreads;
                         acc[q] += __ldcs(cur.part + (size_t)pp * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
                     }
-                __syncthreads();                              // the previous item's products are done with c and t
+                __syncthreads();                              // the previous item's products are done with c
 #pragma unroll
                 for (int q = 0; q < kPer; ++q) s.c[tid + q * kProjThreads] = acc[q];
             } else {
                 // short sequence: fp64 Gram straight from the keys, C[:, rows] = K^T K[:, rows], as fp64 mma.m8n8k4
-                // over four tokens at a time (a warp owns four 8 x 8 tiles of the 128 x 16 slice)
+                // over four tokens at a time
                 const int layer = cur.lh / p.heads, head = cur.lh % p.heads;
                 const __nv_bfloat16* kbase = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
                                              (long long)p.cu_seqlens[cur.b] * kmat.stride_token;
-                constexpr int kTilesPerWarp = (kD / 8) * (kRows / 8) / (kProjThreads / 32);
+                constexpr int kTilesPerWarp = (kD / 8) * (kRows / 8) / kWarps;
                 double d[kTilesPerWarp][2];
 #pragma unroll
                 for (int j = 0; j < kTilesPerWarp; ++j) d[j][0] = d[j][1] = 0.0;
@@ -141,11 +142,12 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
                 auto fetch = [&](int t0) {                    // missing tokens of the last stage are zeros
 #pragma unroll
                     for (int u = 0; u < kLoads; ++u) {
-                        const int i = tid + u * kProjThreads, t = t0 + i / kD;
-                        nxt[u] = t < cur.n_tok ? __bfloat162float(kbase[(long long)t * kmat.stride_token + (i % kD)]) : 0.f;
+                        const int i = tid + u * kProjThreads, t = min(t0 + i / kD, cur.n_tok - 1);
+                        nxt[u] = __bfloat162float(kbase[(long long)t * kmat.stride_token + (i % kD)]);
+                        if (t0 + i / kD >= cur.n_tok) nxt[u] = 0.f;
                     }
                 };
-                fetch(0);
+                if (cur.n_tok > 0) fetch(0);
                 for (int t0 = 0; t0 < cur.n_tok; t0 += kStageTokens) {
                     __syncthreads();
 #pragma unroll
@@ -157,19 +159,16 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
                         const double* krow = s.keys + (ks * 4 + fk) * kD;          // token ks*4 + fk of the stage
 #pragma unroll
                         for (int j = 0; j < kTilesPerWarp; ++j) {
-                            const int tile = warp + j * (kProjThreads / 32);
+                            const int tile = warp + j * kWarps;
                             const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
-                            const double a = krow[mt * 8 + fr];                     // A[channel][token]
-                            const double bv = krow[row0 + nt8 * 8 + fr];            // B[token][channel of the slice]
-                            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                                         : "+d"(d[j][0]), "+d"(d[j][1]) : "d"(a), "d"(bv));
+                            mma_f64(d[j], krow[mt * 8 + fr], krow[row0 + nt8 * 8 + fr]);   // A[channel][token], B[token][channel of the slice]
                         }
                     }
                 }
-                __syncthreads();                              // the previous item's products are done with c and t
+                __syncthreads();                              // the previous item's products are done with c
 #pragma unroll
                 for (int j = 0; j < kTilesPerWarp; ++j) {
-                    const int tile = warp + j * (kProjThreads / 32);
+                    const int tile = warp + j * kWarps;
                     const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
                     s.c[(mt * 8 + fr) * kRows + nt8 * 8 + 2 * fk] = d[j][0];
                     s.c[(mt * 8 + fr) * kRows + nt8 * 8 + 2 * fk + 1] = d[j][1];
@@ -182,10 +181,10 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
         const Item done = cur;
         if (item + (int)gridDim.x < n_items) { cur = decode(item + gridDim.x); prefetch(cur); }
 
-        // Both products run as fp64 mma.m8n8k4 (a warp-wide instruction does 256 FMAs for two 8-byte
-        // shared-memory loads per lane); the contraction is cut into four independent chains.
-        // ---- T_r (16 x MP) = C[rows,:] (16 x 128) Phi (128 x MP) --------------------------------
-        for (int tile = warp; tile < 2 * kNT; tile += kProjThreads / 32) {
+        // ---- T[rows] (32 x MP) = C[rows,:] (32 x 128) Phi (128 x MP): a warp-wide fp64 mma does 256 multiply-adds for two
+        // 8-byte shared-memory loads per lane; the contraction is cut into four independent chains --------------------
+        double* t_rows = t_buf + ((size_t)done.unit * kD + row0) * MP;
+        for (int tile = warp; tile < (kRows / 8) * kNT; tile += kWarps) {
             const int mt = tile / kNT, nt = tile % kNT;
             double d[4][2];
 #pragma unroll
@@ -195,154 +194,59 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     const int k = g * (kD / 4) + k0 + fk;
-                    const double a = s.c[k * kRows + mt * 8 + fr];            // A[row][k] = C[k][row0 + row]
-                    const double bv = s.phi[k * LD + nt * 8 + fr];            // B[k][col]
-                    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                                 : "+d"(d[g][0]), "+d"(d[g][1]) : "d"(a), "d"(bv));
+                    mma_f64(d[g], s.c[k * kRows + mt * 8 + fr], s.phi[k * LD + nt * 8 + fr]);   // A[row][k] = C[k][row0 + row], B[k][col]
                 }
             }
-            s.t[(mt * 8 + fr) * LD + nt * 8 + 2 * fk] = (d[0][0] + d[1][0]) + (d[2][0] + d[3][0]);
-            s.t[(mt * 8 + fr) * LD + nt * 8 + 2 * fk + 1] = (d[0][1] + d[1][1]) + (d[2][1] + d[3][1]);
-        }
-        __syncthreads();
-
-        // ---- G_r (MP x MP) = Phi[rows,:]^T (MP x 16) T_r (16 x MP) ------------------------------
-        {
-            double* out = g_partials + ((size_t)done.unit * kSlices + done.slice) * (MP * MP);
-            for (int tile = warp; tile < kNT * kNT; tile += kProjThreads / 32) {
-                const int mt = tile / kNT, nt = tile % kNT;
-                double d[4][2];
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {                 // four k-steps of 4 rows each, independent
-                    d[g][0] = d[g][1] = 0.0;
-                    const double a = s.phi[(row0 + g * 4 + fk) * LD + mt * 8 + fr];   // A[a][i] = Phi[row0 + i][a]
-                    const double bv = s.t[(g * 4 + fk) * LD + nt * 8 + fr];           // B[i][b] = T_r[i][b]
-                    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                                 : "+d"(d[g][0]), "+d"(d[g][1]) : "d"(a), "d"(bv));
-                }
-                *reinterpret_cast<double2*>(out + (mt * 8 + fr) * MP + nt * 8 + 2 * fk) =
-                    make_double2((d[0][0] + d[1][0]) + (d[2][0] + d[3][0]), (d[0][1] + d[1][1]) + (d[2][1] + d[3][1]));
-            }
+            __stcg(reinterpret_cast<double2*>(t_rows + (size_t)(mt * 8 + fr) * MP + nt * 8 + 2 * fk),
+                   make_double2((d[0][0] + d[1][0]) + (d[2][0] + d[3][0]), (d[0][1] + d[1][1]) + (d[2][1] + d[3][1])));
         }
     }
 }
 
-constexpr int kCholThreads = kD;           // one thread per row of Phi
-
-// Columns of W that a thread holds in registers at a time; a wider sketch is solved block by block,
-// with the finished blocks parked in shared memory (fp64) for the updates of the later ones.
-template <int MP> struct WBlock { static constexpr int value = MP <= 64 ? MP : 64; };
+constexpr int kCholThreads = 128;
+constexpr int kCholWarps = kCholThreads / 32;
 
 template <int MP>
 struct CholSmem {
-    static constexpr int kParked = MP - WBlock<MP>::value;      // columns of W kept for later blocks
-    double g[MP * (MP + 1)];     // G, then L in the lower triangle; odd row stride spreads a column over the banks
-    double inv_diag[MP];         // 1 / L_jj of kept columns, 0 for dropped or padded ones
-    double parked[kParked > 0 ? kParked * kCholThreads : 1];
+    float phi[kD * MP];                    // the sketch, zero in the padded columns
+    union {
+        double t[kTRows * (MP + 4)];       // staged rows of T while G is formed
+        double g[MP * MP];                 // G, then L by columns (and the inverses of its diagonal blocks)
+    } u;
+    double diag0[MP], inv_diag[MP];
     int flags;
 };
 
 template <int MP>
 __global__ void __launch_bounds__(kCholThreads, MP <= 48 ? 4 : (MP <= 64 ? 2 : 1))
-cholesky_kernel(Plan p, const double* __restrict__ g_partials, const float* __restrict__ phi,
+cholesky_kernel(Plan p, const double* __restrict__ t_buf, const float* __restrict__ phi,
                 __nv_bfloat16* __restrict__ w_out, int* __restrict__ status) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     CholSmem<MP>& s = *reinterpret_cast<CholSmem<MP>*>(chol_smem_raw);
-    constexpr int LD = MP + 1;
-    constexpr int kH = (MP + 31) / 32;          // rows of a column per lane
     const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = p.m;
 
     if (tid == 0) s.flags = 0;
+    for (int i = tid; i < kD * MP; i += kCholThreads) {
+        const int row = i / MP, col = i - row * MP;
+        s.phi[i] = col < m ? __ldg(phi + row * m + col) : 0.f;
+    }
     if (tid < MP) s.inv_diag[tid] = 0.0;
     __syncthreads();
-    {   // G = sum of the partial projections
-        const double* src = g_partials + (size_t)unit * kSlices * (MP * MP);
-        bool finite = true;
-        for (int e = tid; e < MP * MP; e += kCholThreads) {
-            double v = 0.0;
-#pragma unroll
-            for (int r = 0; r < kSlices; ++r) v += src[(size_t)r * (MP * MP) + e];
-            s.g[(e / MP) * LD + (e % MP)] = v;
-            finite = finite && isfinite(v);
-        }
-        if (!finite) atomicOr(&s.flags, COMPACTOR_STATUS_NONFINITE);
-    }
+    auto sync = [] { __syncthreads(); };
+    const bool finite = gram_of_sketch<MP, kCholWarps>(t_buf + (size_t)unit * kD * MP, s.phi, s.u.g, s.u.t, tid, sync);
+    if (!finite) atomicOr(&s.flags, COMPACTOR_STATUS_NONFINITE);
     __syncthreads();
     const bool bad = (s.flags & COMPACTOR_STATUS_NONFINITE) != 0;
-
-    // ---- Cholesky, left-looking, one warp: at column j lane l owns rows j+l, j+l+32, ... ---------
-    if (warp == 0 && !bad) {
-        int rank_flag = 0;
-        for (int j = 0; j < m; ++j) {
-            double v[kH];
-#pragma unroll
-            for (int h = 0; h < kH; ++h) {
-                const int i = j + lane + 32 * h;
-                double a0 = 0.0, a1 = 0.0;
-                if (i < m) {
-                    a0 = s.g[i * LD + j];
-                    int c = 0;
-                    for (; c + 2 <= j; c += 2) {
-                        a0 = fma(-s.g[i * LD + c], s.g[j * LD + c], a0);
-                        a1 = fma(-s.g[i * LD + c + 1], s.g[j * LD + c + 1], a1);
-                    }
-                    if (c < j) a0 = fma(-s.g[i * LD + c], s.g[j * LD + c], a0);
-                }
-                v[h] = a0 + a1;
-            }
-            const double piv = __shfl_sync(0xffffffffu, v[0], 0);
-            const double d0 = s.g[j * LD + j];              // still the original diagonal entry
-            const bool keep = piv > kPivotFloor * d0 && d0 > 0.0;
-            const double inv = keep ? rsqrt(piv) : 0.0;
-            if (!keep) rank_flag = 1;
-            __syncwarp();
-#pragma unroll
-            for (int h = 0; h < kH; ++h) {
-                const int i = j + lane + 32 * h;
-                if (i < m) s.g[i * LD + j] = (i == j) ? piv * inv : v[h] * inv;
-            }
-            if (lane == 0) s.inv_diag[j] = inv;
-            __syncwarp();
-        }
-        if (lane == 0 && rank_flag) s.flags |= COMPACTOR_STATUS_RANK;
-    }
+    if (tid < MP) s.diag0[tid] = s.u.g[tid * MP + tid];
     __syncthreads();
-
-    // ---- W = Phi L^-T: forward substitution along the row, a block of columns in registers --------
-    {
-        constexpr int kWB = WBlock<MP>::value;
-        const int row = tid;
-        __nv_bfloat16* w_hi = w_out + (size_t)unit * w_elems_per_unit(MP);
-        __nv_bfloat16* w_lo = w_hi + (size_t)MP * kD;
-#pragma unroll 1
-        for (int c0 = 0; c0 < MP; c0 += kWB) {
-            double r[kWB];
-#pragma unroll
-            for (int c = 0; c < kWB; ++c) r[c] = (c0 + c < m && !bad) ? (double)phi[row * m + c0 + c] : 0.0;
-            for (int j = 0; j < c0; ++j) {                  // what the finished blocks take out of this one
-                const double wj = s.parked[j * kCholThreads + tid];
-#pragma unroll
-                for (int c = 0; c < kWB; ++c) r[c] = fma(-wj, s.g[(c0 + c) * LD + j], r[c]);
-            }
-#pragma unroll
-            for (int j = 0; j < kWB; ++j) {
-                const double wj = r[j] * s.inv_diag[c0 + j];
-                r[j] = wj;
-#pragma unroll
-                for (int c = j + 1; c < kWB; ++c) r[c] = fma(-wj, s.g[(c0 + c) * LD + c0 + j], r[c]);
-            }
-            if (c0 + kWB < MP) {
-#pragma unroll
-                for (int j = 0; j < kWB; ++j) s.parked[(c0 + j) * kCholThreads + tid] = r[j];
-            }
-#pragma unroll
-            for (int j = 0; j < kWB; ++j) {
-                const __nv_bfloat16 hi = __double2bfloat16(r[j]);
-                w_hi[(c0 + j) * kD + row] = hi;
-                w_lo[(c0 + j) * kD + row] = __double2bfloat16(r[j] - (double)__bfloat162float(hi));
-            }
-        }
+    if (!bad) cholesky_panels<MP, kCholWarps>(s.u.g, s.diag0, s.inv_diag, m, tid, &s.flags, sync);
+    __syncthreads();
+    __nv_bfloat16* w_unit = w_out + (size_t)unit * w_elems_per_unit(MP);
+    if (!bad) {
+        for (int rb = warp * 16; rb < kD; rb += kCholWarps * 16) solve_w_tiles<MP>(s.phi, s.u.g, s.inv_diag, rb, lane, w_unit);
+    } else {                                              // a unit with non-finite keys gets W = 0
+        for (int e = tid; e < (int)w_elems_per_unit(MP); e += kCholThreads) w_unit[e] = __float2bfloat16(0.f);
     }
     if (tid == 0 && status != nullptr && s.flags != 0) atomicOr(&status[unit], s.flags);
 }
@@ -358,7 +262,9 @@ template <int MP>
 struct EigSmem {
     static constexpr int kLd = MP + 1;
     double a[MP * kLd];          // G, driven to diagonal form
-    double v[MP * kLd];          // accumulated rotations: columns are the eigenvectors
+    double v[MP * kLd];          // accumulated rotations: columns are the eigenvectors (first: G by columns, as it is formed)
+    double t[kTRows * (MP + 4)]; // staged rows of T while G is formed
+    float phi[kD * MP];
     double rot_c[MP / 2], rot_s[MP / 2];
     int rot_p[MP / 2], rot_q[MP / 2];
     double inv_sqrt[MP];
@@ -368,7 +274,7 @@ struct EigSmem {
 
 template <int MP>
 __global__ void __launch_bounds__(kEigThreads, 3)
-eig_kernel(Plan p, const double* __restrict__ g_partials, const float* __restrict__ phi, double floor,
+eig_kernel(Plan p, const double* __restrict__ t_buf, const float* __restrict__ phi, double floor,
            __nv_bfloat16* __restrict__ w_out, int* __restrict__ status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using Smem = EigSmem<MP>;
@@ -382,18 +288,25 @@ eig_kernel(Plan p, const double* __restrict__ g_partials, const float* __restric
     if (tid == 0) s.flags = 0;
     __syncthreads();
     {
-        const double* src = g_partials + (size_t)unit * kSlices * (MP * MP);
-        bool finite = true;
-        for (int e = tid; e < MP * MP; e += kEigThreads) {
-            double x = 0.0;
-#pragma unroll
-            for (int r = 0; r < kSlices; ++r) x += src[(size_t)r * (MP * MP) + e];
-            const int i = e / MP, j = e % MP;
-            s.a[i * LD + j] = x;
-            s.v[i * LD + j] = (i == j) ? 1.0 : 0.0;
-            finite = finite && isfinite(x);
+        // G = Phi^T T on fp64 mma into `v` (by columns, lower triangle), then mirrored into `a`
+        for (int i = tid; i < kD * MP; i += kEigThreads) {
+            const int row = i / MP, col = i - row * MP;
+            s.phi[i] = col < m ? __ldg(phi + row * m + col) : 0.f;
         }
+        __syncthreads();
+        auto sync = [] { __syncthreads(); };
+        const bool finite = gram_of_sketch<MP, kEigThreads / 32>(t_buf + (size_t)unit * kD * MP, s.phi, s.v, s.t, tid, sync);
         if (!finite) atomicOr(&s.flags, COMPACTOR_STATUS_NONFINITE);
+        __syncthreads();
+        for (int e = tid; e < MP * MP; e += kEigThreads) {
+            const int i = e / MP, j = e % MP;
+            s.a[i * LD + j] = i >= j ? s.v[j * MP + i] : s.v[i * MP + j];
+        }
+        __syncthreads();
+        for (int e = tid; e < MP * MP; e += kEigThreads) {
+            const int i = e / MP, j = e % MP;
+            s.v[i * LD + j] = (i == j) ? 1.0 : 0.0;
+        }
     }
     __syncthreads();
     const bool bad = (s.flags & COMPACTOR_STATUS_NONFINITE) != 0;
@@ -528,15 +441,16 @@ eig_kernel(Plan p, const double* __restrict__ g_partials, const float* __restric
 
 template <int MP>
 cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials, const float* phi,
-                             double* g_partials, __nv_bfloat16* w, int* status, int factorization, double eig_floor,
-                             cudaStream_t stream) {
+                             double* t_buf, __nv_bfloat16* w, int* status, int factorization, double eig_floor,
+                             int sm_count, cudaStream_t stream) {
     const int units = p.layers * p.heads * p.batch;
     const int smem = (int)sizeof(ProjectSmem<MP>);
     cudaError_t e = cudaFuncSetAttribute(project_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     const int n_items = units * kSlices;
-    const int grid = n_items < 2 * 148 ? n_items : 2 * 148;       // two CTAs fit on an SM
-    project_kernel<MP><<<grid, kProjThreads, smem, stream>>>(p, k, partials, phi, g_partials, n_items);
+    const int resident = 2 * sm_count;                            // two CTAs fit on an SM
+    const int grid = n_items < resident ? n_items : resident;
+    project_kernel<MP><<<grid, kProjThreads, smem, stream>>>(p, k, partials, phi, t_buf, n_items);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (factorization == COMPACTOR_FACTOR_EIG) {
@@ -544,7 +458,7 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
             const int esmem = (int)sizeof(EigSmem<MP>);
             e = cudaFuncSetAttribute(eig_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, esmem);
             if (e != cudaSuccess) return e;
-            eig_kernel<MP><<<units, kEigThreads, esmem, stream>>>(p, g_partials, phi, eig_floor, w, status);
+            eig_kernel<MP><<<units, kEigThreads, esmem, stream>>>(p, t_buf, phi, eig_floor, w, status);
         } else {
             return cudaErrorInvalidValue;        // two m x m fp64 matrices no longer fit in shared memory
         }
@@ -552,22 +466,23 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
         const int csmem = (int)sizeof(CholSmem<MP>);
         e = cudaFuncSetAttribute(cholesky_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, csmem);
         if (e != cudaSuccess) return e;
-        cholesky_kernel<MP><<<units, kCholThreads, csmem, stream>>>(p, g_partials, phi, w, status);
+        cholesky_kernel<MP><<<units, kCholThreads, csmem, stream>>>(p, t_buf, phi, w, status);
     }
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* g_partials,
-                          __nv_bfloat16* w, int* status, int factorization, double eig_floor, cudaStream_t stream) {
+cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* t_buf,
+                          __nv_bfloat16* w, int* status, int factorization, double eig_floor, int sm_count,
+                          cudaStream_t stream) {
     if (p.layers * p.heads * p.batch == 0) return cudaSuccess;
     switch (p.mp) {
-        case 16: return launch_factor_mp<16>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
-        case 32: return launch_factor_mp<32>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
-        case 48: return launch_factor_mp<48>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
-        case 64: return launch_factor_mp<64>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
-        case 128: return launch_factor_mp<128>(p, k, partials, phi, g_partials, w, status, factorization, eig_floor, stream);
+        case 16: return launch_factor_mp<16>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
+        case 32: return launch_factor_mp<32>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
+        case 48: return launch_factor_mp<48>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
+        case 64: return launch_factor_mp<64>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
+        case 128: return launch_factor_mp<128>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -28,12 +28,14 @@
 // further waits fall through (control flow stays the same, so no thread is left at a barrier),
 // and the unit is flagged COMPACTOR_STATUS_TIMEOUT.
 #include "common.cuh"
+#include "factor_math.cuh"
 #include "sm100.cuh"
 
 namespace compactor {
 namespace {
 
 using namespace sm100;
+using namespace factor_math;
 
 constexpr int kTile = 128;
 constexpr int kBoxBytes = kTile * 128;     // 64 channels x 128 tokens x 2 B
@@ -48,11 +50,8 @@ constexpr int kQueue = 3;                  // pieces handed over inside a CTA (t
 constexpr uint32_t kTmemCols = 512;        // two Gram accumulators (128 columns each) + two scoring accumulators
 constexpr uint32_t kScoreCol0 = 256;
 constexpr int kOutTiles = 4;               // tiles whose scores leave together
-constexpr double kPivotFloor = 9.5367431640625e-07;   // 2^-20
 constexpr int kExactGramTokens = 256;      // units this short take their Gram matrix in fp64 straight from the keys
 constexpr int kStageTokens = 8;
-constexpr int kTChunk = 32;                // rows of T staged at a time for G = Phi^T T
-constexpr int kPanel = 8;                  // columns per panel of the Cholesky factorisation
 constexpr int kLdC = kD + 4;               // row stride (doubles) of the staged rows of C: fragment loads without bank conflicts
 
 #ifdef COMPACTOR_SWEEP_PROFILE
@@ -79,7 +78,7 @@ struct __align__(1024) SweepSmem {
     float phi[kD * MP];                    // the sketch, zero in the padded columns
     union Scratch {
         struct { double c[8 * kLdC]; double keys[kStageTokens * kD]; } slice;
-        double t[kTChunk * kLdT];
+        double t[kTRows * kLdT];
         struct { double g[MP * kLd]; double diag0[MP]; double inv_diag[MP]; } chol;
     } scratch;
     float obuf[2][kOutTiles * kTile];
@@ -114,11 +113,6 @@ __device__ __forceinline__ void st_release_u32(unsigned* p, unsigned v) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory"); }
-
-__device__ __forceinline__ void mma_f64(double (&d)[2], double a, double b) {
-    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                 : "+d"(d[0]), "+d"(d[1]) : "d"(a), "d"(b));
-}
 
 __device__ __forceinline__ int unit_pieces(const Plan& p, int unit) {
     const int b = unit % p.batch;
@@ -157,171 +151,6 @@ __device__ void advance_w_prefix(const SweepArgs& a) {
         if (ld_acquire_u32(reinterpret_cast<const unsigned*>(a.w_ready) + wu) == 0u) return;
         __threadfence();
         atomicCAS(&a.sched->sstate, ss, ss + 1ull);
-    }
-}
-
-// 1 / sqrt(x) for a positive, finite, normal x: single-precision seed on x scaled by an even power of two
-// into [1, 4), one Newton step in double precision (relative error of the order of 1e-13: the factor it
-// scales stays consistent, L L^T = G to that accuracy, far below what the scores resolve), scaled back.
-// The chain of 48 dependent pivots is what the factorisation's latency consists of, so the conversions
-// between the two formats are done on the bit patterns (integer instructions have a fraction of the
-// latency of the conversion instructions).
-__device__ __forceinline__ double fast_rsqrt(double x) {
-    const int hi = __double2hiint(x), lo = __double2loint(x);
-    const int eh = (((hi >> 20) & 0x7ff) - 1023) >> 1;
-    const int hs = hi - ((2 * eh) << 20);                                   // x * 2^(-2 eh), in [1, 4)
-    const double xs = __hiloint2double(hs, lo);
-    const float xf = __int_as_float(((hs - ((1023 - 127) << 20)) << 3) | (int)((unsigned)lo >> 29));   // xs truncated to fp32
-    const int yb = __float_as_int(rsqrtf(xf));                              // in (0.5, 1]
-    double y = __hiloint2double((int)((unsigned)yb >> 3) + ((1023 - 127) << 20), yb << 29);
-    const double h = 0.5 * xs;
-    y = y * fma(-h * y, y, 1.5);
-    return __hiloint2double(__double2hiint(y) - (eh << 20), __double2loint(y));
-}
-
-// One panel (columns j0 .. j1-1, at most eight) of the right-looking Cholesky factorisation, by one warp.
-// `g` holds the lower triangle by columns, g[c * LD + i] = A[i][c] for i >= c.  Every lane factors the
-// panel's 8 x 8 diagonal block itself (the same arithmetic in all lanes: no pivot has to travel), then
-// solves the panel entries of its own rows (lane and lane + 32) against it.  Also leaves the inverse of
-// the diagonal block's factor, X = L_JJ^-1, below the diagonal in the free triangle of `g`
-// (g[(j0 + n) * LD + j0 + k] = X[n][k], k < n; the diagonal of X is inv_diag).  Pivots not larger than
-// 2^-20 of their original diagonal entry are dropped (their column of L and of X is zero).
-// Returns true if a pivot was dropped.
-template <int LD>
-__device__ __noinline__ bool factor_panel(double* g, const double* diag0, double* inv_diag, int j0, int j1, int m, int lane) {
-    double dd[kPanel][kPanel];                    // lower triangle of the diagonal block
-#pragma unroll
-    for (int r = 0; r < kPanel; ++r)
-#pragma unroll
-        for (int c = 0; c <= r; ++c) {               // loads are unconditional (they then travel together); masked afterwards
-            const double v = g[(j0 + c) * LD + j0 + r];
-            dd[r][c] = (j0 + r < j1) ? v : 0.0;
-        }
-    const int r0 = lane, r1 = lane + 32;
-    double a0[kPanel], a1[kPanel];
-#pragma unroll
-    for (int c = 0; c < kPanel; ++c) {
-        const double v0 = g[(j0 + c) * LD + min(r0, LD - 1)], v1 = g[(j0 + c) * LD + min(r1, LD - 1)];
-        a0[c] = (r0 < m && j0 + c < j1) ? v0 : 0.0;
-        a1[c] = (r1 < m && j0 + c < j1) ? v1 : 0.0;
-    }
-    // One straight line of code (no branches): the pivot chain, the solves of the lane's rows and the inverse of the
-    // diagonal block are independent chains of double-precision operations, and the compiler interleaves them.
-    // Columns past j1 (a short last panel) have a zero pivot: they are "dropped" (zero column) without being counted.
-    double inv[kPanel];
-    bool dropped = false;
-#pragma unroll
-    for (int c = 0; c < kPanel; ++c) {
-        const double piv = dd[c][c], d0 = diag0[min(j0 + c, LD - 1)];
-        const bool keep = piv > kPivotFloor * d0 && d0 > 0.0;
-        inv[c] = keep ? fast_rsqrt(keep ? piv : 1.0) : 0.0;
-        dropped = dropped || (!keep && j0 + c < j1);
-        dd[c][c] = piv * inv[c];
-#pragma unroll
-        for (int r = c + 1; r < kPanel; ++r) dd[r][c] *= inv[c];
-#pragma unroll
-        for (int r = c + 1; r < kPanel; ++r)
-#pragma unroll
-            for (int c2 = c + 1; c2 <= r; ++c2) dd[r][c2] = fma(-dd[r][c], dd[c2][c], dd[r][c2]);
-        // the lane's rows: l[c] = (a[c] - sum_{c' < c} l[c'] L_JJ[c][c']) / L_JJ[c][c], right-looking
-        a0[c] *= inv[c];
-        a1[c] *= inv[c];
-#pragma unroll
-        for (int c2 = c + 1; c2 < kPanel; ++c2) {
-            a0[c2] = fma(-a0[c], dd[c2][c], a0[c2]);
-            a1[c2] = fma(-a1[c], dd[c2][c], a1[c2]);
-        }
-    }
-#pragma unroll
-    for (int c = 0; c < kPanel; ++c) {
-        if (j0 + c < j1) {
-            if (r0 < m && r0 >= j0 + c) g[(j0 + c) * LD + r0] = a0[c];
-            if (r1 < m && r1 >= j0 + c) g[(j0 + c) * LD + r1] = a1[c];
-        }
-    }
-    // X = L_JJ^-1 by forward substitution (every lane computes it, lane k stores column k):
-    // x[k] = inv[k], x[n] = -inv[n] sum_{t=k}^{n-1} L_JJ[n][t] x[t], right-looking
-#pragma unroll
-    for (int k = 0; k < kPanel; ++k) {
-        double x[kPanel];
-#pragma unroll
-        for (int n = k + 1; n < kPanel; ++n) x[n] = 0.0;
-        x[k] = inv[k];
-#pragma unroll
-        for (int t = k; t < kPanel; ++t) {
-            if (t > k) x[t] *= inv[t];
-#pragma unroll
-            for (int n = t + 1; n < kPanel; ++n) x[n] = fma(-dd[n][t], x[t], x[n]);
-        }
-        if (lane == k) {
-            if (j0 + k < j1) inv_diag[j0 + k] = inv[k];
-#pragma unroll
-            for (int n = k + 1; n < kPanel; ++n)
-                if (j0 + n < j1) g[(j0 + n) * LD + j0 + k] = x[n];
-        }
-    }
-    return dropped;
-}
-
-// W = Phi L^-T for the 16 rows of Phi that one warp owns, as a blocked forward substitution on fp64
-// mma.m8n8k4: W_J = (Phi_J - sum_{I<J} W_I L_JI^T) X_JJ^T, the blocks of W kept in registers as A
-// fragments.  Each 8 x 8 block of the result is split into two bf16 terms and stored at
-// w_hi[col * 128 + row] and w_hi[(MP + col) * 128 + row].
-template <int MP>
-__device__ __noinline__ void solve_w_tiles(const float* phi, const double* g, const double* inv_diag, int row_base,
-                                           int lane, __nv_bfloat16* w_hi) {
-    constexpr int LD = MP, kNB = MP / 8;
-    const int fr = lane >> 2, fk = lane & 3;
-    __nv_bfloat16* w_lo = w_hi + (size_t)MP * kD;
-    double wa[2][kNB][2];                         // [m-tile][block][k-step]: A fragments of the finished blocks
-#pragma unroll
-    for (int J = 0; J < kNB; ++J) {
-        double d[2][2];
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-            const int row = row_base + mt * 8 + fr;
-            d[mt][0] = (double)phi[row * MP + J * 8 + 2 * fk];
-            d[mt][1] = (double)phi[row * MP + J * 8 + 2 * fk + 1];
-        }
-#pragma unroll
-        for (int I = 0; I < J; ++I)
-#pragma unroll
-            for (int sk = 0; sk < 2; ++sk) {
-                const double b = -g[(I * 8 + 4 * sk + fk) * LD + J * 8 + fr];       // -(L_JI^T)[k][n] = -L[J*8+n][I*8+k]
-                mma_f64(d[0], wa[0][I][sk], b);
-                mma_f64(d[1], wa[1][I][sk], b);
-            }
-        // right-hand block times X_JJ^T: fragments of the left operand come from the accumulator by quad shuffles
-        double e[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
-#pragma unroll
-        for (int sk = 0; sk < 2; ++sk) {
-            const int k = 4 * sk + fk, n = fr;                                        // B[k][n] = X[n][k]
-            const double xg = g[(J * 8 + n) * LD + J * 8 + k], xd = inv_diag[J * 8 + n];    // both loaded, one chosen
-            const double b = k < n ? xg : (k == n ? xd : 0.0);
-            const int src = (lane & ~3) | (2 * sk + (fk >> 1));
-#pragma unroll
-            for (int mt = 0; mt < 2; ++mt) {
-                const double v0 = __shfl_sync(0xffffffffu, d[mt][0], src), v1 = __shfl_sync(0xffffffffu, d[mt][1], src);
-                mma_f64(e[mt], (fk & 1) ? v1 : v0, b);
-            }
-        }
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-            const int row = row_base + mt * 8 + fr;
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-                const int col = J * 8 + 2 * fk + q;
-                const __nv_bfloat16 hi = __double2bfloat16(e[mt][q]);
-                w_hi[col * kD + row] = hi;
-                w_lo[col * kD + row] = __double2bfloat16(e[mt][q] - (double)__bfloat162float(hi));
-            }
-#pragma unroll
-            for (int sk = 0; sk < 2; ++sk) {
-                const int src = (lane & ~3) | (2 * sk + (fk >> 1));
-                const double v0 = __shfl_sync(0xffffffffu, e[mt][0], src), v1 = __shfl_sync(0xffffffffu, e[mt][1], src);
-                wa[mt][J][sk] = (fk & 1) ? v1 : v0;
-            }
-        }
     }
 }
 
@@ -866,59 +695,12 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
             PROF_T(tw2);
 
             // ================================================================ the unit's last slice is in: G, Cholesky, W
-            constexpr int LD = Smem::kLd, LDT = Smem::kLdT, kNT = MP / 8;
-            constexpr int kLower = kNT * (kNT + 1) / 2;
-            constexpr int kMaxTiles = (kLower + kWorkerWarps - 1) / kWorkerWarps;
             const int m = p.m;
-            double* g = s.scratch.chol.g;                 // upper storage: g[c * LD + i] = A[i][c] for i >= c
+            double* g = s.scratch.chol.g;                 // by columns: g[c * MP + i] = A[i][c] for i >= c
+            auto wsync = [] { workers_sync(); };
             {
                 // ---- G = Phi^T T, lower-triangular 8 x 8 tiles only, T staged 32 rows at a time
-                double d[kMaxTiles][2];
-                int tmt[kMaxTiles], tnt[kMaxTiles];
-#pragma unroll
-                for (int si = 0; si < kMaxTiles; ++si) {
-                    d[si][0] = d[si][1] = 0.0;
-                    int rem = wwarp + kWorkerWarps * si, mt = 0;
-                    while (rem > mt) { rem -= mt + 1; ++mt; }
-                    tmt[si] = mt; tnt[si] = rem;
-                }
-                const double* t_unit = a.t_buf + (size_t)unit * kD * MP;
-                // all of T travels at once (one round of L2 latency); it is staged 32 rows at a time from registers
-                constexpr int kPerChunk = kTChunk * MP / kWorkers;
-                double tv[kD / kTChunk][kPerChunk];
-#pragma unroll
-                for (int chunk = 0; chunk < kD / kTChunk; ++chunk)
-#pragma unroll
-                    for (int u = 0; u < kPerChunk; ++u)
-                        tv[chunk][u] = __ldcg(t_unit + (size_t)chunk * kTChunk * MP + wtid + u * kWorkers);
-#pragma unroll
-                for (int chunk = 0; chunk < kD / kTChunk; ++chunk) {
-                    if (chunk > 0) workers_sync();
-#pragma unroll
-                    for (int u = 0; u < kPerChunk; ++u) {
-                        const int e = wtid + u * kWorkers, rr = e / MP, cc = e - rr * MP;
-                        s.scratch.t[rr * LDT + cc] = tv[chunk][u];
-                    }
-                    workers_sync();
-#pragma unroll
-                    for (int si = 0; si < kMaxTiles; ++si) {
-                        if (wwarp + kWorkerWarps * si >= kLower) continue;
-#pragma unroll
-                        for (int k0 = 0; k0 < kTChunk; k0 += 4)
-                            mma_f64(d[si], (double)s.phi[(chunk * kTChunk + k0 + fk) * MP + tmt[si] * 8 + fr],
-                                    s.scratch.t[(k0 + fk) * LDT + tnt[si] * 8 + fr]);
-                    }
-                }
-                workers_sync();
-                bool finite = true;
-#pragma unroll
-                for (int si = 0; si < kMaxTiles; ++si) {
-                    if (wwarp + kWorkerWarps * si >= kLower) continue;
-                    // fragment (row mt*8 + fr, columns nt*8 + 2 fk, + 1), stored by column
-                    g[(tnt[si] * 8 + 2 * fk) * LD + tmt[si] * 8 + fr] = d[si][0];
-                    g[(tnt[si] * 8 + 2 * fk + 1) * LD + tmt[si] * 8 + fr] = d[si][1];
-                    finite = finite && isfinite(d[si][0]) && isfinite(d[si][1]);
-                }
+                const bool finite = gram_of_sketch<MP, kWorkerWarps>(a.t_buf + (size_t)unit * kD * MP, s.phi, g, s.scratch.t, wtid, wsync);
                 if (!finite) atomicOr(&s.flags, COMPACTOR_STATUS_NONFINITE);
                 if (wtid < MP) s.scratch.chol.inv_diag[wtid] = 0.0;
             }
@@ -926,44 +708,10 @@ sweep_kernel(const __grid_constant__ SweepArgs a, const __grid_constant__ CUtens
             if (wtid == 0) PROF_ADD(13, tw2);
             PROF_T(tw3);
             const bool bad = (s.flags & COMPACTOR_STATUS_NONFINITE) != 0;
-            if (wtid < MP) s.scratch.chol.diag0[wtid] = g[wtid * LD + wtid];
+            if (wtid < MP) s.scratch.chol.diag0[wtid] = g[wtid * MP + wtid];
             workers_sync();
             // ---- Cholesky, right-looking by panels of eight columns: one warp factors the panel, all update what follows
-            if (!bad) {
-                for (int j0 = 0; j0 < m; j0 += kPanel) {
-                    const int j1 = min(j0 + kPanel, m);
-                    PROF_T(tpan);
-                    if (wwarp == 0) {
-                        const bool dropped = factor_panel<LD>(g, s.scratch.chol.diag0, s.scratch.chol.inv_diag, j0, j1, m, lane);
-                        if (lane == 0 && dropped) atomicOr(&s.flags, COMPACTOR_STATUS_RANK);
-                        if (lane == 0) PROF_ADD(17, tpan);
-                    }
-                    workers_sync();
-                    if (wtid == 0) PROF_ADD(18, tpan);
-                    // trailing block, rows and columns j1 .. : A_ij -= L_i L_j^T by 8 x 8 tiles on fp64 mma (lower tiles only;
-                    // rows and columns past m hold zeros)
-                    const int nb = (MP - j1) / 8;
-                    if (j1 < m && nb > 0) {
-                        for (int tile = wwarp; tile < nb * (nb + 1) / 2; tile += kWorkerWarps) {
-                            int rem = tile, bi = 0;
-                            while (rem > bi) { rem -= bi + 1; ++bi; }
-                            const int bj = rem;
-                            double* cp = g + (j1 + 8 * bj + 2 * fk) * LD + j1 + 8 * bi + fr;      // fragment (row fr, columns 2 fk, + 1)
-                            double d[2] = {cp[0], cp[LD]};
-#pragma unroll
-                            for (int sk = 0; sk < 2; ++sk) {
-                                const double av = g[(j0 + 4 * sk + fk) * LD + j1 + 8 * bi + fr];   // L[j1 + 8 bi + fr][j0 + k]
-                                const double bv = g[(j0 + 4 * sk + fk) * LD + j1 + 8 * bj + fr];   // (L_j^T)[k][n] = L[j1 + 8 bj + n][j0 + k]
-                                mma_f64(d, -av, bv);
-                            }
-                            cp[0] = d[0];
-                            cp[LD] = d[1];
-                        }
-                        workers_sync();
-                        if (wtid == 0) PROF_ADD(19, tpan);
-                    }
-                }
-            }
+            if (!bad) cholesky_panels<MP, kWorkerWarps>(g, s.scratch.chol.diag0, s.scratch.chol.inv_diag, m, wtid, &s.flags, wsync);
             workers_sync();
             if (wtid == 0) PROF_ADD(14, tw3);
             PROF_T(tw4);

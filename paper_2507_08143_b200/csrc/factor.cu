@@ -36,12 +36,12 @@ template <int MP>
 struct ProjectSmem {
     static constexpr int kLd = MP + 4;     // row stride (doubles): the four k-rows of a B fragment land in distinct banks
     double phi[kD * kLd];                  // Phi widened, [channel][column]
-    double c[kD * kRows];                  // C[k][row0 + i] at [k * kRows + i]  (C is symmetric)
+    static constexpr int kLdc = kRows + 4; // stride of a k-row of c: the four k-rows of an A fragment land in distinct banks
+    double c[kD * kLdc];                   // C[k][row0 + i] at [k * kLdc + i]  (C is symmetric)
     double keys[kStageTokens * kD];
 };
 
-// Persistent: each CTA loads Phi once and then walks (unit, slice) items with a grid stride; the
-// global loads of the next item's partials are in flight while the current item is multiplied.
+// Persistent: each CTA loads Phi once and then walks (unit, slice) items with a grid stride.
 template <int MP>
 __global__ void __launch_bounds__(kProjThreads, 2)
 project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const float* __restrict__ phi,
@@ -51,7 +51,7 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
     Smem& s = *reinterpret_cast<Smem*>(smem_raw);
     constexpr int LD = Smem::kLd;
     constexpr int kPer = kD * kRows / kProjThreads;     // elements of the C slice per thread: e = tid + 256 q
-    constexpr int kInFlight = 2;                        // partials loaded ahead per item
+    constexpr int kInFlight = 1;                        // partials loaded together (more would spill at two CTAs per SM)
     constexpr int kWarps = kProjThreads / 32;
     const int m = p.m, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
@@ -75,111 +75,92 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
         it.part = partials + ((size_t)it.lh * p.total_chunks + chunk_begin) * kGramElems;
         return it;
     };
-    double pre[kInFlight][kPer];
-    auto prefetch = [&](const Item& it) {
-        const bool any = it.n_part > 0 && it.n_tok > kExactGramTokens;      // the same for the whole CTA
-#pragma unroll
-        for (int u = 0; u < kInFlight; ++u)
-#pragma unroll
-            for (int q = 0; q < kPer; ++q) {
-                const int e = tid + q * kProjThreads;
-                pre[u][q] = 0.0;
-                if (any) {
-                    // The loads are unconditional (partials past the last one re-read the last and are masked below).
-                    // volatile: keeps the load here, ahead of the matrix products, instead of at its first use.
-                    const int uu = u < it.n_part ? u : it.n_part - 1;
-                    const double* src = it.part + (size_t)uu * kGramElems + (e / kRows) * kD + it.slice * kRows + (e % kRows);
-                    asm volatile("ld.global.cs.f64 %0, [%1];" : "=d"(pre[u][q]) : "l"(src));
-                }
-            }
-        if (any) {
-#pragma unroll
-            for (int u = 0; u < kInFlight; ++u)
-                if (u >= it.n_part) {
-#pragma unroll
-                    for (int q = 0; q < kPer; ++q) pre[u][q] = 0.0;
-                }
-        }
-    };
-
-    int item = blockIdx.x;
-    Item cur;
-    if (item < n_items) { cur = decode(item); prefetch(cur); }
-    for (; item < n_items; item += gridDim.x) {
+    constexpr int LDC = Smem::kLdc;
+    // Two CTAs share an SM: while one waits for its partial sums the other multiplies.
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const Item cur = decode(item);
+        const Item done = cur;
         const int row0 = cur.slice * kRows;
         // ---- the item's 32 columns of C (= 32 rows, by symmetry), summed over the partials ------
-        {
+        if (cur.n_tok > kExactGramTokens) {
             double acc[kPer];
 #pragma unroll
-            for (int q = 0; q < kPer; ++q) {
-                acc[q] = 0.0;
+            for (int q = 0; q < kPer; ++q) acc[q] = 0.0;
+            for (int pp = 0; pp < cur.n_part; pp += kInFlight) {
+                double v[kInFlight][kPer];
 #pragma unroll
-                for (int u = 0; u < kInFlight; ++u) acc[q] += pre[u][q];
-            }
-            if (cur.n_tok > kExactGramTokens) {
-                for (int pp = kInFlight; pp < cur.n_part; ++pp)           // more partials than the look-ahead holds
+                for (int u = 0; u < kInFlight; ++u) {
+                    // unconditional loads (a partial past the last one re-reads the last and is not added): loads under
+                    // a per-load condition are issued one after the other instead of together
+                    const int uu = pp + u < cur.n_part ? pp + u : cur.n_part - 1;
 #pragma unroll
                     for (int q = 0; q < kPer; ++q) {
                         const int e = tid + q * kProjThreads;
-                        acc[q] += __ldcs(cur.part + (size_t)pp * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
-                    }
-                __syncthreads();                              // the previous item's products are done with c
-#pragma unroll
-                for (int q = 0; q < kPer; ++q) s.c[tid + q * kProjThreads] = acc[q];
-            } else {
-                // short sequence: fp64 Gram straight from the keys, C[:, rows] = K^T K[:, rows], as fp64 mma.m8n8k4
-                // over four tokens at a time
-                const int layer = cur.lh / p.heads, head = cur.lh % p.heads;
-                const __nv_bfloat16* kbase = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
-                                             (long long)p.cu_seqlens[cur.b] * kmat.stride_token;
-                constexpr int kTilesPerWarp = (kD / 8) * (kRows / 8) / kWarps;
-                double d[kTilesPerWarp][2];
-#pragma unroll
-                for (int j = 0; j < kTilesPerWarp; ++j) d[j][0] = d[j][1] = 0.0;
-                // the keys of the next stage are on their way while the current stage is multiplied
-                constexpr int kLoads = kStageTokens * kD / kProjThreads;
-                float nxt[kLoads];
-                auto fetch = [&](int t0) {                    // missing tokens of the last stage are zeros
-#pragma unroll
-                    for (int u = 0; u < kLoads; ++u) {
-                        const int i = tid + u * kProjThreads, t = min(t0 + i / kD, cur.n_tok - 1);
-                        nxt[u] = __bfloat162float(kbase[(long long)t * kmat.stride_token + (i % kD)]);
-                        if (t0 + i / kD >= cur.n_tok) nxt[u] = 0.f;
-                    }
-                };
-                if (cur.n_tok > 0) fetch(0);
-                for (int t0 = 0; t0 < cur.n_tok; t0 += kStageTokens) {
-                    __syncthreads();
-#pragma unroll
-                    for (int u = 0; u < kLoads; ++u) s.keys[tid + u * kProjThreads] = (double)nxt[u];
-                    __syncthreads();
-                    if (t0 + kStageTokens < cur.n_tok) fetch(t0 + kStageTokens);
-#pragma unroll
-                    for (int ks = 0; ks < kStageTokens / 4; ++ks) {
-                        const double* krow = s.keys + (ks * 4 + fk) * kD;          // token ks*4 + fk of the stage
-#pragma unroll
-                        for (int j = 0; j < kTilesPerWarp; ++j) {
-                            const int tile = warp + j * kWarps;
-                            const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
-                            mma_f64(d[j], krow[mt * 8 + fr], krow[row0 + nt8 * 8 + fr]);   // A[channel][token], B[token][channel of the slice]
-                        }
+                        v[u][q] = __ldcs(cur.part + (size_t)uu * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
                     }
                 }
-                __syncthreads();                              // the previous item's products are done with c
 #pragma unroll
-                for (int j = 0; j < kTilesPerWarp; ++j) {
-                    const int tile = warp + j * kWarps;
-                    const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
-                    s.c[(mt * 8 + fr) * kRows + nt8 * 8 + 2 * fk] = d[j][0];
-                    s.c[(mt * 8 + fr) * kRows + nt8 * 8 + 2 * fk + 1] = d[j][1];
+                for (int u = 0; u < kInFlight; ++u)
+                    if (pp + u < cur.n_part) {
+#pragma unroll
+                        for (int q = 0; q < kPer; ++q) acc[q] += v[u][q];
+                    }
+            }
+            __syncthreads();                              // the previous item's products are done with c
+#pragma unroll
+            for (int q = 0; q < kPer; ++q) {
+                const int e = tid + q * kProjThreads;
+                s.c[(e / kRows) * LDC + (e % kRows)] = acc[q];
+            }
+        } else {
+            // short sequence: fp64 Gram straight from the keys, C[:, rows] = K^T K[:, rows], as fp64 mma.m8n8k4
+            // over four tokens at a time
+            const int layer = cur.lh / p.heads, head = cur.lh % p.heads;
+            const __nv_bfloat16* kbase = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
+                                         (long long)p.cu_seqlens[cur.b] * kmat.stride_token;
+            constexpr int kTilesPerWarp = (kD / 8) * (kRows / 8) / kWarps;
+            double d[kTilesPerWarp][2];
+#pragma unroll
+            for (int j = 0; j < kTilesPerWarp; ++j) d[j][0] = d[j][1] = 0.0;
+            // the keys of the next stage are on their way while the current stage is multiplied
+            constexpr int kLoads = kStageTokens * kD / kProjThreads;
+            float nxt[kLoads];
+            auto fetch = [&](int t0) {                    // missing tokens of the last stage are zeros
+#pragma unroll
+                for (int u = 0; u < kLoads; ++u) {
+                    const int i = tid + u * kProjThreads, t = min(t0 + i / kD, cur.n_tok - 1);
+                    nxt[u] = __bfloat162float(kbase[(long long)t * kmat.stride_token + (i % kD)]);
+                    if (t0 + i / kD >= cur.n_tok) nxt[u] = 0.f;
                 }
+            };
+            if (cur.n_tok > 0) fetch(0);
+            for (int t0 = 0; t0 < cur.n_tok; t0 += kStageTokens) {
+                __syncthreads();
+#pragma unroll
+                for (int u = 0; u < kLoads; ++u) s.keys[tid + u * kProjThreads] = (double)nxt[u];
+                __syncthreads();
+                if (t0 + kStageTokens < cur.n_tok) fetch(t0 + kStageTokens);
+#pragma unroll
+                for (int ks = 0; ks < kStageTokens / 4; ++ks) {
+                    const double* krow = s.keys + (ks * 4 + fk) * kD;          // token ks*4 + fk of the stage
+#pragma unroll
+                    for (int j = 0; j < kTilesPerWarp; ++j) {
+                        const int tile = warp + j * kWarps;
+                        const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
+                        mma_f64(d[j], krow[mt * 8 + fr], krow[row0 + nt8 * 8 + fr]);   // A[channel][token], B[token][channel of the slice]
+                    }
+                }
+            }
+            __syncthreads();                              // the previous item's products are done with c
+#pragma unroll
+            for (int j = 0; j < kTilesPerWarp; ++j) {
+                const int tile = warp + j * kWarps;
+                const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
+                s.c[(mt * 8 + fr) * LDC + nt8 * 8 + 2 * fk] = d[j][0];
+                s.c[(mt * 8 + fr) * LDC + nt8 * 8 + 2 * fk + 1] = d[j][1];
             }
         }
         __syncthreads();
-
-        // look ahead: the next item's partials travel while this item is multiplied
-        const Item done = cur;
-        if (item + (int)gridDim.x < n_items) { cur = decode(item + gridDim.x); prefetch(cur); }
 
         // ---- T[rows] (32 x MP) = C[rows,:] (32 x 128) Phi (128 x MP): a warp-wide fp64 mma does 256 multiply-adds for two
         // 8-byte shared-memory loads per lane; the contraction is cut into four independent chains --------------------
@@ -194,7 +175,7 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
 #pragma unroll
                 for (int g = 0; g < 4; ++g) {
                     const int k = g * (kD / 4) + k0 + fk;
-                    mma_f64(d[g], s.c[k * kRows + mt * 8 + fr], s.phi[k * LD + nt * 8 + fr]);   // A[row][k] = C[k][row0 + row], B[k][col]
+                    mma_f64(d[g], s.c[k * LDC + mt * 8 + fr], s.phi[k * LD + nt * 8 + fr]);   // A[row][k] = C[k][row0 + row], B[k][col]
                 }
             }
             __stcg(reinterpret_cast<double2*>(t_rows + (size_t)(mt * 8 + fr) * MP + nt * 8 + 2 * fk),

@@ -153,9 +153,10 @@ int compactor_nll(const void* logits, int32_t logits_dtype, int64_t rows, int32_
 
 /*
  * Bytes of device workspace that compactor_score and compactor_compress need for this shape.
- * compactor_select and compactor_compact only use a small table at its start and accept any
- * workspace of at least 16*(batch+1) bytes rounded up to 256.  The workspace must be 256-byte
- * aligned; its contents need not be preserved between calls.  Returns 0 for an invalid shape.
+ * compactor_select and compactor_compact only need a small table at its start and accept any
+ * workspace of at least 16*(batch+1) bytes rounded up to 256 (compactor_select uses whatever
+ * follows the table as scratch, see there).  The workspace must be 256-byte aligned; its
+ * contents need not be preserved between calls.  Returns 0 for an invalid shape.
  */
 size_t compactor_workspace_bytes(const compactor_shape* shape);
 
@@ -205,6 +206,10 @@ int compactor_score_variant(const compactor_shape* shape, compactor_mat k_score,
  *   idx_out      device int32 [layers][heads][total_keep]: for each unit the indices (local to
  *                the sequence, 0-based) of its keep_counts[b] largest scores, ascending.  Equal
  *                scores are ranked by lower index first.  NaN scores rank above +inf.
+ * One CTA selects a unit.  Where that would leave most of the GPU idle (fewer units than SMs and
+ * sequences of 10^5 tokens or more) and the workspace is the size compactor_workspace_bytes()
+ * gives, every score vector is cut into slices that share a histogram and a candidate list in the
+ * workspace; the indices are the same either way.
  */
 int compactor_select(const compactor_shape* shape, const float* scores,
                      const int32_t* keep_counts, int32_t* idx_out,
@@ -289,7 +294,9 @@ int compactor_attention_scores_status(const compactor_shape* shape, compactor_ma
  *                     [off[h], off[h+1]) with off = head_offsets_out[l][b][0 .. heads]; indices are
  *                     local to the sequence and ascending within a head.
  *   head_offsets_out  device int32 [layers][batch][heads + 1], off[0] = 0, off[heads] = heads * keep_counts[b].
- * heads must not exceed 64.  Workspace: compactor_across_heads_workspace_bytes().
+ * heads must not exceed 64.  Workspace: compactor_across_heads_workspace_bytes() (the tables, and
+ * per (layer, sequence) a histogram, a candidate list and per-slice counts: every head's scores are
+ * cut into slices that are counted and emitted by CTAs of their own).
  * compactor_compact_across_heads gathers K/V rows in exactly that order into
  * k_out / v_out [layers][heads * total_keep][d] (bit copies; out-of-range indices are skipped).
  */
@@ -353,7 +360,7 @@ int compactor_compress_full(const compactor_shape* shape, const compactor_option
  * no workspace argument: the scratch is a fixed array of compactor_builtin_scratch_bytes()
  * (32 MiB) inside the library, resident on every device the process uses from the first use of
  * the library on that device until the process exits.  The call allocates and frees nothing.
- *   - Size limit: the scratch must hold 16*(batch+1) bytes of tables, about 160 KiB per unit
+ *   - Size limit: the scratch must hold 16*(batch+1) bytes of tables, about 72 KiB per unit
  *     (at m = 48) and 128 KiB per Gram block (blocks are lengthened up to 65536 tokens to make it
  *     fit, i.e. down to 2 bytes per token per (layer, head)).  A larger problem is refused with
  *     COMPACTOR_E_TOO_LARGE before anything is enqueued; split it by layers or use

@@ -4,6 +4,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <mutex>
 #include <vector>
 
@@ -37,6 +38,22 @@ int sm_count() {
     return cached[dev];
 }
 
+// Slices per score vector for the selection spread over several CTAs: enough CTAs for two per SM, no
+// slice shorter than 8192 scores.
+constexpr int kMaxSelectParts = 64;
+int select_parts(long long vectors, long long max_n) {
+    const long long want = (2LL * sm_count() + vectors - 1) / (vectors > 0 ? vectors : 1);
+    long long parts = want < 1 ? 1 : want;
+    if (parts > max_n / 8192) parts = max_n / 8192;
+    if (parts > kMaxSelectParts) parts = kMaxSelectParts;
+    return parts < 1 ? 1 : (int)parts;
+}
+long long longest_sequence(const compactor_shape* s) {
+    long long m = 0;
+    for (int b = 0; b < s->batch; ++b) m = std::max<long long>(m, s->cu_seqlens[b + 1] - s->cu_seqlens[b]);
+    return m;
+}
+
 // The fused persistent sweep is switched on with COMPACTOR_FUSED_SWEEP=1 (it does not yet beat the
 // separate kernels; see sweep.cu).
 // 0: separate kernels; 1: one launch (Gram, factor and scoring pieces interleaved, keys meant to stay in L2);
@@ -53,6 +70,7 @@ struct HostPlan {
     std::vector<int> tables;       // cu_seqlens | cu_keep | cu_chunks | cu_schunks, each batch+1
     size_t off_tables, off_w, off_gpart, off_partials, off_scores, total_bytes;
     int units;
+    long long max_n;               // longest sequence
     // fused sweep (Cholesky route, padded sketch of at most kFusedMaxMp columns)
     bool fused;
     int slices, window, n_slots, max_pieces, resident16;
@@ -101,6 +119,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     p.layers = s->layers; p.heads = s->heads; p.batch = s->batch;
     p.m = s->m; p.mp = s->m <= 64 ? (s->m + 15) / 16 * 16 : 128;
     p.total_tokens = s->cu_seqlens[s->batch];
+    hp->max_n = longest_sequence(s);
     hp->units = s->layers * s->heads * s->batch;
     hp->fused = allow_fused && p.mp <= kFusedMaxMp && fused_sweep_enabled();
     hp->slices = 0; hp->window = 0; hp->n_slots = 0; hp->max_pieces = 0; hp->total_pieces = 0;
@@ -352,9 +371,47 @@ int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn,
         CK(launch_score(hp.plan, k, w, scores, status, stream));
         CK(mk.mark(3, stream));
     }
-    if (attn != nullptr) CK(launch_blend(hp.plan, attn, lambda, scores, stream));
+    if (attn != nullptr) {
+        // a few long units: cut into slices (W and the Gram partials are dead by now; their place holds the slices' statistics)
+        int parts = 1;
+        if (2 * hp.units <= sm_count() && hp.max_n >= 65536) parts = select_parts(hp.units, hp.max_n);
+        if (sizeof(double) * 4 * (size_t)hp.units * parts > hp.off_scores - hp.off_w) parts = 1;
+        CK(launch_blend(hp.plan, attn, lambda, scores, parts, reinterpret_cast<double*>(ws + hp.off_w), stream));
+    }
     CK(mk.mark(4, stream));
     return COMPACTOR_OK;
+}
+
+// Per-head selection.  One CTA per unit keeps every SM busy when there are many units; a few long
+// units (one layer of a long context) are cut into slices instead, which needs `scratch` for the shared
+// histograms and candidate lists.  Both routes give the same indices.
+cudaError_t select_per_head(const HostPlan& hp, const compactor_shape* shape, const float* scores, int* idx,
+                            char* scratch, size_t scratch_bytes, cudaStream_t st) {
+    // rough costs in microseconds: one CTA walks a unit's scores four times; the sliced route pays four small launches
+    // and then shares all scores between the SMs
+    const long long max_n = longest_sequence(shape);
+    const double t_single = 12.0 + 0.37e-3 * (double)max_n;
+    const double t_sliced = 40.0 + 6.0e-6 * (double)hp.plan.total_tokens * shape->layers * shape->heads;
+    if (hp.units <= sm_count() && t_sliced < 0.8 * t_single && scratch != nullptr) {
+        const int parts = select_parts(hp.units, max_n);
+        const MultiSelectLayout l = multi_select_layout(shape->layers, shape->heads, shape->batch, hp.plan.total_tokens,
+                                                        false, kMaxSelectParts);
+        if (parts > 1 && l.total <= scratch_bytes)
+            return launch_select_multi(hp.plan, scores, idx, nullptr, multi_select_at(scratch, l, parts, false), st);
+    }
+    return launch_select(hp.plan, scores, idx, st);
+}
+
+// Selection across heads: always the route with one CTA per (head, slice).
+cudaError_t select_across(const HostPlan& hp, const compactor_shape* shape, const float* scores, int* idx,
+                          int* head_offsets, char* scratch, cudaStream_t st) {
+    const int parts = select_parts(hp.units, longest_sequence(shape));
+    const MultiSelectLayout l = multi_select_layout(shape->layers, shape->heads, shape->batch, hp.plan.total_tokens,
+                                                    true, kMaxSelectParts);
+    return launch_select_multi(hp.plan, scores, idx, head_offsets, multi_select_at(scratch, l, parts, true), st);
+}
+size_t across_scratch_bytes(const compactor_shape* shape, long long total_tokens) {
+    return multi_select_layout(shape->layers, shape->heads, shape->batch, total_tokens, true, kMaxSelectParts).total;
 }
 
 }  // namespace
@@ -472,11 +529,11 @@ int compactor_select(const compactor_shape* shape, const float* scores, const in
     if (scores == nullptr || idx_out == nullptr || workspace == nullptr || !set_keep(shape, keep_counts, &hp))
         return COMPACTOR_E_INVALID_ARGUMENT;
     if (((uintptr_t)workspace & 255) != 0) return COMPACTOR_E_INVALID_ARGUMENT;
-    if (workspace_bytes < hp.off_w) return COMPACTOR_E_WORKSPACE;      // only the tables are used
+    if (workspace_bytes < hp.off_w) return COMPACTOR_E_WORKSPACE;      // the tables; the rest, if any, is scratch
     if (hp.plan.total_keep == 0) return COMPACTOR_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     CK(upload_tables(&hp, workspace, st));
-    CK(launch_select(hp.plan, scores, idx_out, st));
+    CK(select_per_head(hp, shape, scores, idx_out, static_cast<char*>(workspace) + hp.off_w, workspace_bytes - hp.off_w, st));
     return COMPACTOR_OK;
 }
 
@@ -519,7 +576,9 @@ static int compress_impl(const compactor_shape* shape, compactor_mat k_score, co
     CK(upload_tables(&hp, workspace, st));
     int rc = run_scoring(hp, to_mat(k_score), phi, attn_scores, lambda, scores, status, ws, st, mk);
     if (rc != COMPACTOR_OK) return rc;
-    if (hp.plan.total_keep > 0) CK(launch_select(hp.plan, scores, idx_out, st));
+    // W, the projections and the Gram partials are dead once the scores exist: the selection may use their place
+    if (hp.plan.total_keep > 0)
+        CK(select_per_head(hp, shape, scores, idx_out, ws + hp.off_w, hp.off_scores - hp.off_w, st));
     CK(mk.mark(5, st));
     if (hp.plan.total_keep > 0)
         CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out,
@@ -692,7 +751,7 @@ extern "C" int compactor_attention_scores(const compactor_shape* shape, compacto
 extern "C" size_t compactor_across_heads_workspace_bytes(const compactor_shape* shape) {
     HostPlan hp; int err = 0;
     if (!make_plan(shape, &hp, &err)) return 0;
-    return hp.off_w + align_up(sizeof(int32_t) * (size_t)shape->layers * shape->batch * (shape->heads + 1));
+    return hp.off_w + across_scratch_bytes(shape, hp.plan.total_tokens);
 }
 
 extern "C" int compactor_select_across_heads(const compactor_shape* shape, const float* scores,
@@ -709,10 +768,7 @@ extern "C" int compactor_select_across_heads(const compactor_shape* shape, const
     if (hp.plan.total_tokens == 0) return COMPACTOR_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     CK(upload_tables(&hp, workspace, st));
-    char* ws = static_cast<char*>(workspace) + hp.off_w;
-    uint32_t* thr = reinterpret_cast<uint32_t*>(ws);                                  // [layers * batch]
-    int* ties = reinterpret_cast<int*>(ws) + (size_t)shape->layers * shape->batch;    // [layers * batch * heads]
-    CK(launch_select_across(hp.plan, scores, idx_out, head_offsets_out, thr, ties, st));
+    CK(select_across(hp, shape, scores, idx_out, head_offsets_out, static_cast<char*>(workspace) + hp.off_w, st));
     return COMPACTOR_OK;
 }
 
@@ -764,8 +820,7 @@ bool full_layout(const compactor_shape* shape, const compactor_options* opt, Ful
         off += fl->attn_ws_bytes;
     }
     fl->off_across = off;
-    if (opt->selection == COMPACTOR_SELECT_ACROSS_HEADS)
-        off += align_up(sizeof(int32_t) * (size_t)shape->layers * shape->batch * (shape->heads + 1));
+    if (opt->selection == COMPACTOR_SELECT_ACROSS_HEADS) off += align_up(across_scratch_bytes(shape, hp.plan.total_tokens));
     fl->total = off;
     return true;
 }
@@ -830,14 +885,12 @@ extern "C" int compactor_compress_full(const compactor_shape* shape, const compa
     if (rc != COMPACTOR_OK) return rc;
     if (!across) {
         if (hp.plan.total_keep > 0) {
-            CK(launch_select(hp.plan, scores, idx_out, st));
+            CK(select_per_head(hp, shape, scores, idx_out, ws + hp.off_w, hp.off_scores - hp.off_w, st));
             CK(launch_compact(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out,
                               static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));
         }
     } else {
-        uint32_t* thr = reinterpret_cast<uint32_t*>(ws + fl.off_across);
-        int* ties = reinterpret_cast<int*>(thr) + (size_t)shape->layers * shape->batch;
-        CK(launch_select_across(hp.plan, scores, idx_out, head_offsets_out, thr, ties, st));
+        CK(select_across(hp, shape, scores, idx_out, head_offsets_out, ws + fl.off_across, st));
         if (hp.plan.total_keep > 0)
             CK(launch_compact_across(hp.plan, to_mat(k_cache), to_mat(v_cache), idx_out, head_offsets_out,
                                      static_cast<__nv_bfloat16*>(k_out), static_cast<__nv_bfloat16*>(v_out), st));

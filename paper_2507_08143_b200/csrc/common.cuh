@@ -94,7 +94,9 @@ cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, c
 cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
                          cudaStream_t stream);
 cudaError_t launch_sweep(const SweepArgs& a, int sm_count, cudaStream_t stream);
-cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* scores, cudaStream_t stream);
+// parts > 1 (with `stats`, 4 doubles per unit and part): every unit's vectors are cut into that many slices.
+cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* scores, int parts, double* stats,
+                         cudaStream_t stream);
 cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStream_t stream);
 cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int* idx,
                            __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream);
@@ -103,8 +105,56 @@ cudaError_t launch_nll(const void* logits, int is_fp32, long long rows, int voca
                        const int* targets, int batch, const int* cu_rows_host, float* row_nll, double* nll_out,
                        cudaStream_t stream);
 
-cudaError_t launch_select_across(const Plan& p, const float* scores, int* idx, int* head_offsets, uint32_t* thr,
-                                 int* ties, cudaStream_t stream);
+// Scratch of the selection that spreads a score vector over several CTAs (select.cu).  A group is what
+// shares a threshold: one unit, or, when selecting across heads, a (layer, sequence) pair with all its heads.
+constexpr int kSelStateInts = 2176;       // per group: 2048 histogram bins, range, counters, per-head counts
+constexpr int kSelCandBase = 4096;        // candidate capacity of a group: this + (scores of the group) / kSelCandDiv
+constexpr int kSelCandDiv = 256;
+struct MultiSelect {
+    int* state;                // [groups][kSelStateInts]
+    uint2* cand;               // (key, head) pairs; a group's list starts where decode_group() says
+    int2* counts;              // [units][parts]: scores above / at the threshold per slice
+    uint32_t* thr;             // [groups]
+    int* ties;                 // [units]
+    long long cand_per_outer;  // list entries per layer (across heads) or per (layer, head)
+    int parts;                 // slices per score vector
+    int across;
+};
+struct MultiSelectLayout {
+    size_t off_state, off_cand, off_counts, off_thr, off_ties, total;
+    long long cand_per_outer;
+};
+// Offsets (relative to a 256-byte aligned base) of the scratch for the given problem.
+inline MultiSelectLayout multi_select_layout(int layers, int heads, int batch, long long total_tokens, bool across,
+                                             int parts) {
+    auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+    const size_t outer = across ? (size_t)layers : (size_t)layers * heads;
+    const size_t groups = outer * batch, units = (size_t)layers * heads * batch;
+    MultiSelectLayout l;
+    l.cand_per_outer = (long long)batch * (kSelCandBase + 1) + ((long long)(across ? heads : 1) * total_tokens) / kSelCandDiv + 1;
+    size_t off = 0;
+    l.off_state = off;  off += up(sizeof(int) * groups * kSelStateInts);
+    l.off_cand = off;   off += up(sizeof(uint2) * outer * (size_t)l.cand_per_outer);
+    l.off_counts = off; off += up(sizeof(int2) * units * (size_t)parts);
+    l.off_thr = off;    off += up(sizeof(uint32_t) * groups);
+    l.off_ties = off;   off += up(sizeof(int) * units);
+    l.total = off;
+    return l;
+}
+inline MultiSelect multi_select_at(char* base, const MultiSelectLayout& l, int parts, bool across) {
+    MultiSelect m;
+    m.state = reinterpret_cast<int*>(base + l.off_state);
+    m.cand = reinterpret_cast<uint2*>(base + l.off_cand);
+    m.counts = reinterpret_cast<int2*>(base + l.off_counts);
+    m.thr = reinterpret_cast<uint32_t*>(base + l.off_thr);
+    m.ties = reinterpret_cast<int*>(base + l.off_ties);
+    m.cand_per_outer = l.cand_per_outer;
+    m.parts = parts;
+    m.across = across ? 1 : 0;
+    return m;
+}
+cudaError_t launch_select_multi(const Plan& p, const float* scores, int* idx, int* head_offsets, const MultiSelect& m,
+                                cudaStream_t stream);
 cudaError_t launch_compact_across(const Plan& p, const Mat& k, const Mat& v, const int* idx, const int* head_offsets,
                                   __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream);
 cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_per_kv, float scale, int pool,

@@ -130,6 +130,51 @@ __device__ uint32_t radix_select(SelectSmem& s, int want, int* ties, Visit visit
     return prefix;
 }
 
+// Value range of a score vector from its first kSample entries: leaves in shared memory the lower end,
+// the scale that maps the sampled range onto bins 1 .. kBins-2, and `fallback` when the sample is not
+// finite or has no width.  Every CTA that is given the same sample arrives at the same numbers.
+__device__ void compute_range(SelectSmem& s, const float* __restrict__ sample, int n_sample) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float lo = INFINITY, hi = -INFINITY;
+    bool finite = true;
+    float smp[kSample / kThreads];
+#pragma unroll
+    for (int u = 0; u < kSample / kThreads; ++u) {
+        const int i = u * kThreads + tid;
+        smp[u] = sample[i < n_sample ? i : 0];
+    }
+#pragma unroll
+    for (int u = 0; u < kSample / kThreads; ++u) {
+        finite = finite && isfinite(smp[u]);
+        lo = fminf(lo, smp[u]); hi = fmaxf(hi, smp[u]);
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+    }
+    const int all_finite = __syncthreads_and(finite ? 1 : 0);
+    if (lane == 0) { s.red[0][warp] = lo; s.red[1][warp] = hi; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < kWarps; ++w) { lo = fminf(lo, s.red[0][w]); hi = fmaxf(hi, s.red[1][w]); }
+        const float width = hi - lo;
+        const float scale = (float)(kBins - 2) / width;              // sampled range -> bins 1 .. kBins-2
+        s.fallback = !(all_finite && width > 0.f && isfinite(width) && isfinite(scale));
+        s.lo = lo;
+        s.scale = s.fallback ? 0.f : scale;
+        s.n_cand = 0;
+    }
+    __syncthreads();
+}
+
+// Bin of a score: monotone in v (subtraction, multiplication by a positive constant, clamping and
+// truncation all are), so the bins order the scores exactly; values outside the sampled range land in
+// the end bins.
+__device__ __forceinline__ int bin_of(float v, float lo, float scale) {
+    return (int)fminf(fmaxf((v - lo) * scale + 1.0f, 0.0f), (float)(kBins - 1));
+}
+
 // Key of the `want`-th largest of the values that `visit(f)` enumerates (f(value) is called once per
 // value, in any order, by any thread), and through *ties how many values equal to that key belong
 // to the top `want`.  `sample` / `n_sample` are some of the values, used to guess their range.
@@ -137,49 +182,12 @@ template <class Visit>
 __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __restrict__ sample, int n_sample,
                                    int want_total, int* ties, bool* all_finite_out = nullptr) {
     if (all_finite_out != nullptr) *all_finite_out = false;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // ---- value range from a sample ------------------------------------------------------------
-    {
-        float lo = INFINITY, hi = -INFINITY;
-        bool finite = true;
-        float smp[kSample / kThreads];
-#pragma unroll
-        for (int u = 0; u < kSample / kThreads; ++u) {
-            const int i = u * kThreads + tid;
-            smp[u] = sample[i < n_sample ? i : 0];
-        }
-#pragma unroll
-        for (int u = 0; u < kSample / kThreads; ++u) {
-            finite = finite && isfinite(smp[u]);
-            lo = fminf(lo, smp[u]); hi = fmaxf(hi, smp[u]);
-        }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
-            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
-        }
-        const int all_finite = __syncthreads_and(finite ? 1 : 0);
-        if (lane == 0) { s.red[0][warp] = lo; s.red[1][warp] = hi; }
-        __syncthreads();
-        if (tid == 0) {
-            for (int w = 1; w < kWarps; ++w) { lo = fminf(lo, s.red[0][w]); hi = fmaxf(hi, s.red[1][w]); }
-            const float width = hi - lo;
-            const float scale = (float)(kBins - 2) / width;              // sampled range -> bins 1 .. kBins-2
-            s.fallback = !(all_finite && width > 0.f && isfinite(width) && isfinite(scale));
-            s.lo = lo;
-            s.scale = s.fallback ? 0.f : scale;
-            s.n_cand = 0;
-        }
-        __syncthreads();
-    }
+    const int tid = threadIdx.x;
+    compute_range(s, sample, n_sample);
 
     if (!s.fallback) {
         const float lo = s.lo, scale = s.scale;
-        // monotone in v: subtraction, multiplication by a positive constant, clamping and truncation all are
-        auto bin_of = [&](float v) {
-            const float x = fminf(fmaxf((v - lo) * scale + 1.0f, 0.0f), (float)(kBins - 1));
-            return (int)x;
-        };
+        auto bin_of = [&](float v) { return compactor::bin_of(v, lo, scale); };
         for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
         __syncthreads();
         int nonfinite = 0;
@@ -218,9 +226,11 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
 // The pass is bound by instruction issue, hence four scores per load and per scan.
 // kPlain: every score is known to be finite, so that comparing the floats themselves orders them as the
 // keys do (and -0 == +0 either way); that saves the key mapping, which is most of the work per score.
+// A CTA may be given a slice of the vector: `index_base` is the index of sc[0] in the whole vector and
+// gt0 / eq0 count the scores above / at the threshold that precede the slice.
 template <bool kPlain>
 __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n, uint32_t thr, int ties,
-                             int* __restrict__ out) {
+                             int* __restrict__ out, int index_base = 0, int gt0 = 0, int eq0 = 0) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int head = min(n, (int)((4 - ((reinterpret_cast<uintptr_t>(sc) >> 2) & 3)) & 3));
     const int n_vec = (n - head) >> 2;
@@ -281,17 +291,17 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
             const int t_eq = __shfl_up_sync(0xffffffffu, incl_eq, off);
             if (lane >= off) { incl_gt += t_gt; incl_eq += t_eq; }
         }
-        base_gt = head_gt + __shfl_sync(0xffffffffu, incl_gt - c_gt, warp);  // exclusive prefixes of this warp
-        base_eq = head_eq + __shfl_sync(0xffffffffu, incl_eq - c_eq, warp);
+        base_gt = gt0 + head_gt + __shfl_sync(0xffffffffu, incl_gt - c_gt, warp);  // exclusive prefixes of this warp
+        base_eq = eq0 + head_eq + __shfl_sync(0xffffffffu, incl_eq - c_eq, warp);
     }
 
     // ---- emission: head, stretches, tail ----------------------------------------------------------
     if (tid == 0) {
-        int g = 0, e = 0;
+        int g = gt0, e = eq0;
         for (int i = 0; i < head; ++i) {
             const uint32_t key = order_key(sc[i]);
-            if (key > thr) out[g + min(e, ties)] = i;
-            else if (key == thr && e < ties) out[g + e] = i;
+            if (key > thr) out[g + min(e, ties)] = index_base + i;
+            else if (key == thr && e < ties) out[g + e] = index_base + i;
             g += key > thr; e += key == thr;
         }
     }
@@ -317,7 +327,7 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
             }
             int gt_before = base_gt + ((incl - mine) & 0xffff);
             int eq_before = base_eq + ((incl - mine) >> 16);
-            const int i0 = head + 4 * vi;
+            const int i0 = index_base + head + 4 * vi;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 if ((g >> j) & 1) { out[gt_before + min(eq_before, ties)] = i0 + j; ++gt_before; }
@@ -331,8 +341,8 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
     if (warp == kWarps - 1 && lane == 0) {                // the tail follows the last stretch
         for (int i = tail_begin; i < n; ++i) {
             const uint32_t key = order_key(sc[i]);
-            if (key > thr) out[base_gt + min(base_eq, ties)] = i;
-            else if (key == thr && base_eq < ties) out[base_gt + base_eq] = i;
+            if (key > thr) out[base_gt + min(base_eq, ties)] = index_base + i;
+            else if (key == thr && base_eq < ties) out[base_gt + base_eq] = index_base + i;
             base_gt += key > thr; base_eq += key == thr;
         }
     }
@@ -360,53 +370,222 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
     else emit_ordered<false>(s, sc, n, thr, ties, out);
 }
 
-// ---- selection across the heads of a layer (Section 3.4's alternative) -------------------------
-// Step 1, one CTA per (layer, sequence): the key of the (heads * kk)-th largest score over all heads,
-// how many scores each head keeps (ties go to the lower head first, then to the lower index), and
-// the heads' offsets inside the sequence's block of the output.
+// ---- selection spread over several CTAs -----------------------------------------------------------
+// Used where one CTA per score vector leaves most of the GPU idle: selection across the heads of a
+// layer (Section 3.4's alternative: one threshold per layer and sequence over heads * n scores) and
+// per-head selection of a few long sequences.  A "group" is what shares a threshold: a (layer,
+// sequence) pair with all its heads, or one unit.  Every head's vector is cut into `parts` slices,
+// one CTA each:
+//   1. histogram: the group's value range from the first scores of its first head (every CTA arrives
+//      at the same numbers), a value-linear histogram of the slice in shared memory, added into the
+//      group's histogram in global memory;
+//   2. candidates: every CTA finds the threshold bin in the finished histogram, appends the slice's
+//      members of that bin as (key, head) pairs to the group's list and counts, per head, the scores in
+//      higher bins;
+//   3. finalize, one CTA per group: exact radix select among the candidates, per-head counts above
+//      and at the threshold (ties go to the lower head first, then to the lower index), the heads'
+//      offsets.  Groups whose scores defeat the histogram (non-finite values, no spread, an overfull
+//      bin) are redone here by one CTA over all scores, as the single-CTA selection would;
+//      it also turns the candidates into per-slice counts of scores above / at the threshold;
+//   4. ordered emission of every slice at its offset.
+// Per-group scratch words: histogram, range, candidate counter, flags, per-head counts.
+constexpr int kStLo = kBins, kStScale = kBins + 1, kStCand = kBins + 2, kStFlags = kBins + 3, kStAbove = kBins + 4;
+static_assert(kStAbove + 64 <= kSelStateInts, "per-group scratch too small");
+static_assert(kCand / 2 >= 64 * 64, "per-slice counts of a group live in the candidate array");
+
+struct Slice {
+    int part, unit, b, lh, layer, head;
+    int group, hg, hi;         // group index, heads per group, this head's index inside the group
+    int n, kk, begin, end;     // the slice is [begin, end) of the unit's n scores
+    long long cand_begin;      // the group's candidate list
+    int cand_cap;
+};
+
+__device__ __forceinline__ Slice decode_group(const Plan& p, const MultiSelect& m, int group) {
+    Slice c;
+    c.b = group % p.batch;
+    const int outer = group / p.batch;
+    c.group = group;
+    c.hg = m.across ? p.heads : 1;
+    c.layer = m.across ? outer : outer / p.heads;
+    c.head = m.across ? 0 : outer % p.heads;
+    c.lh = c.layer * p.heads + c.head;
+    c.hi = 0;
+    c.unit = c.lh * p.batch + c.b;
+    c.n = p.cu_seqlens[c.b + 1] - p.cu_seqlens[c.b];
+    c.kk = p.cu_keep[c.b + 1] - p.cu_keep[c.b];
+    c.part = 0; c.begin = 0; c.end = c.n;
+    c.cand_begin = (long long)outer * m.cand_per_outer + (long long)c.b * (kSelCandBase + 1) +
+                   ((long long)c.hg * p.cu_seqlens[c.b]) / kSelCandDiv;
+    c.cand_cap = kSelCandBase + (int)(((long long)c.hg * c.n) / kSelCandDiv);
+    return c;
+}
+
+__device__ __forceinline__ Slice decode_slice(const Plan& p, const MultiSelect& m, int block) {
+    const int part = block % m.parts, unit = block / m.parts;
+    const int b = unit % p.batch, lh = unit / p.batch;
+    const int layer = lh / p.heads, head = lh % p.heads;
+    Slice c = decode_group(p, m, m.across ? layer * p.batch + b : unit);
+    c.part = part; c.unit = unit; c.lh = lh; c.head = head;
+    c.hi = m.across ? head : 0;
+    const int len = (((c.n + m.parts - 1) / m.parts) + 3) & ~3;
+    c.begin = min(c.n, part * len);
+    c.end = min(c.n, c.begin + len);
+    return c;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
-across_threshold_kernel(Plan p, const float* __restrict__ scores, uint32_t* __restrict__ thr_out,
-                        int* __restrict__ ties_out, int* __restrict__ head_offsets) {
+multi_hist_kernel(Plan p, const float* __restrict__ scores, MultiSelect m) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    const Slice c = decode_slice(p, m, blockIdx.x);
+    if (c.kk <= 0 || c.n <= 0 || c.kk >= c.n) return;
+    const int tid = threadIdx.x;
+    int* st = m.state + (size_t)c.group * kSelStateInts;
+    const float* first = scores + (size_t)(c.lh - c.hi) * p.total_tokens + p.cu_seqlens[c.b];   // the group's first head
+    compute_range(s, first, c.n);
+    if (s.fallback) {
+        if (tid == 0) atomicOr(&st[kStFlags], 1);
+        return;
+    }
+    const float lo = s.lo, scale = s.scale;
+    if (c.part == 0 && c.hi == 0 && tid == 0) { st[kStLo] = __float_as_int(lo); st[kStScale] = __float_as_int(scale); }
+    for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
+    __syncthreads();
+    int nonfinite = 0;
+    for_each_score(first + (size_t)c.hi * p.total_tokens + c.begin, c.end - c.begin, [&](float v) {
+        if (!isfinite(v)) nonfinite = 1;
+        atomicAdd(&s.hist[bin_of(v, lo, scale)], 1);
+    });
+    const int any_nonfinite = __syncthreads_or(nonfinite);
+    for (int i = tid; i < kBins; i += kThreads)
+        if (s.hist[i] != 0) atomicAdd(&st[i], s.hist[i]);
+    if (any_nonfinite && tid == 0) atomicOr(&st[kStFlags], 1);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+multi_candidates_kernel(Plan p, const float* __restrict__ scores, MultiSelect m) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    const Slice c = decode_slice(p, m, blockIdx.x);
+    if (c.kk <= 0 || c.n <= 0 || c.kk >= c.n) return;
+    const int tid = threadIdx.x, lane = tid & 31;
+    int* st = m.state + (size_t)c.group * kSelStateInts;
+    if ((st[kStFlags] & 1) != 0) return;                  // set by the histogram pass: the same for every CTA of the group
+    const float lo = __int_as_float(st[kStLo]), scale = __int_as_float(st[kStScale]);
+    for (int i = tid; i < kBins; i += kThreads) s.hist[i] = st[i];
+    if (tid == 0) s.n_cand = 0;                           // here: the slice's scores in bins above the threshold bin
+    __syncthreads();
+    pick_bin(s, kBins, c.hg * c.kk);
+    const int tbin = s.bin;
+    if (s.hist[tbin] > c.cand_cap) {                      // every CTA of the group sees the same histogram
+        if (tid == 0) atomicOr(&st[kStFlags], 2);
+        return;
+    }
+    uint2* cand = m.cand + c.cand_begin;
+    int above = 0;
+    for_each_score(scores + (size_t)c.lh * p.total_tokens + p.cu_seqlens[c.b] + c.begin, c.end - c.begin, [&](float v) {
+        const int bin = bin_of(v, lo, scale);
+        above += bin > tbin;
+        if (bin == tbin) {
+            const int pos = atomicAdd(&st[kStCand], 1);
+            if (pos < c.cand_cap) cand[pos] = make_uint2(order_key(v), (uint32_t)(c.hi * m.parts + c.part));
+        }
+    });
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xffffffffu, above, d);
+    if (lane == 0 && above != 0) atomicAdd(&s.n_cand, above);       // zeroed by pick_bin's caller below
+    __syncthreads();
+    if (tid == 0) {
+        m.counts[blockIdx.x] = make_int2(s.n_cand, 0);
+        if (s.n_cand != 0) atomicAdd(&st[kStAbove + c.hi], s.n_cand);
+    }
+}
+
+// One CTA per group.  Writes the group's threshold key, every head's share of the ties and, when
+// selecting across heads, the heads' offsets inside the sequence's block of the output.
+__global__ void __launch_bounds__(kThreads, 1)
+multi_finalize_kernel(Plan p, const float* __restrict__ scores, MultiSelect m, int* __restrict__ head_offsets) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
     __shared__ int head_gt[64], head_eq[64];
-    const int layer = blockIdx.x / p.batch, b = blockIdx.x % p.batch;
-    const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
-    const int kk = p.cu_keep[b + 1] - p.cu_keep[b];
-    const int H = p.heads, tid = threadIdx.x;
-    int* offs = head_offsets + ((size_t)layer * p.batch + b) * (H + 1);
-    int* ties_h = ties_out + ((size_t)layer * p.batch + b) * H;
-    const float* base = scores + (size_t)layer * H * p.total_tokens + p.cu_seqlens[b];
+    const Slice c = decode_group(p, m, blockIdx.x);
+    const int H = c.hg, n = c.n, kk = c.kk, tid = threadIdx.x;
+    int* offs = head_offsets != nullptr ? head_offsets + (size_t)c.group * (H + 1) : nullptr;
+    auto unit_of = [&](int h) { return (c.lh + h) * p.batch + c.b; };
     if (kk <= 0 || n <= 0) {
-        for (int h = tid; h <= H; h += kThreads) offs[h] = 0;
+        if (offs != nullptr) for (int h = tid; h <= H; h += kThreads) offs[h] = 0;
         return;
     }
     if (kk >= n) {                                         // everything is kept
-        for (int h = tid; h <= H; h += kThreads) offs[h] = h * n;
-        for (int h = tid; h < H; h += kThreads) ties_h[h] = n;
-        if (tid == 0) thr_out[blockIdx.x] = 0u;           // every key is >= 0: all scores count as ties or above
+        if (offs != nullptr) for (int h = tid; h <= H; h += kThreads) offs[h] = h * n;
+        for (int h = tid; h < H; h += kThreads) m.ties[unit_of(h)] = n;
+        if (tid == 0) m.thr[c.group] = 0u;                 // every key is >= 0: all scores count as ties or above
         return;
     }
-    auto visit_all = [&](auto f) {
-        for (int h = 0; h < H; ++h) for_each_score(base + (size_t)h * p.total_tokens, n, f);
-    };
+    int* st = m.state + (size_t)c.group * kSelStateInts;
+    const float* base = scores + (size_t)c.lh * p.total_tokens + p.cu_seqlens[c.b];
+    // scores above / at the threshold per slice of the group (head-major), so that a slice can be emitted on its own;
+    // they live where the single-CTA route keeps its candidates (at most 64 heads x 64 slices)
+    int* slice_gt = reinterpret_cast<int*>(s.cand);
+    int* slice_eq = slice_gt + kCand / 2;
+    const int n_slices = H * m.parts;
+    const bool fast = st[kStFlags] == 0;
     int ties = 0;
-    const uint32_t thr = find_threshold(s, visit_all, base, n, H * kk, &ties);
-    // per-head counts above and at the threshold
-    for (int h = tid; h < H; h += kThreads) { head_gt[h] = 0; head_eq[h] = 0; }
-    __syncthreads();
-    for (int h = 0; h < H; ++h) {
-        int gt = 0, eq = 0;
-        for_each_score(base + (size_t)h * p.total_tokens, n, [&](float v) {
-            const uint32_t key = order_key(v);
-            gt += key > thr; eq += key == thr;
+    uint32_t thr;
+    if (fast) {
+        for (int i = tid; i < kBins; i += kThreads) s.hist[i] = st[i];
+        for (int i = tid; i < n_slices; i += kThreads) { slice_gt[i] = 0; slice_eq[i] = 0; }
+        __syncthreads();
+        pick_bin(s, kBins, H * kk);
+        const int want = s.remaining;
+        const int nc = min(st[kStCand], c.cand_cap);
+        const uint2* cand = m.cand + c.cand_begin;
+        __syncthreads();
+        thr = radix_select(s, want, &ties, [&](auto tally) {
+            for (int i = tid; i < nc; i += kThreads) tally(cand[i].x);
         });
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            gt += __shfl_xor_sync(0xffffffffu, gt, d);
-            eq += __shfl_xor_sync(0xffffffffu, eq, d);
+        for (int i = tid; i < nc; i += kThreads) {
+            const uint2 e = cand[i];
+            if (e.x > thr) atomicAdd(&slice_gt[e.y], 1);
+            else if (e.x == thr) atomicAdd(&slice_eq[e.y], 1);
         }
-        if ((tid & 31) == 0) { atomicAdd(&head_gt[h], gt); atomicAdd(&head_eq[h], eq); }
+        __syncthreads();
+    } else {
+        auto visit_all = [&](auto f) {
+            for (int h = 0; h < H; ++h) for_each_score(base + (size_t)h * p.total_tokens, n, f);
+        };
+        thr = find_threshold(s, visit_all, base, n, H * kk, &ties);
+        __syncthreads();
+        for (int i = tid; i < n_slices; i += kThreads) { slice_gt[i] = 0; slice_eq[i] = 0; }
+        __syncthreads();
+        const int len = (((n + m.parts - 1) / m.parts) + 3) & ~3;
+        for (int i = 0; i < n_slices; ++i) {
+            const int h = i / m.parts, part = i % m.parts;
+            const int begin = min(n, part * len), end = min(n, begin + len);
+            int gt = 0, eq = 0;
+            for_each_score(base + (size_t)h * p.total_tokens + begin, end - begin, [&](float v) {
+                const uint32_t key = order_key(v);
+                gt += key > thr; eq += key == thr;
+            });
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                gt += __shfl_xor_sync(0xffffffffu, gt, d);
+                eq += __shfl_xor_sync(0xffffffffu, eq, d);
+            }
+            if ((tid & 31) == 0) { atomicAdd(&slice_gt[i], gt); atomicAdd(&slice_eq[i], eq); }
+        }
+        __syncthreads();
+    }
+    for (int i = tid; i < n_slices; i += kThreads) {
+        int2* dst = &m.counts[(size_t)unit_of(i / m.parts) * m.parts + i % m.parts];
+        const int above = fast ? dst->x : 0;               // left there by the candidates pass
+        *dst = make_int2(above + slice_gt[i], slice_eq[i]);
+    }
+    for (int h = tid; h < H; h += kThreads) {
+        int gt = fast ? st[kStAbove + h] : 0, eq = 0;
+        for (int q = 0; q < m.parts; ++q) { gt += slice_gt[h * m.parts + q]; eq += slice_eq[h * m.parts + q]; }
+        head_gt[h] = gt; head_eq[h] = eq;
     }
     __syncthreads();
     if (tid == 0) {
@@ -414,38 +593,44 @@ across_threshold_kernel(Plan p, const float* __restrict__ scores, uint32_t* __re
         for (int h = 0; h < H; ++h) {
             const int take = min(left, head_eq[h]);
             left -= take;
-            ties_h[h] = take;
-            offs[h] = off;
+            m.ties[unit_of(h)] = take;
+            if (offs != nullptr) offs[h] = off;
             off += head_gt[h] + take;
         }
-        offs[H] = off;
-        thr_out[blockIdx.x] = thr;
+        if (offs != nullptr) offs[H] = off;
+        m.thr[c.group] = thr;
     }
 }
 
-// Step 2, one CTA per (layer, head, sequence): the head's kept indices, ascending.
+// One CTA per slice: the slice's kept indices, ascending, at their place in the head's output.
 __global__ void __launch_bounds__(kThreads, 1)
-across_emit_kernel(Plan p, const float* __restrict__ scores, const uint32_t* __restrict__ thr_in,
-                   const int* __restrict__ ties_in, const int* __restrict__ head_offsets, int* __restrict__ idx_out) {
+multi_emit_kernel(Plan p, const float* __restrict__ scores, MultiSelect m, const int* __restrict__ head_offsets,
+                  int* __restrict__ idx_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
-    const int unit = blockIdx.x;
-    const int b = unit % p.batch, lh = unit / p.batch;
-    const int layer = lh / p.heads, head = lh % p.heads;
-    const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
-    const int kk = p.cu_keep[b + 1] - p.cu_keep[b];
-    if (kk <= 0 || n <= 0) return;
-    const size_t lb = (size_t)layer * p.batch + b;
-    const int off = head_offsets[lb * (p.heads + 1) + head];
-    const int count = head_offsets[lb * (p.heads + 1) + head + 1] - off;
-    if (count <= 0) return;
-    const float* sc = scores + (size_t)lh * p.total_tokens + p.cu_seqlens[b];
-    int* out = idx_out + (size_t)layer * p.heads * p.total_keep + (size_t)p.heads * p.cu_keep[b] + off;
-    if (kk >= n) {
-        for (int i = threadIdx.x; i < n; i += kThreads) out[i] = i;
+    const Slice c = decode_slice(p, m, blockIdx.x);
+    if (c.kk <= 0 || c.n <= 0) return;
+    int* out;
+    if (m.across) {
+        const int* offs = head_offsets + (size_t)c.group * (p.heads + 1);
+        if (offs[c.head + 1] - offs[c.head] <= 0) return;
+        out = idx_out + (size_t)c.layer * p.heads * p.total_keep + (size_t)p.heads * p.cu_keep[c.b] + offs[c.head];
+    } else {
+        out = idx_out + (size_t)c.lh * p.total_keep + p.cu_keep[c.b];
+    }
+    if (c.kk >= c.n) {
+        for (int i = c.begin + threadIdx.x; i < c.end; i += kThreads) out[i] = i;
         return;
     }
-    emit_ordered<false>(s, sc, n, thr_in[lb], ties_in[lb * p.heads + head], out);
+    int gt0 = 0, eq0 = 0;
+    for (int q = 0; q < c.part; ++q) {
+        const int2 v = m.counts[(size_t)c.unit * m.parts + q];
+        gt0 += v.x; eq0 += v.y;
+    }
+    const float* sc = scores + (size_t)c.lh * p.total_tokens + p.cu_seqlens[c.b] + c.begin;
+    const bool plain = m.state[(size_t)c.group * kSelStateInts + kStFlags] == 0;     // every score was seen and is finite
+    if (plain) emit_ordered<true>(s, sc, c.end - c.begin, m.thr[c.group], m.ties[c.unit], out, c.begin, gt0, eq0);
+    else emit_ordered<false>(s, sc, c.end - c.begin, m.thr[c.group], m.ties[c.unit], out, c.begin, gt0, eq0);
 }
 
 // Eq. 6: s = z(a) + lambda z(o), population standard deviation, per unit.  Overwrites the
@@ -500,6 +685,102 @@ blend_kernel(Plan p, const float* __restrict__ attn, float lambda, float* __rest
         o[i] = (float)(((double)a[i] - mean_a) * inv_a + ((double)o[i] - mean_o) * inv_o);
 }
 
+// The blend for a few long units: every unit's vectors are cut into `parts` slices.  First kernel: mean and
+// sum of squared deviations of a and o per slice; second kernel: every CTA merges its unit's slices in a
+// fixed order (pairwise update of count, mean and squared deviations), then rewrites its own slice.
+__device__ __forceinline__ void block_sum2(double x, double y, double (*red)[kWarps], double* out) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        x += __shfl_xor_sync(0xffffffffu, x, d);
+        y += __shfl_xor_sync(0xffffffffu, y, d);
+    }
+    __syncthreads();                                      // earlier readers of red / out are done
+    if (lane == 0) { red[0][warp] = x; red[1][warp] = y; }
+    __syncthreads();
+    if (warp == 0) {
+        double u = red[0][lane], v = red[1][lane];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            u += __shfl_xor_sync(0xffffffffu, u, d);
+            v += __shfl_xor_sync(0xffffffffu, v, d);
+        }
+        if (lane == 0) { out[0] = u; out[1] = v; }
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ void blend_slice(int n, int parts, int part, int* begin, int* end) {
+    const int len = (n + parts - 1) / parts;
+    *begin = min(n, part * len);
+    *end = min(n, *begin + len);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+blend_stats_kernel(Plan p, const float* __restrict__ attn, const float* __restrict__ scores, int parts,
+                   double* __restrict__ stats) {
+    __shared__ double red[2][kWarps];
+    __shared__ double tot[2];
+    const int part = blockIdx.x % parts, unit = blockIdx.x / parts;
+    const int b = unit % p.batch, lh = unit / p.batch;
+    const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+    int begin, end;
+    blend_slice(n, parts, part, &begin, &end);
+    const int cnt = end - begin;
+    double* out = stats + (size_t)blockIdx.x * 4;
+    if (cnt <= 0) {
+        if (threadIdx.x < 4) out[threadIdx.x] = 0.0;
+        return;
+    }
+    const size_t off = (size_t)lh * p.total_tokens + p.cu_seqlens[b] + begin;
+    const float* a = attn + off;
+    const float* o = scores + off;
+    double sa = 0.0, so = 0.0;
+    for (int i = threadIdx.x; i < cnt; i += kThreads) { sa += (double)a[i]; so += (double)o[i]; }
+    block_sum2(sa, so, red, tot);
+    const double mean_a = tot[0] / cnt, mean_o = tot[1] / cnt;
+    double va = 0.0, vo = 0.0;
+    for (int i = threadIdx.x; i < cnt; i += kThreads) {
+        const double da = (double)a[i] - mean_a, d_o = (double)o[i] - mean_o;
+        va = fma(da, da, va); vo = fma(d_o, d_o, vo);
+    }
+    block_sum2(va, vo, red, tot);
+    if (threadIdx.x == 0) { out[0] = mean_a; out[1] = tot[0]; out[2] = mean_o; out[3] = tot[1]; }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+blend_apply_kernel(Plan p, const float* __restrict__ attn, float lambda, float* __restrict__ scores, int parts,
+                   const double* __restrict__ stats) {
+    const int part = blockIdx.x % parts, unit = blockIdx.x / parts;
+    const int b = unit % p.batch, lh = unit / p.batch;
+    const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+    int begin, end;
+    blend_slice(n, parts, part, &begin, &end);
+    if (end <= begin) return;
+    // every thread of every CTA of the unit merges the slices in the same order: the same statistics everywhere
+    double cnt = 0.0, mean_a = 0.0, m2_a = 0.0, mean_o = 0.0, m2_o = 0.0;
+    for (int q = 0; q < parts; ++q) {
+        int qb, qe;
+        blend_slice(n, parts, q, &qb, &qe);
+        const double c = (double)(qe - qb);
+        if (c <= 0.0) continue;
+        const double* st = stats + ((size_t)unit * parts + q) * 4;
+        const double tot = cnt + c;
+        const double da = st[0] - mean_a, d_o = st[2] - mean_o;
+        mean_a += da * (c / tot);  m2_a += st[1] + da * da * (cnt * c / tot);
+        mean_o += d_o * (c / tot); m2_o += st[3] + d_o * d_o * (cnt * c / tot);
+        cnt = tot;
+    }
+    const double sd_a = sqrt(m2_a / n), sd_o = sqrt(m2_o / n);
+    const double inv_a = sd_a > 0.0 ? 1.0 / sd_a : 0.0;
+    const double inv_o = sd_o > 0.0 ? (double)lambda / sd_o : 0.0;
+    const size_t off = (size_t)lh * p.total_tokens + p.cu_seqlens[b];
+    const float* a = attn + off;
+    float* o = scores + off;
+    for (int i = begin + threadIdx.x; i < end; i += kThreads)
+        o[i] = (float)(((double)a[i] - mean_a) * inv_a + ((double)o[i] - mean_o) * inv_o);
+}
+
 }  // namespace
 
 cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStream_t stream) {
@@ -512,26 +793,39 @@ cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStre
     return cudaGetLastError();
 }
 
-cudaError_t launch_select_across(const Plan& p, const float* scores, int* idx, int* head_offsets, uint32_t* thr,
-                                 int* ties, cudaStream_t stream) {
+cudaError_t launch_select_multi(const Plan& p, const float* scores, int* idx, int* head_offsets, const MultiSelect& m,
+                                cudaStream_t stream) {
     const int units = p.layers * p.heads * p.batch;
-    if (units == 0 || p.heads > 64) return units == 0 ? cudaSuccess : cudaErrorInvalidValue;
+    if (units == 0) return cudaSuccess;
+    if (m.parts < 1 || (m.across && (p.heads > 64 || head_offsets == nullptr))) return cudaErrorInvalidValue;
+    const int groups = m.across ? p.layers * p.batch : units;
     const int smem = (int)sizeof(SelectSmem);
-    cudaError_t e = cudaFuncSetAttribute(across_threshold_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(across_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    across_threshold_kernel<<<p.layers * p.batch, kThreads, smem, stream>>>(p, scores, thr, ties, head_offsets);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    across_emit_kernel<<<units, kThreads, smem, stream>>>(p, scores, thr, ties, head_offsets, idx);
+    cudaError_t e;
+    if ((e = cudaFuncSetAttribute(multi_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(multi_candidates_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(multi_finalize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
+    if ((e = cudaFuncSetAttribute(multi_emit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(m.state, 0, sizeof(int) * (size_t)groups * kSelStateInts, stream)) != cudaSuccess) return e;
+    const unsigned slices = (unsigned)units * (unsigned)m.parts;
+    multi_hist_kernel<<<slices, kThreads, smem, stream>>>(p, scores, m);
+    multi_candidates_kernel<<<slices, kThreads, smem, stream>>>(p, scores, m);
+    multi_finalize_kernel<<<groups, kThreads, smem, stream>>>(p, scores, m, m.across ? head_offsets : nullptr);
+    if (p.total_keep > 0) {
+        multi_emit_kernel<<<slices, kThreads, smem, stream>>>(p, scores, m, head_offsets, idx);
+    }
     return cudaGetLastError();
 }
 
-cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* scores, cudaStream_t stream) {
+cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* scores, int parts, double* stats,
+                         cudaStream_t stream) {
     const int units = p.layers * p.heads * p.batch;
     if (units == 0 || p.total_tokens == 0) return cudaSuccess;
-    blend_kernel<<<units, kThreads, 0, stream>>>(p, attn, lambda, scores);
+    if (parts > 1 && stats != nullptr) {
+        blend_stats_kernel<<<units * parts, kThreads, 0, stream>>>(p, attn, scores, parts, stats);
+        blend_apply_kernel<<<units * parts, kThreads, 0, stream>>>(p, attn, lambda, scores, parts, stats);
+    } else {
+        blend_kernel<<<units, kThreads, 0, stream>>>(p, attn, lambda, scores);
+    }
     return cudaGetLastError();
 }
 

@@ -109,3 +109,18 @@ def test_across_heads_long_sequence_large_budget(B):
     s[0, 0] += 1.0                                         # the first head takes most of the budget
     s[0, 2] = np.round(s[0, 2], 1)
     _select_and_check(B, shape, torch.from_numpy(s).cuda(), [kk])
+
+
+def test_across_heads_scores_that_defeat_the_histogram(B):
+    # non-finite scores, and a bulk far narrower than the sampled range (every score in one bin): both groups are
+    # redone by one CTA over all scores, and the neighbouring well-behaved layer is not disturbed
+    rng = np.random.default_rng(6)
+    n = 90000
+    shape = B.Shape(3, 2, 128, 48, [n, 2000])
+    T = shape.total_tokens
+    s = rng.standard_normal((3, 2, T)).astype(np.float32)
+    s[0, 1, 5::11] = np.inf
+    s[0, 0, 6::13] = -np.inf
+    s[1] *= 1e-4
+    s[1, 0, 3] = 1000.0; s[1, 0, 9] = -1000.0              # the range estimate spans 2000, the bulk 1e-3
+    _select_and_check(B, shape, torch.from_numpy(s).cuda(), [30000, 700])

@@ -47,6 +47,14 @@ def test_c0_with_attention_blend(B):
     print(f"c0 blend: err {worst:.2e}")
 
 
+def test_blend_and_selection_of_a_few_long_units(B):
+    # two heads of one layer with a long and a short sequence: the blend's statistics and the selection are taken
+    # over slices of the long vectors by many CTAs; the result must still be the oracle's
+    w = inputs.Workload("few-long", 1, 2, 128, [140000, 300], [0.3, 0.5], p=0.7, seed=13)
+    worst, band, _ = _run_workload(B, w, attn=True, device="cuda")
+    print(f"few long units, blended: err {worst:.2e}")
+
+
 def test_ragged_small_sequences(B):
     # lengths around the tile, chunk and sketch sizes, including an empty sequence
     w = inputs.Workload("ragged-small", 2, 2, 128, [1000, 129, 0, 128, 127, 2500, 49, 300],
@@ -191,6 +199,40 @@ def test_select_long_sequences_and_large_keep_counts(B, n, keep):
     idx = idx.cpu().numpy()
     for h in range(2):
         np.testing.assert_array_equal(idx[0, h], orc.top_k_indices(s[0, h].astype(np.float64), keep), err_msg=f"head {h}")
+
+
+def test_select_few_long_units_spread_over_several_ctas(B):
+    # fewer units than SMs and long sequences: with the whole workspace the selection cuts every score vector into
+    # slices (shared histogram, candidate list, per-slice emission); with room for the tables only it runs one CTA
+    # per unit.  Both must give the oracle's indices.
+    rng = np.random.default_rng(17)
+    seqlens = [140000, 5, 40000, 0, 33001]
+    keep = [50000, 5, 1, 0, 33000]
+    L, Hh = 1, 3
+    shape = B.Shape(L, Hh, 128, 48, seqlens)
+    T = shape.total_tokens
+    cu = shape.cu_seqlens
+    s = rng.standard_normal((L, Hh, T)).astype(np.float32)
+    s[0, 1] = np.round(s[0, 1], 1)                       # heavy ties
+    s[0, 1, cu[2]:cu[3]] = 0.25                          # a constant sequence
+    s[0, 2, 5::11] = np.inf                              # non-finite scores: the slices fall back to one CTA
+    s[0, 2, 6::13] = -np.inf
+    s[0, 0, cu[4]:cu[5]] *= 1e-4                         # a bulk far narrower than the sampled range
+    s[0, 0, cu[4] + 3] = 1000.0
+    sc = torch.from_numpy(s).cuda()
+    ck = np.concatenate([[0], np.cumsum(keep)])
+    results = []
+    for ws in (B.alloc_workspace(shape), torch.empty(4096, dtype=torch.uint8, device="cuda")):
+        idx = torch.full((L, Hh, sum(keep)), -1, dtype=torch.int32, device="cuda")
+        B.select(shape, sc, keep, idx, ws)
+        torch.cuda.synchronize()
+        results.append(idx.cpu().numpy())
+    np.testing.assert_array_equal(results[0], results[1])
+    for h in range(Hh):
+        for b in range(len(seqlens)):
+            got = results[0][0, h, ck[b]:ck[b + 1]]
+            seg = s[0, h, cu[b]:cu[b + 1]].astype(np.float64)
+            np.testing.assert_array_equal(got, orc.top_k_indices(seg, keep[b]), err_msg=f"{h},{b}")
 
 
 def test_compact_bit_exact_and_skips_bad_indices(B):

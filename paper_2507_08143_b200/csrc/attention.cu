@@ -8,15 +8,17 @@
 // loads an item's keys once and streams the query heads' rows in halves of 128 through a two-slot ring
 // (TMA, 128-byte swizzle).  One thread of warp 1 issues, per half, S = Q_half K^T (tcgen05.mma,
 // 128 x 256 fp32) into one of two accumulators in tensor memory, so that the products of the next half
-// run beside the softmax of the current one.  Warps 2-9 share the 128 query rows (a pair of warps per
-// 32 rows, 128 keys each): row maximum, e = 2^(scale log2e (s - max)) written as fp16 into shared memory
+// run beside the softmax of the current one.  Warps 2-17 share the 128 query rows (four warps per
+// 32 rows, 64 keys each): row maximum, e = 2^(scale log2e (s - max)) written as fp16 into shared memory
 // in the layout of an MN-major operand, and the reciprocal of the row sum (two fp16 terms) into rows 0
 // and 1 of a small K-major operand w.  A second MMA, E^T w (keys x 2: the half's normalised column
-// sums), lands in 32 columns of the half's own S accumulator once the softmax warps are done with S; each
-// warp adds the sums of its 128 keys to a register per thread and writes them at the end of the item.
-// The softmax warps are bound by instruction issue and latency (two warps per scheduler), not by the
-// exponential unit: hence packed fp32x2 arithmetic, three-input maxima, tensor-memory loads one
-// step ahead, and the first exponentials of a half computed before the wait for the E buffer.
+// sums), lands in 32 columns of the half's own S accumulator once the softmax warps are done with S; two
+// warps of each four add the sums of 128 keys each to a register per thread and write them at the end of
+// the item.  The exponential phase runs at about 12 of the 16 exponentials per clock an SM can do, with the
+// issue slots and the half-rate integer pipe close to their limits as well (moving a share of the
+// exponentials to a polynomial on the FMA pipe made it slower): hence packed fp32x2 arithmetic,
+// three-input maxima, tensor-memory loads one step ahead, four warps per scheduler, and the first
+// exponentials of a half computed before the wait for the E buffer.
 #include <cuda_fp16.h>
 
 #include "common.cuh"
@@ -29,8 +31,8 @@ using namespace sm100;
 
 constexpr int kChunk = 256;
 constexpr int kHalf = 128;
-constexpr int kSoftmaxWarps = 8;           // two warps per query row quadrant: each takes 128 of the 256 keys
-constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
+constexpr int kSplitDefault = 4;
+constexpr int kMaxSplit = 4;               // softmax warps per query row quadrant (each takes 256 / split keys): 2 or 4
 constexpr int kKBox = kChunk * 128;        // 64 channels x 256 tokens x 2 B
 constexpr int kQBox = kHalf * 128;         // 64 channels x 128 rows
 constexpr int kPBlock = kHalf * 128;       // 128 rows x 64 keys, fp16
@@ -47,8 +49,8 @@ struct __align__(1024) AttnSmem {
     uint64_t p_ready;          // E and the weights of a half are in shared memory, its S is consumed
     uint64_t c_full[2];        // the half's column sums are in its accumulator; E and the weights may be overwritten
     uint64_t drained[2];       // the column sums have been taken out: the accumulator may be overwritten
-    float xmax[2][kHalf];      // row maxima / row sums of the two column halves, exchanged between warp pairs
-    float xsum[2][kHalf];
+    float xmax[kMaxSplit][kHalf];   // row maxima / row sums of the key ranges, exchanged between the warps of a quadrant
+    float xsum[kMaxSplit][kHalf];
     uint32_t tmem_base;
     int abort;
     int abort_mma;             // set by the MMA warp alone, before it wakes the softmax warps: they all see the same value
@@ -83,8 +85,9 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-__device__ __forceinline__ void softmax_pair_sync(int q) {     // the two warps that share 32 query rows
-    asm volatile("bar.sync %0, 64;" :: "r"(q + 1) : "memory");
+template <int kSplit>
+__device__ __forceinline__ void softmax_quad_sync(int q) {     // the warps that share 32 query rows
+    asm volatile("bar.sync %0, %1;" :: "r"(q + 1), "n"(32 * kSplit) : "memory");
 }
 
 // Where a work item (one chunk of one layer and KV head) lies.
@@ -103,11 +106,16 @@ __device__ __forceinline__ AttnItem attn_item(const Plan& p, int item) {
 
 // Persistent: CTA c takes items c, c + grid, ...; barriers, tensor memory and the zeroed weight operand are set
 // up once.  Halves are numbered through all of a CTA's items (g), which fixes every barrier's phase.
-__global__ void __launch_bounds__(kThreads, 1)
+template <int kSplit>
+__global__ void __launch_bounds__(64 + 128 * kSplit, 1)
 attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_constant__ CUtensorMap kmap,
                  int q_per_kv, float scale_log2e, int n_items, float* __restrict__ out, int* __restrict__ status) {
     extern __shared__ unsigned char smem_raw[];
     AttnSmem& s = *reinterpret_cast<AttnSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
+    constexpr int kSoftmaxWarps = 4 * kSplit;
+    constexpr int kThreads = 64 + 32 * kSoftmaxWarps;
+    constexpr int kCols = kChunk / kSplit;             // keys per softmax warp
+    constexpr int kStep = kCols / 4;                   // columns per tensor-memory load: 32 or 16
     const int n_iter = 2 * q_per_kv;                   // halves of 128 query rows per item (even)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int my_items = ((int)blockIdx.x < n_items) ? (n_items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
@@ -219,19 +227,22 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         }
     } else {
         const int q = warp & 3;                              // TMEM lane quadrant
-        const int ch = (warp - 2) >> 2;                      // which 128 of the 256 keys
+        const int ch = (warp - 2) >> 2;                      // which kCols of the 256 keys
         const int row = q * 32 + lane;                       // query row within the half = TMEM lane
         const uint32_t quad_addr = tmem + ((uint32_t)(q * 32) << 16);
         float col = 0.f;                                     // column sum of key ch * 128 + `row` (TMEM lane = key here)
-        auto take_column_sums = [&](int g) {                 // each warp takes the key half that it also exponentiates
-            uint32_t c[2];
-            tmem_ld_32x32b_x2(quad_addr + (uint32_t)(g & 1) * 256 + ch * 16, c);
-            tmem_ld_wait();
-            col += __uint_as_float(c[0]) + __uint_as_float(c[1]);        // hi and lo weights
+        // the sums of keys 0-127 and 128-255 lie in columns 0-15 and 16-31: the quadrant's first two warps take one each
+        auto take_column_sums = [&](int g) {
+            if (ch < 2) {
+                uint32_t c[2];
+                tmem_ld_32x32b_x2(quad_addr + (uint32_t)(g & 1) * 256 + ch * 16, c);
+                tmem_ld_wait();
+                col += __uint_as_float(c[0]) + __uint_as_float(c[1]);    // hi and lo weights
+            }
         };
         auto write_result = [&](const AttnItem& a) {         // an item's column sums are complete
             float* dst = out + (size_t)a.lh * p.total_tokens + a.tok_begin;
-            if (ch * kHalf + row < a.n_tok) dst[ch * kHalf + row] = col;
+            if (ch < 2 && ch * kHalf + row < a.n_tok) dst[ch * kHalf + row] = col;
             col = 0.f;
         };
         const int n_halves = my_items * n_iter;
@@ -250,50 +261,51 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             const bool full = n_tok == kChunk;               // only the last chunk of a sequence needs masks
             wait_ft(&s.s_full[g & 1], (g >> 1) & 1);
             tc_fence_after_sync();
-            const uint32_t lane_addr = quad_addr + (uint32_t)(g & 1) * 256 + ch * 128;
+            const uint32_t lane_addr = quad_addr + (uint32_t)(g & 1) * 256 + ch * kCols;
             const bool row_valid = (it & 1) * kHalf + row < n_tok;
             // the load of the next 32 columns is in flight while this thread works on the current ones
-            uint32_t ra[32], rb[32];
+            uint32_t ra[kStep], rb[kStep];
             float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            auto max_of = [&](const uint32_t (&x)[32], int c0) {
+            auto max_of = [&](const uint32_t (&x)[kStep], int c0) {
                 if (full) {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2)
+                    for (int i = 0; i < kStep; i += 2)
                         m4[(i >> 1) & 3] = max3(m4[(i >> 1) & 3], __uint_as_float(x[i]), __uint_as_float(x[i + 1]));
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (ch * 128 + c0 + i < n_tok) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(x[i]));
+                    for (int i = 0; i < kStep; ++i)
+                        if (ch * kCols + c0 + i < n_tok) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(x[i]));
                 }
             };
-            tmem_ld_32x32b_x32(lane_addr, ra);
+            tmem_ld_cols(lane_addr, ra);
             tmem_ld_wait_for(ra);
-            tmem_ld_32x32b_x32(lane_addr + 32, rb);
+            tmem_ld_cols(lane_addr + kStep, rb);
             max_of(ra, 0);
             tmem_ld_wait_for(rb);
-            tmem_ld_32x32b_x32(lane_addr + 64, ra);
-            max_of(rb, 32);
+            tmem_ld_cols(lane_addr + 2 * kStep, ra);
+            max_of(rb, kStep);
             tmem_ld_wait_for(ra);
-            tmem_ld_32x32b_x32(lane_addr + 96, rb);
-            max_of(ra, 64);
+            tmem_ld_cols(lane_addr + 3 * kStep, rb);
+            max_of(ra, 2 * kStep);
             tmem_ld_wait_for(rb);
-            max_of(rb, 96);
+            max_of(rb, 3 * kStep);
             s.xmax[ch][row] = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-            softmax_pair_sync(q);
-            const float mx = fmaxf(s.xmax[0][row], s.xmax[1][row]);      // finite: key 0 of the chunk always exists
+            softmax_quad_sync<kSplit>(q);
+            float mx = fmaxf(s.xmax[0][row], s.xmax[1][row]);            // finite: key 0 of the chunk always exists
+            if (kSplit == 4) mx = fmaxf(mx, fmaxf(s.xmax[2][row], s.xmax[3][row]));
             const float bias = -mx * scale_log2e;
             uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};     // four pairs of partial row sums
             const uint64_t scale2 = pack2(scale_log2e, scale_log2e), bias2 = pack2(bias, bias);
-            uint32_t packed[16];
-            auto exp_of = [&](const uint32_t (&r)[32], int c0) {
+            uint32_t packed[kStep / 2];
+            auto exp_of = [&](const uint32_t (&r)[kStep], int c0) {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) {
+                for (int i = 0; i < kStep; i += 2) {
                     float y0, y1;
                     unpack2(fma2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), scale2, bias2), y0, y1);
                     float e0 = ex2_approx(y0), e1 = ex2_approx(y1);
                     if (!full) {
-                        if (!row_valid || ch * 128 + c0 + i >= n_tok) e0 = 0.f;
-                        if (!row_valid || ch * 128 + c0 + i + 1 >= n_tok) e1 = 0.f;
+                        if (!row_valid || ch * kCols + c0 + i >= n_tok) e0 = 0.f;
+                        if (!row_valid || ch * kCols + c0 + i + 1 >= n_tok) e1 = 0.f;
                     }
                     sum2[(i >> 1) & 3] = add2(sum2[(i >> 1) & 3], pack2(e0, e1));
                     const __half2 h = __floats2half2_rn(e0, e1);
@@ -301,18 +313,18 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                 }
             };
             auto store = [&](int c0) {
-                const int col = ch * 128 + c0;
+                const int col = ch * kCols + c0;
                 unsigned char* blk = s.p + (col >> 6) * kPBlock + row * 128;
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < kStep / 8; ++j) {
                     const int piece = ((col & 63) >> 3) + j;
                     *reinterpret_cast<uint4*>(blk + ((piece ^ (row & 7)) << 4)) =
                         make_uint4(packed[4 * j], packed[4 * j + 1], packed[4 * j + 2], packed[4 * j + 3]);
                 }
             };
-            tmem_ld_32x32b_x32(lane_addr, ra);
+            tmem_ld_cols(lane_addr, ra);
             tmem_ld_wait_for(ra);
-            tmem_ld_32x32b_x32(lane_addr + 32, rb);
+            tmem_ld_cols(lane_addr + kStep, rb);
             exp_of(ra, 0);                                   // the first exponentials need no room in shared memory yet
             if (g > 0) {
                 // E and the weights of the previous half have been multiplied: they may be overwritten,
@@ -322,30 +334,31 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
                 take_column_sums(g - 1);
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&s.drained[(g - 1) & 1]);
+                if (lane == 0 && ch < 2) mbar_arrive(&s.drained[(g - 1) & 1]);
                 if (it == 0) write_result(prev);             // that was the last half of the previous item
             }
             store(0);
             tmem_ld_wait_for(rb);
-            tmem_ld_32x32b_x32(lane_addr + 64, ra);
-            exp_of(rb, 32);
-            store(32);
+            tmem_ld_cols(lane_addr + 2 * kStep, ra);
+            exp_of(rb, kStep);
+            store(kStep);
             tmem_ld_wait_for(ra);
-            tmem_ld_32x32b_x32(lane_addr + 96, rb);
-            exp_of(ra, 64);
-            store(64);
+            tmem_ld_cols(lane_addr + 3 * kStep, rb);
+            exp_of(ra, 2 * kStep);
+            store(2 * kStep);
             tmem_ld_wait_for(rb);
-            exp_of(rb, 96);
-            store(96);
+            exp_of(rb, 3 * kStep);
+            store(3 * kStep);
             {
                 float lo, hi;
                 unpack2(add2(add2(sum2[0], sum2[1]), add2(sum2[2], sum2[3])), lo, hi);
                 s.xsum[ch][row] = lo + hi;
             }
-            softmax_pair_sync(q);
+            softmax_quad_sync<kSplit>(q);
             if (ch == 0) {
                 // 1 / (row sum) as two fp16 terms in rows 0 and 1 of the weight operand (row 1 is swizzled by its index)
-                const float sum = s.xsum[0][row] + s.xsum[1][row];
+                float sum = s.xsum[0][row] + s.xsum[1][row];
+                if (kSplit == 4) sum += s.xsum[2][row] + s.xsum[3][row];
                 const float wgt = (row_valid && sum > 0.f) ? 1.0f / sum : 0.f;
                 const __half w_hi = __float2half_rn(wgt);
                 const __half w_lo = __float2half_rn(wgt - __half2float(w_hi));
@@ -404,16 +417,18 @@ cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_pe
                             k.stride_token, kChunk))
         return cudaErrorInvalidValue;
     const int smem = (int)sizeof(AttnSmem) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
     float* dst = pool > 1 ? raw : out;
     const long long n_items = (long long)p.total_chunks * p.layers * p.heads;
     if (n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
     int dev = 0, n_sm = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
     const int grid = (int)(n_items < n_sm ? n_items : n_sm);          // one CTA per SM (shared memory)
-    attention_kernel<<<grid, kThreads, smem, stream>>>(p, qmap, kmap, q_per_kv, scale * 1.4426950408889634f,
-                                                       (int)n_items, dst, status);
+    cudaError_t e = cudaFuncSetAttribute(attention_kernel<kSplitDefault>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    attention_kernel<kSplitDefault><<<grid, 64 + 128 * kSplitDefault, smem, stream>>>(
+        p, qmap, kmap, q_per_kv, scale * 1.4426950408889634f, (int)n_items, dst, status);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess || pool <= 1) return e;
     pool_kernel<<<dim3((p.total_tokens + 255) / 256, p.layers * p.heads), 256, 0, stream>>>(p, raw, out, pool);

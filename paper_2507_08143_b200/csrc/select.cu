@@ -33,8 +33,10 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 struct SelectSmem {
     int hist[kBins];
     uint32_t cand[kCand];
+    unsigned char cand_warp[kCand];   // which warp's stretch a candidate lies in (255: the unaligned head or tail)
     int cnt[2][kSub][kWarps];      // per-warp packed counts of the ordered pass, double buffered
     int row_total[2][kSub];
+    int stage[kWarps][512];        // kept indices of 4 x 128 scores per warp, in output order
     int warp_sums[kWarps];
     float red[2][kWarps];
     int bin;          // chosen bin of the current pass
@@ -169,10 +171,11 @@ __device__ void compute_range(SelectSmem& s, const float* __restrict__ sample, i
 }
 
 // Bin of a score: monotone in v (subtraction, multiplication by a positive constant, clamping and
-// truncation all are), so the bins order the scores exactly; values outside the sampled range land in
+// rounding all are; the rounding is an addition, cheaper than a float-to-int conversion), so the bins order the scores exactly; values outside the sampled range land in
 // the end bins.
 __device__ __forceinline__ int bin_of(float v, float lo, float scale) {
-    return (int)fminf(fmaxf((v - lo) * scale + 1.0f, 0.0f), (float)(kBins - 1));
+    const float x = fminf(fmaxf((v - lo) * scale + 1.0f, 0.0f), (float)(kBins - 1));
+    return __float_as_int(x + 8388608.0f) & (2 * kBins - 1);   // round to nearest: at 2^23 the integer sits in the low mantissa bits
 }
 
 // Key of the `want`-th largest of the values that `visit(f)` enumerates (f(value) is called once per
@@ -217,6 +220,104 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
     });
 }
 
+// The threshold of one finite score vector together with what the ordered pass needs to start: per warp
+// stretch (the same cut as emit_ordered's) the number of scores above and at the threshold.  First pass:
+// the value-linear histogram (this is the pass that brings the scores in from HBM).  Second pass: a warp
+// counts the scores of its stretch in bins above the threshold bin and lists the members of that bin
+// with its own number; once the exact key is known among the listed ones, they are added to the counts
+// of their warps, so the ordered pass need not count again.  Returns false (and has written nothing that
+// matters) when the histogram route does not apply: the caller then takes find_threshold and the
+// counting emit_ordered.
+__device__ bool threshold_with_counts(SelectSmem& s, const float* __restrict__ sc, int n, int want_total,
+                                      uint32_t* thr_out, int* ties_out) {
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    compute_range(s, sc, n);
+    if (s.fallback) return false;
+    const float lo = s.lo, scale = s.scale;
+    for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
+    __syncthreads();
+    int nonfinite = 0;
+    for_each_score(sc, n, [&](float v) {
+        if (!isfinite(v)) nonfinite = 1;
+        atomicAdd(&s.hist[bin_of(v, lo, scale)], 1);
+    });
+    const int any_nonfinite = __syncthreads_or(nonfinite);
+    pick_bin(s, kBins, want_total);
+    const int tbin = s.bin, want = s.remaining;
+    const int members = s.hist[tbin];
+    __syncthreads();
+    if (any_nonfinite || members > kCand) return false;
+
+    const int head = min(n, (int)((4 - ((reinterpret_cast<uintptr_t>(sc) >> 2) & 3)) & 3));
+    const int n_vec = (n - head) >> 2;
+    const float4* body = reinterpret_cast<const float4*>(sc + head);
+    const int per_warp = (((n_vec + kWarps - 1) / kWarps) + 31) & ~31;
+    const int vbegin = min(n_vec, warp * per_warp), vend = min(n_vec, vbegin + per_warp);
+    auto candidate = [&](float v, int tag) {
+        const int pos = atomicAdd(&s.n_cand, 1);
+        s.cand[pos] = order_key(v);
+        s.cand_warp[pos] = (unsigned char)tag;
+    };
+    int above = 0;
+    constexpr int kAhead = 4;
+    for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
+        float4 q[kAhead];
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+            const int vi = v0 + u * 32 + lane;
+            q[u] = vi < vend ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) {
+            if (v0 + u * 32 + lane < vend) {
+                const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int bin = bin_of(x[j], lo, scale);
+                    above += bin > tbin;
+                    if (bin == tbin) candidate(x[j], warp);
+                }
+            }
+        }
+    }
+    if (tid < head) { if (bin_of(sc[tid], lo, scale) == tbin) candidate(sc[tid], 255); }
+    for (int i = head + 4 * n_vec + tid; i < n; i += kThreads)
+        if (bin_of(sc[i], lo, scale) == tbin) candidate(sc[i], 255);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xffffffffu, above, d);
+    if (lane == 0) { s.cnt[0][0][warp] = above; s.cnt[1][0][warp] = 0; }
+    __syncthreads();
+    const int nc = s.n_cand;
+    uint32_t thr;
+    int ties;
+    if (nc <= 64) {
+        // few candidates: every one of them counts the others above and equal to itself
+        if (tid < nc) {
+            const uint32_t mine = s.cand[tid];
+            int gt = 0, eq = 0;
+            for (int j = 0; j < nc; ++j) { const uint32_t o = s.cand[j]; gt += o > mine; eq += o == mine; }
+            if (gt < want && want <= gt + eq) { s.bin = (int)mine; s.remaining = want - gt; }   // the same pair from every holder of that key
+        }
+        __syncthreads();
+        thr = (uint32_t)s.bin;
+        ties = s.remaining;
+    } else {
+        thr = radix_select(s, want, &ties, [&](auto tally) {
+            for (int i = tid; i < nc; i += kThreads) tally(s.cand[i]);
+        });
+    }
+    for (int i = tid; i < nc; i += kThreads) {
+        const int w = s.cand_warp[i];
+        if (w < kWarps) {
+            if (s.cand[i] > thr) atomicAdd(&s.cnt[0][0][w], 1);
+            else if (s.cand[i] == thr) atomicAdd(&s.cnt[1][0][w], 1);
+        }
+    }
+    *thr_out = thr;
+    *ties_out = ties;
+    return true;                                           // emit_ordered synchronises before it reads the counts
+}
+
 // Ordered pass over one score vector: writes, ascending, the indices of the scores whose key exceeds
 // `thr` and of the first `ties` scores whose key equals it.  The vector is cut into an unaligned
 // head (0-3 scores), a 16-byte aligned body and a tail (0-3 scores).  Every warp owns a contiguous
@@ -228,7 +329,8 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
 // keys do (and -0 == +0 either way); that saves the key mapping, which is most of the work per score.
 // A CTA may be given a slice of the vector: `index_base` is the index of sc[0] in the whole vector and
 // gt0 / eq0 count the scores above / at the threshold that precede the slice.
-template <bool kPlain>
+// kCounted: the per-warp counts of the body are already in shared memory (threshold_with_counts left them).
+template <bool kPlain, bool kCounted = false>
 __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n, uint32_t thr, int ties,
                              int* __restrict__ out, int index_base = 0, int gt0 = 0, int eq0 = 0) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -258,28 +360,30 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
         const uint32_t key = order_key(sc[i]);
         head_gt += key > thr; head_eq += key == thr;
     }
-    int cnt_gt = 0, cnt_eq = 0;                         // full-width counters: a stretch may hold more than 2^16 scores
-    for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
-        float4 q[kAhead];
+    if (!kCounted) {
+        int cnt_gt = 0, cnt_eq = 0;                     // full-width counters: a stretch may hold more than 2^16 scores
+        for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
+            float4 q[kAhead];
 #pragma unroll
-        for (int u = 0; u < kAhead; ++u) {
-            const int vi = v0 + u * 32 + lane;
-            q[u] = vi < vend ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int u = 0; u < kAhead; ++u) {
+                const int vi = v0 + u * 32 + lane;
+                q[u] = vi < vend ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < kAhead; ++u) {
+                int g, e;
+                flags(q[u], g, e);
+                if (v0 + u * 32 + lane < vend) { cnt_gt += __popc(g); cnt_eq += __popc(e); }
+            }
         }
 #pragma unroll
-        for (int u = 0; u < kAhead; ++u) {
-            int g, e;
-            flags(q[u], g, e);
-            if (v0 + u * 32 + lane < vend) { cnt_gt += __popc(g); cnt_eq += __popc(e); }
+        for (int d = 16; d > 0; d >>= 1) {
+            cnt_gt += __shfl_xor_sync(0xffffffffu, cnt_gt, d);
+            cnt_eq += __shfl_xor_sync(0xffffffffu, cnt_eq, d);
         }
+        __syncthreads();                                // earlier users of the shared arrays are done
+        if (lane == 0) { s.cnt[0][0][warp] = cnt_gt; s.cnt[1][0][warp] = cnt_eq; }
     }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-        cnt_gt += __shfl_xor_sync(0xffffffffu, cnt_gt, d);
-        cnt_eq += __shfl_xor_sync(0xffffffffu, cnt_eq, d);
-    }
-    __syncthreads();                                    // earlier users of the shared arrays are done
-    if (lane == 0) { s.cnt[0][0][warp] = cnt_gt; s.cnt[1][0][warp] = cnt_eq; }
     __syncthreads();
     int base_gt, base_eq;
     {
@@ -305,38 +409,70 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
             g += key > thr; e += key == thr;
         }
     }
-    for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
-        float4 q[kAhead];
+    // A warp takes 512 scores at a time, 16 consecutive ones per lane: one packed shuffle scan of the lanes' counts
+    // gives every lane its place (population counts and votes per score were the bottleneck before), the kept
+    // indices go to the warp's staging buffer in output order and leave through coalesced stores.
+    int* stage = s.stage[warp];
+    auto above = [&](float x) { return kPlain ? x > thr_f : order_key(x) > thr; };
+    auto equal = [&](float x) { return kPlain ? x == thr_f : order_key(x) == thr; };
+    auto load4 = [&](int v0, float4 (&q)[kAhead]) {
 #pragma unroll
         for (int u = 0; u < kAhead; ++u) {
-            const int vi = v0 + u * 32 + lane;
+            const int vi = v0 + kAhead * lane + u;
             q[u] = vi < vend ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
+    };
+    float4 q[kAhead];
+    load4(vbegin, q);
+    for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
+        float4 nx[kAhead];
+        load4(v0 + 32 * kAhead, nx);                     // the next 512 scores are on their way while these are placed
+        const int ties_before = min(base_eq, ties);      // ties already emitted
+        uint32_t gbits = 0, ebits = 0;                   // this lane's 16 scores: above / at the threshold
 #pragma unroll
         for (int u = 0; u < kAhead; ++u) {
-            const int vi = v0 + u * 32 + lane;
-            int g, e;
-            flags(q[u], g, e);
-            if (vi >= vend) { g = 0; e = 0; }
-            const int mine = __popc(g) | (__popc(e) << 16);
-            int incl = mine;
+            if (v0 + kAhead * lane + u < vend) {
+                const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const int t = __shfl_up_sync(0xffffffffu, incl, off);
-                if (lane >= off) incl += t;
+                for (int j = 0; j < 4; ++j) {
+                    if (above(x[j])) gbits |= 1u << (4 * u + j);
+                    else if (equal(x[j])) ebits |= 1u << (4 * u + j);
+                }
             }
-            int gt_before = base_gt + ((incl - mine) & 0xffff);
-            int eq_before = base_eq + ((incl - mine) >> 16);
-            const int i0 = index_base + head + 4 * vi;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if ((g >> j) & 1) { out[gt_before + min(eq_before, ties)] = i0 + j; ++gt_before; }
-                else if ((e >> j) & 1) { if (eq_before < ties) out[gt_before + eq_before] = i0 + j; ++eq_before; }
-            }
-            const int total = __shfl_sync(0xffffffffu, incl, 31);
-            base_gt += total & 0xffff;
-            base_eq += total >> 16;
         }
+        const int mine = __popc(gbits) | (__popc(ebits) << 16);
+        int incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += t;
+        }
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        const int mgt = total & 0xffff, meq = total >> 16;
+        int g_loc = (incl - mine) & 0xffff, q_loc = (incl - mine) >> 16;
+        const int i0 = index_base + head + 4 * (v0 + kAhead * lane);
+        if (meq == 0) {                                  // the common case: no score of these 512 equals the threshold
+            const int shift = min(base_eq, ties) - ties_before;      // zero; kept for symmetry with the general case
+            int* dst = stage + g_loc + shift;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if ((gbits >> j) & 1) *dst++ = i0 + j;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                if ((gbits >> j) & 1) { stage[g_loc + min(base_eq + q_loc, ties) - ties_before] = i0 + j; ++g_loc; }
+                else if ((ebits >> j) & 1) { if (base_eq + q_loc < ties) stage[g_loc + q_loc] = i0 + j; ++q_loc; }
+            }
+        }
+        __syncwarp();
+        const int count = mgt + min(base_eq + meq, ties) - ties_before;
+        int* dst = out + base_gt + ties_before;
+        for (int i = lane; i < count; i += 32) dst[i] = stage[i];
+        __syncwarp();
+        base_gt += mgt;
+        base_eq += meq;
+#pragma unroll
+        for (int u = 0; u < kAhead; ++u) q[u] = nx[u];
     }
     if (warp == kWarps - 1 && lane == 0) {                // the tail follows the last stretch
         for (int i = tail_begin; i < n; ++i) {
@@ -364,8 +500,13 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
         return;
     }
     int ties = 0;
+    uint32_t thr;
+    if (threshold_with_counts(s, sc, n, kk, &thr, &ties)) {
+        emit_ordered<true, true>(s, sc, n, thr, ties, out);
+        return;
+    }
     bool all_finite = false;
-    const uint32_t thr = find_threshold(s, [&](auto f) { for_each_score(sc, n, f); }, sc, n, kk, &ties, &all_finite);
+    thr = find_threshold(s, [&](auto f) { for_each_score(sc, n, f); }, sc, n, kk, &ties, &all_finite);
     if (all_finite) emit_ordered<true>(s, sc, n, thr, ties, out);
     else emit_ordered<false>(s, sc, n, thr, ties, out);
 }

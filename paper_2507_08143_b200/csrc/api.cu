@@ -194,15 +194,31 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
         }
         return t;
     };
+    // Sequences of one length give CTAs of one duration, which run in waves; a ragged batch gives CTAs of
+    // all durations, and then the sweep takes the average load of an SM plus about half a block at its end.
+    bool ragged = false;
+    for (int b = 1; b < s->batch; ++b)
+        ragged = ragged || (s->cu_seqlens[b + 1] - s->cu_seqlens[b]) != (s->cu_seqlens[1] - s->cu_seqlens[0]);
+    const double lh = (double)s->layers * s->heads;
+    const double stream_us = lh * (double)p.total_tokens * 256.0 / 44e3 / kFallbackSmCount;   // 44 GB/s = 44e3 B/us per SM
+    auto ragged_cost = [&](int c, double setup_us) {
+        const double ctas = (double)count_chunks(c) * lh;
+        const double longest = (double)(hp->max_n < c ? hp->max_n : c);
+        return ctas * setup_us / kFallbackSmCount + stream_us + 0.5 * (setup_us + longest * 256.0 / 44e3);
+    };
     int chunk = kMaxChunk;
     double best = 1e300;
     for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
-        const double ctas = (double)count_chunks(c) * s->layers * s->heads;
+        const double ctas = (double)count_chunks(c) * lh;
         const double waves = ceil(ctas / kFallbackSmCount);
-        const double per_cta_us = 4.0 + c * 256.0 / 44e3;             // 44 GB/s = 44e3 B/us per SM
+        const double per_cta_us = 4.0 + c * 256.0 / 44e3;
         const double partial_us = ctas * 2.0 * 131072.0 / 6.4e6;      // written once, read once at 6.4 TB/s
-        const double cost = waves * per_cta_us + partial_us;
+        const double cost = (ragged ? ragged_cost(c, 4.0) : waves * per_cta_us) + partial_us;
         if (cost < best * 0.999) { best = cost; chunk = c; }
+    }
+    if (const char* e = getenv("COMPACTOR_GRAM_BLOCK")) {               // tuning aid
+        const long v = strtol(e, nullptr, 10);
+        if (v >= kMinChunk && v <= kMaxChunk && (v & (v - 1)) == 0) chunk = (int)v;
     }
     p.chunk = chunk;
     long long tc = count_chunks(chunk);
@@ -213,10 +229,15 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     int schunk = kMaxChunk;
     best = 1e300;
     for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
-        const double ctas = (double)count_chunks(c) * s->layers * s->heads;
+        const double ctas = (double)count_chunks(c) * lh;
         const double per_cta_us = 2.0 + c * 256.0 / 44e3;
-        const double cost = (ctas / kFallbackSmCount < 1.0 ? 1.0 : ctas / kFallbackSmCount) * per_cta_us + 0.5 * per_cta_us;
+        const double cost = ragged ? ragged_cost(c, 2.0)
+                                   : (ctas / kFallbackSmCount < 1.0 ? 1.0 : ctas / kFallbackSmCount) * per_cta_us + 0.5 * per_cta_us;
         if (cost < best * 0.999) { best = cost; schunk = c; }
+    }
+    if (const char* e = getenv("COMPACTOR_SCORE_BLOCK")) {              // tuning aid
+        const long v = strtol(e, nullptr, 10);
+        if (v >= kMinChunk && v <= kMaxChunk && (v & (v - 1)) == 0) schunk = (int)v;
     }
     p.schunk = schunk;
     tc = count_chunks(schunk);

@@ -7,10 +7,13 @@
 // histogram on the leading float bits would pile everything into a dozen bins.  Instead the range
 // is estimated from the first few thousand scores, a 2048-bin histogram linear in the score value
 // is taken over all of them (values outside the estimate fall into the end bins; the binning is
-// monotone, so it orders exactly), the bin holding the kk-th largest is found, its members are
-// collected in shared memory and the exact key is found there by a three-pass radix select.
-// Inputs that defeat this (non-finite values, a constant score, more members than fit) take the
-// same three-pass radix select over global memory.
+// monotone, so it orders exactly) and the bin holding the kk-th largest is found.  A second pass, cut
+// the way the ordered pass is, counts per warp the scores in higher bins and lists the members of that
+// bin; the exact key is found among them (a few hundred) and they are added to their warps' counts, so
+// the ordered pass starts from finished counts.  Inputs that defeat this (non-finite values, a constant
+// score, more members than fit) take a three-pass radix select over global memory and an ordered pass
+// that counts for itself.  Where one CTA per score vector would leave most SMs idle, the vectors are cut
+// into slices over many CTAs (the multi_* kernels below).
 #include "common.cuh"
 
 namespace compactor {
@@ -322,9 +325,9 @@ __device__ bool threshold_with_counts(SelectSmem& s, const float* __restrict__ s
 // `thr` and of the first `ties` scores whose key equals it.  The vector is cut into an unaligned
 // head (0-3 scores), a 16-byte aligned body and a tail (0-3 scores).  Every warp owns a contiguous
 // stretch of the body, read as float4 (four consecutive scores per lane): it first counts its
-// scores above and at the threshold, one block-wide scan turns the counts into output offsets, and
-// then each warp emits its stretch on its own (a shuffle scan of per-lane counts per 128 scores).
-// The pass is bound by instruction issue, hence four scores per load and per scan.
+// scores above and at the threshold (unless the caller has them already), one block-wide scan turns
+// the counts into output offsets, and then each warp emits its stretch on its own, 512 scores at a
+// time (see the loop).
 // kPlain: every score is known to be finite, so that comparing the floats themselves orders them as the
 // keys do (and -0 == +0 either way); that saves the key mapping, which is most of the work per score.
 // A CTA may be given a slice of the vector: `index_base` is the index of sc[0] in the whole vector and

@@ -38,6 +38,16 @@ int sm_count() {
     return cached[dev];
 }
 
+}  // namespace
+namespace compactor {
+// COMPACTOR_NO_PDL=1 launches every kernel fully serialised (a measuring aid).
+bool pdl_enabled() {
+    const char* e = getenv("COMPACTOR_NO_PDL");
+    return e == nullptr || e[0] != '1';
+}
+}  // namespace compactor
+namespace {
+
 // Slices per score vector for the selection spread over several CTAs: enough CTAs for two per SM, no
 // slice shorter than 8192 scores.
 constexpr int kMaxSelectParts = 64;

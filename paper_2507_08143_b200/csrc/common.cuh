@@ -85,6 +85,28 @@ __device__ __forceinline__ int find_segment(const int* __restrict__ table, int n
     return lo;
 }
 
+// Programmatic dependent launch.  A kernel of the fused call's chain is launched so that it may start
+// while its predecessor in the stream is still running: its CTAs are scheduled as soon as every CTA of the
+// predecessor has called pdl_trigger() (first thing) or exited, do their set-up (shared memory, barriers,
+// operands that come from the caller), and then pdl_wait() until the predecessor has finished and its
+// writes are visible.  Everything a kernel reads that an earlier kernel of the call wrote is read after
+// pdl_wait(); a kernel launched without the attribute passes through both calls.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                  Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // Kernel launchers (each defined next to its kernel).  All enqueue on `stream` and return the
 // launch status.
 cudaError_t launch_gram(const Plan& p, const Mat& k, double* partials, int* status, cudaStream_t stream);

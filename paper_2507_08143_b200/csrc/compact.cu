@@ -29,6 +29,8 @@ __device__ __forceinline__ void st_stream(uint4* p, const uint4& v) {
 __global__ void __launch_bounds__(kThreads)
 compact_kernel(Plan p, Mat k, Mat v, const int* __restrict__ idx,
                __nv_bfloat16* __restrict__ k_out, __nv_bfloat16* __restrict__ v_out) {
+    pdl_trigger();
+    pdl_wait();                                            // the indices are complete
     const int lh = blockIdx.y;
     const int layer = lh / p.heads, head = lh % p.heads;
     const int piece = threadIdx.x & 15, sub = threadIdx.x >> 4;
@@ -77,6 +79,8 @@ compact_kernel(Plan p, Mat k, Mat v, const int* __restrict__ idx,
 __global__ void __launch_bounds__(kThreads)
 compact_across_kernel(Plan p, Mat k, Mat v, const int* __restrict__ idx, const int* __restrict__ head_offsets,
                       __nv_bfloat16* __restrict__ k_out, __nv_bfloat16* __restrict__ v_out) {
+    pdl_trigger();
+    pdl_wait();                                            // indices and head offsets are complete
     const int layer = blockIdx.y;
     const int piece = threadIdx.x & 15, sub = threadIdx.x >> 4;
     const long long rows_per_layer = (long long)p.heads * p.total_keep;
@@ -128,16 +132,16 @@ cudaError_t launch_compact_across(const Plan& p, const Mat& k, const Mat& v, con
     const long long rows = (long long)p.heads * p.total_keep;
     if (rows == 0 || p.layers == 0) return cudaSuccess;
     dim3 grid((unsigned)((rows + kRowsPerCta - 1) / kRowsPerCta), p.layers);
-    compact_across_kernel<<<grid, kThreads, 0, stream>>>(p, k, v, idx, head_offsets, k_out, v_out);
-    return cudaGetLastError();
+    cudaError_t e = launch_chained(compact_across_kernel, grid, dim3(kThreads), 0, stream, p, k, v, idx, head_offsets, k_out, v_out);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int* idx,
                            __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream) {
     if (p.total_keep == 0 || p.layers * p.heads == 0) return cudaSuccess;
     dim3 grid((p.total_keep + kRowsPerCta - 1) / kRowsPerCta, p.layers * p.heads);
-    compact_kernel<<<grid, kThreads, 0, stream>>>(p, k, v, idx, k_out, v_out);
-    return cudaGetLastError();
+    cudaError_t e = launch_chained(compact_kernel, grid, dim3(kThreads), 0, stream, p, k, v, idx, k_out, v_out);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace compactor

@@ -58,10 +58,12 @@ project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const floa
     const int fr = lane >> 2, fk = lane & 3;            // fragment coordinates: A[fr][fk], B[fk][fr], C[fr][2 fk, 2 fk + 1]
     constexpr int kNT = MP / 8;                         // 8-column tiles
 
+    pdl_trigger();
     for (int i = tid; i < kD * MP; i += kProjThreads) {   // Phi, widened
         const int row = i / MP, col = i - row * MP;
         s.phi[row * LD + col] = (col < m) ? (double)__ldg(phi + row * m + col) : 0.0;
     }
+    pdl_wait();                                           // the Gram partials are complete
 
     // Item bookkeeping and the look-ahead loads.
     struct Item { int unit, slice, b, lh, n_part, n_tok; const double* part; };
@@ -207,12 +209,14 @@ cholesky_kernel(Plan p, const double* __restrict__ t_buf, const float* __restric
     const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int m = p.m;
 
+    pdl_trigger();
     if (tid == 0) s.flags = 0;
     for (int i = tid; i < kD * MP; i += kCholThreads) {
         const int row = i / MP, col = i - row * MP;
         s.phi[i] = col < m ? __ldg(phi + row * m + col) : 0.f;
     }
     if (tid < MP) s.inv_diag[tid] = 0.0;
+    pdl_wait();                                           // T = C Phi of every unit is complete
     __syncthreads();
     auto sync = [] { __syncthreads(); };
     const bool finite = gram_of_sketch<MP, kCholWarps>(t_buf + (size_t)unit * kD * MP, s.phi, s.u.g, s.u.t, tid, sync);
@@ -431,7 +435,8 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
     const int n_items = units * kSlices;
     const int resident = 2 * sm_count;                            // two CTAs fit on an SM
     const int grid = n_items < resident ? n_items : resident;
-    project_kernel<MP><<<grid, kProjThreads, smem, stream>>>(p, k, partials, phi, t_buf, n_items);
+    e = launch_chained(project_kernel<MP>, dim3(grid), dim3(kProjThreads), smem, stream, p, k, partials, phi, t_buf, n_items);
+    if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (factorization == COMPACTOR_FACTOR_EIG) {
@@ -447,7 +452,8 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
         const int csmem = (int)sizeof(CholSmem<MP>);
         e = cudaFuncSetAttribute(cholesky_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, csmem);
         if (e != cudaSuccess) return e;
-        cholesky_kernel<MP><<<units, kCholThreads, csmem, stream>>>(p, t_buf, phi, w, status);
+        e = launch_chained(cholesky_kernel<MP>, dim3(units), dim3(kCholThreads), csmem, stream, p, (const double*)t_buf, phi, w, status);
+        if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();
 }

@@ -41,6 +41,7 @@ struct __align__(1024) GramSmem {
 __global__ void __launch_bounds__(kThreads, 1)
 gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, double* __restrict__ partials,
             int* __restrict__ status) {
+    pdl_trigger();
     extern __shared__ unsigned char smem_raw[];
     GramSmem& s = *reinterpret_cast<GramSmem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
     const int chunk_id = blockIdx.x;

@@ -60,6 +60,7 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
     constexpr uint32_t kCols = BufCols<MP>::value;
     constexpr uint32_t kTmemCols = kCols * kBufs;
     Smem& s = *reinterpret_cast<Smem*>(smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u));
+    pdl_trigger();
     const int chunk_id = blockIdx.x;
     const int lh = blockIdx.y;
     const int layer = lh / p.heads, head = lh % p.heads;
@@ -89,6 +90,15 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
 
     if (warp == 0) {
         if (lane == 0) {
+            // the first key tiles come from the caller and are fetched at once; W is the factor stage's and must wait for it
+            int t = 0;
+            for (; t < n_tiles && t < kStages; ++t) {
+                mbar_arrive_expect_tx(&s.full[t], kTileBytes);
+                const int tok = tok_begin + t * kTile;
+                tma_load_4d(s.tiles[t], &kmap, &s.full[t], 0, tok, head, layer);
+                tma_load_4d(s.tiles[t] + kBoxBytes, &kmap, &s.full[t], 64, tok, head, layer);
+            }
+            pdl_wait();
             mbar_arrive_expect_tx(&s.w_full, 4 * MP * 128);
 #pragma unroll
             for (int term = 0; term < 2; ++term)
@@ -96,7 +106,7 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
                 for (int half = 0; half < 2; ++half)
                     tma_load_2d(Fused<MP>::value ? s.w[half][term] : s.w[term][half], &wmap, &s.w_full, half * 64,
                                 (unit * 2 + term) * MP);
-            for (int t = 0; t < n_tiles; ++t) {
+            for (; t < n_tiles; ++t) {
                 const int stage = t % kStages, round = t / kStages;
                 if (round > 0 && !mbar_wait(&s.empty[stage], (round - 1) & 1)) { s.abort = 1; break; }
                 if (*(volatile int*)&s.abort) break;
@@ -225,7 +235,8 @@ cudaError_t launch_score_mp(const Plan& p, const CUtensorMap& kmap, const CUtens
     cudaError_t e = cudaFuncSetAttribute(score_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(p.total_schunks, p.layers * p.heads);
-    score_kernel<MP><<<grid, kThreads, smem, stream>>>(p, kmap, wmap, scores, status);
+    e = launch_chained(score_kernel<MP>, grid, dim3(kThreads), smem, stream, p, kmap, wmap, scores, status);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 

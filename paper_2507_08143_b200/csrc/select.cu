@@ -491,10 +491,12 @@ __global__ void __launch_bounds__(kThreads, 1)
 select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    pdl_trigger();
     const int unit = blockIdx.x;
     const int b = unit % p.batch, lh = unit / p.batch;
     const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
     const int kk = p.cu_keep[b + 1] - p.cu_keep[b];
+    pdl_wait();                                            // the scores are complete
     if (kk <= 0 || n <= 0) return;
     const float* sc = scores + (size_t)lh * p.total_tokens + p.cu_seqlens[b];
     int* out = idx_out + (size_t)lh * p.total_keep + p.cu_keep[b];
@@ -582,6 +584,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 multi_hist_kernel(Plan p, const float* __restrict__ scores, MultiSelect m) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    pdl_trigger();
     const Slice c = decode_slice(p, m, blockIdx.x);
     if (c.kk <= 0 || c.n <= 0 || c.kk >= c.n) return;
     const int tid = threadIdx.x;
@@ -611,7 +614,9 @@ __global__ void __launch_bounds__(kThreads, 1)
 multi_candidates_kernel(Plan p, const float* __restrict__ scores, MultiSelect m) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    pdl_trigger();
     const Slice c = decode_slice(p, m, blockIdx.x);
+    pdl_wait();                                            // the groups' histograms are complete
     if (c.kk <= 0 || c.n <= 0 || c.kk >= c.n) return;
     const int tid = threadIdx.x, lane = tid & 31;
     int* st = m.state + (size_t)c.group * kSelStateInts;
@@ -653,7 +658,9 @@ multi_finalize_kernel(Plan p, const float* __restrict__ scores, MultiSelect m, i
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
     __shared__ int head_gt[64], head_eq[64];
+    pdl_trigger();
     const Slice c = decode_group(p, m, blockIdx.x);
+    pdl_wait();                                            // the candidate lists are complete
     const int H = c.hg, n = c.n, kk = c.kk, tid = threadIdx.x;
     int* offs = head_offsets != nullptr ? head_offsets + (size_t)c.group * (H + 1) : nullptr;
     auto unit_of = [&](int h) { return (c.lh + h) * p.batch + c.b; };
@@ -752,7 +759,9 @@ multi_emit_kernel(Plan p, const float* __restrict__ scores, MultiSelect m, const
                   int* __restrict__ idx_out) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SelectSmem& s = *reinterpret_cast<SelectSmem*>(smem_raw);
+    pdl_trigger();
     const Slice c = decode_slice(p, m, blockIdx.x);
+    pdl_wait();                                            // thresholds, offsets and slice counts are complete
     if (c.kk <= 0 || c.n <= 0) return;
     int* out;
     if (m.across) {
@@ -783,6 +792,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 blend_kernel(Plan p, const float* __restrict__ attn, float lambda, float* __restrict__ scores) {
     __shared__ double red[4][kWarps];
     __shared__ double stats[4];
+    pdl_trigger();
+    pdl_wait();                                            // the leverage scores are complete
     const int unit = blockIdx.x;
     const int b = unit % p.batch, lh = unit / p.batch;
     const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
@@ -865,6 +876,8 @@ blend_stats_kernel(Plan p, const float* __restrict__ attn, const float* __restri
                    double* __restrict__ stats) {
     __shared__ double red[2][kWarps];
     __shared__ double tot[2];
+    pdl_trigger();
+    pdl_wait();                                            // the leverage scores are complete
     const int part = blockIdx.x % parts, unit = blockIdx.x / parts;
     const int b = unit % p.batch, lh = unit / p.batch;
     const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
@@ -895,6 +908,8 @@ blend_stats_kernel(Plan p, const float* __restrict__ attn, const float* __restri
 __global__ void __launch_bounds__(kThreads, 1)
 blend_apply_kernel(Plan p, const float* __restrict__ attn, float lambda, float* __restrict__ scores, int parts,
                    const double* __restrict__ stats) {
+    pdl_trigger();
+    pdl_wait();                                            // the slices' statistics are complete
     const int part = blockIdx.x % parts, unit = blockIdx.x / parts;
     const int b = unit % p.batch, lh = unit / p.batch;
     const int n = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
@@ -933,8 +948,8 @@ cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStre
     const int smem = (int)sizeof(SelectSmem);
     cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    select_kernel<<<units, kThreads, smem, stream>>>(p, scores, idx);
-    return cudaGetLastError();
+    e = launch_chained(select_kernel, dim3(units), dim3(kThreads), smem, stream, p, scores, idx);
+    return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t launch_select_multi(const Plan& p, const float* scores, int* idx, int* head_offsets, const MultiSelect& m,
@@ -952,10 +967,12 @@ cudaError_t launch_select_multi(const Plan& p, const float* scores, int* idx, in
     if ((e = cudaMemsetAsync(m.state, 0, sizeof(int) * (size_t)groups * kSelStateInts, stream)) != cudaSuccess) return e;
     const unsigned slices = (unsigned)units * (unsigned)m.parts;
     multi_hist_kernel<<<slices, kThreads, smem, stream>>>(p, scores, m);
-    multi_candidates_kernel<<<slices, kThreads, smem, stream>>>(p, scores, m);
-    multi_finalize_kernel<<<groups, kThreads, smem, stream>>>(p, scores, m, m.across ? head_offsets : nullptr);
+    if ((e = launch_chained(multi_candidates_kernel, dim3(slices), dim3(kThreads), smem, stream, p, scores, m)) != cudaSuccess) return e;
+    if ((e = launch_chained(multi_finalize_kernel, dim3(groups), dim3(kThreads), smem, stream, p, scores, m,
+                            m.across ? head_offsets : (int*)nullptr)) != cudaSuccess) return e;
     if (p.total_keep > 0) {
-        multi_emit_kernel<<<slices, kThreads, smem, stream>>>(p, scores, m, head_offsets, idx);
+        if ((e = launch_chained(multi_emit_kernel, dim3(slices), dim3(kThreads), smem, stream, p, scores, m,
+                                (const int*)head_offsets, idx)) != cudaSuccess) return e;
     }
     return cudaGetLastError();
 }
@@ -965,10 +982,15 @@ cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* 
     const int units = p.layers * p.heads * p.batch;
     if (units == 0 || p.total_tokens == 0) return cudaSuccess;
     if (parts > 1 && stats != nullptr) {
-        blend_stats_kernel<<<units * parts, kThreads, 0, stream>>>(p, attn, scores, parts, stats);
-        blend_apply_kernel<<<units * parts, kThreads, 0, stream>>>(p, attn, lambda, scores, parts, stats);
+        cudaError_t e = launch_chained(blend_stats_kernel, dim3(units * parts), dim3(kThreads), 0, stream, p, attn,
+                                       (const float*)scores, parts, stats);
+        if (e != cudaSuccess) return e;
+        e = launch_chained(blend_apply_kernel, dim3(units * parts), dim3(kThreads), 0, stream, p, attn, lambda, scores, parts,
+                           (const double*)stats);
+        if (e != cudaSuccess) return e;
     } else {
-        blend_kernel<<<units, kThreads, 0, stream>>>(p, attn, lambda, scores);
+        cudaError_t e = launch_chained(blend_kernel, dim3(units), dim3(kThreads), 0, stream, p, attn, lambda, scores);
+        if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();
 }

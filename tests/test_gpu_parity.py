@@ -396,3 +396,23 @@ def test_fused_sweep_kernel_gives_the_same_answers(B, name, monkeypatch):
     nonempty = [b for b, n in enumerate(w.seqlens) if n >= 48]
     assert np.all(st[:, nonempty] == 0)
     print(f"fused sweep, {w.name}: max rel score err {worst:.2e}")
+
+
+def test_dependent_launches_change_nothing(B, monkeypatch):
+    # the kernels of a call are launched so that each may set up while its predecessor drains; with every launch fully
+    # serialised (a switch the library reads at every call) the outputs must be the same bits, with and without the blend
+    w = inputs.Workload("chain", 2, 2, 128, [5000, 300, 0, 70000], [0.3, 0.5, 0.5, 0.2], p=0.7, seed=19)
+    _, kr, v = [None if t is None else t.cuda() for t in inputs.make_tensors(w, device="cpu", want_pre=False)]
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    phi = inputs.make_sketch_matrix(w.d, w.m, w.seed)
+    keep = _keep(B, w)
+    a = inputs.make_attention_scores(w, seed=3, device="cuda")
+    for attn in (None, a):
+        monkeypatch.setenv("COMPACTOR_NO_PDL", "1")
+        serial = H.run_compress(B, shape, kr, kr, v, phi, keep, attn=attn)
+        monkeypatch.setenv("COMPACTOR_NO_PDL", "0")
+        for _ in range(3):
+            chained = H.run_compress(B, shape, kr, kr, v, phi, keep, attn=attn)
+            for x, y in zip(serial, chained):
+                assert torch.equal(x.view(torch.int16) if x.dtype == torch.bfloat16 else x,
+                                   y.view(torch.int16) if y.dtype == torch.bfloat16 else y)

@@ -344,13 +344,23 @@ def time_workload(B, inputs, torch, name, mode, steps, warmup):
     for _ in range(max(warmup, 3)):
         B.compress(shape, k_score, kr, v, phi_d, keep, idx, k_out, v_out, ws, status=status)
     torch.cuda.synchronize()
-    for es in ev:
+    for es in ev:                                         # stage times: the same call with markers between its kernels
         if small:
             flush.zero_()
         B.compress_profiled(shape, k_score, kr, v, phi_d, keep, idx, k_out, v_out, ws, es, status=status)
     torch.cuda.synchronize()
     assert int(status.max().item()) == 0
-    ms = statistics.median(es[0].elapsed_time(es[-1]) for es in ev)
+    pairs = []                                            # the step itself: the plain call, nothing between its kernels,
+    for _ in range(steps):                                # steps enqueued back to back (the flush is outside the events)
+        if small:
+            flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        B.compress(shape, k_score, kr, v, phi_d, keep, idx, k_out, v_out, ws, status=status)
+        e1.record()
+        pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    ms = statistics.median(a.elapsed_time(b) for a, b in pairs)
     stage_ms = {nm: statistics.median(es[j].elapsed_time(es[j + 1]) for es in ev) for j, nm in enumerate(B.STAGE_NAMES)}
     peak, _ = measured_peak()
     b_alg = algorithmic_bytes(w, keep, mode)
@@ -363,6 +373,41 @@ def time_workload(B, inputs, torch, name, mode, steps, warmup):
             "l2": "flushed before every step" if small else "inputs exceed L2"}
 
 
+def time_full_variant(B, inputs, torch, name, selection, factorization, steps, warmup):
+    """A workload through compactor_compress_full without the attention term: selection across the heads of a
+    layer, or the eigendecomposition route of the scorer, at full size."""
+    w = inputs.workload(name)
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    keep = [B.keep_count(n, r) for n, r in zip(w.seqlens, w.ratios)]
+    phi_d = inputs.make_sketch_matrix(w.d, w.m, w.seed).cuda()
+    _, kr, v = inputs.make_tensors(w, device="cuda", want_pre=False)
+    total_keep = sum(keep)
+    idx = torch.empty(w.layers, w.heads * total_keep, dtype=torch.int32, device="cuda")
+    offs = torch.empty(w.layers, w.batch, w.heads + 1, dtype=torch.int32, device="cuda")
+    k_out = torch.empty(w.layers, w.heads * total_keep, w.d, dtype=torch.bfloat16, device="cuda")
+    v_out = torch.empty_like(k_out)
+    status = torch.zeros(w.units, dtype=torch.int32, device="cuda")
+    opt = B.options(selection=selection, factorization=factorization, eig_floor=1e-6, lam=0.0, q_per_kv=0)
+    ws = torch.empty(B.compress_full_workspace_bytes(shape, opt), dtype=torch.uint8, device="cuda")
+    call = lambda: B.compress_full(shape, opt, None, kr, kr, v, phi_d, keep, idx, k_out, v_out, ws,
+                                   head_offsets_out=offs, status=status)
+    for _ in range(max(warmup, 3)):
+        call()
+    pairs = []
+    for _ in range(steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); call(); e1.record()
+        pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    ms = statistics.median(a.elapsed_time(b) for a, b in pairs)
+    timeouts = int((status & 4).max().item())             # 4 = a bounded wait ran out; the eigen route reports floored eigenvalues with 2
+    del kr, v, idx, k_out, v_out, ws
+    torch.cuda.empty_cache()
+    assert timeouts == 0
+    return {"workload": w.name, "units": w.units, "tokens": w.total_tokens, "ms_per_step": round(ms, 4),
+            "tokens_per_s": round(w.total_tokens / (ms * 1e-3))}
+
+
 def extra_measurements(args, B, inputs, torch):
     """The other benchmark workloads, the attention term, the full method and the NLL pass: a few timed
     steps each (medians of CUDA-event times), reported beside the headline."""
@@ -370,6 +415,11 @@ def extra_measurements(args, B, inputs, torch):
     steps = 5
     for key, name, mode in (("c1", "c1", "aliased"), ("c2", "c2", "aliased"), ("c4", "c4", "aliased"), ("c3-paper", "c3", "paper")):
         out["other_workloads"][key] = time_workload(B, inputs, torch, name, mode, steps, 3)
+    # the headline workload through the one-call entry point: selection across heads (Section 3.4), and the
+    # eigendecomposition route of Appendix C with its floor
+    out["other_workloads"]["c3-across-heads"] = time_full_variant(B, inputs, torch, "c3", B.SELECT_ACROSS_HEADS,
+                                                                  B.FACTOR_CHOLESKY, steps, 3)
+    out["other_workloads"]["c3-eig-route"] = time_full_variant(B, inputs, torch, "c3", B.SELECT_PER_HEAD, B.FACTOR_EIG, steps, 3)
     # the paper's Fig. 1 shape at n = 131072: one layer, 8 KV heads x 4 query heads, batch 1
     n, G = 131072, 4
     w = inputs.Workload("fig1-n131072", 1, 8, 128, [n], [0.3], p=0.7, n_out=4, theta=5e5, seed=100)

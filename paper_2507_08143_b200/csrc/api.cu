@@ -41,10 +41,19 @@ int sm_count() {
 }  // namespace
 namespace compactor {
 // COMPACTOR_NO_PDL=1 launches every kernel fully serialised (a measuring aid).
-bool pdl_enabled() {
+// Chained launches pay where a call's grids do not fill the GPU for long (its kernels are then a chain of
+// latencies); on the large workloads they were measured to cost time (C3 +3.5 %, C4 +9 % with every kernel
+// chained), so a call chains its kernels only if its keys are at most this many bytes.
+constexpr long long kChainMaxKeyBytes = 600LL << 20;
+thread_local bool t_chain = false;        // set by make_plan() for the call that this thread is making
+bool pdl_enabled(int which) {
     const char* e = getenv("COMPACTOR_NO_PDL");
-    return e == nullptr || e[0] != '1';
+    if (e != nullptr && e[0] == '1') return false;
+    const char* m = getenv("COMPACTOR_PDL_MASK");               // tuning aid: chain these kernels whatever the size
+    if (m != nullptr) return (strtol(m, nullptr, 10) & which) != 0;
+    return t_chain;
 }
+void set_chain_for(long long key_bytes) { t_chain = key_bytes <= kChainMaxKeyBytes; }
 }  // namespace compactor
 namespace {
 
@@ -130,6 +139,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     p.m = s->m; p.mp = s->m <= 64 ? (s->m + 15) / 16 * 16 : 128;
     p.total_tokens = s->cu_seqlens[s->batch];
     hp->max_n = longest_sequence(s);
+    compactor::set_chain_for((long long)s->layers * s->heads * p.total_tokens * kD * 2);
     hp->units = s->layers * s->heads * s->batch;
     hp->fused = allow_fused && p.mp <= kFusedMaxMp && fused_sweep_enabled();
     hp->slices = 0; hp->window = 0; hp->n_slots = 0; hp->max_pieces = 0; hp->total_pieces = 0;

@@ -132,7 +132,7 @@ cudaError_t launch_compact_across(const Plan& p, const Mat& k, const Mat& v, con
     const long long rows = (long long)p.heads * p.total_keep;
     if (rows == 0 || p.layers == 0) return cudaSuccess;
     dim3 grid((unsigned)((rows + kRowsPerCta - 1) / kRowsPerCta), p.layers);
-    cudaError_t e = launch_chained(compact_across_kernel, grid, dim3(kThreads), 0, stream, p, k, v, idx, head_offsets, k_out, v_out);
+    cudaError_t e = launch_chained(kPdlCompact, compact_across_kernel, grid, dim3(kThreads), 0, stream, p, k, v, idx, head_offsets, k_out, v_out);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -140,7 +140,7 @@ cudaError_t launch_compact(const Plan& p, const Mat& k, const Mat& v, const int*
                            __nv_bfloat16* k_out, __nv_bfloat16* v_out, cudaStream_t stream) {
     if (p.total_keep == 0 || p.layers * p.heads == 0) return cudaSuccess;
     dim3 grid((p.total_keep + kRowsPerCta - 1) / kRowsPerCta, p.layers * p.heads);
-    cudaError_t e = launch_chained(compact_kernel, grid, dim3(kThreads), 0, stream, p, k, v, idx, k_out, v_out);
+    cudaError_t e = launch_chained(kPdlCompact, compact_kernel, grid, dim3(kThreads), 0, stream, p, k, v, idx, k_out, v_out);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 

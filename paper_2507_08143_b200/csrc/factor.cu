@@ -435,7 +435,7 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
     const int n_items = units * kSlices;
     const int resident = 2 * sm_count;                            // two CTAs fit on an SM
     const int grid = n_items < resident ? n_items : resident;
-    e = launch_chained(project_kernel<MP>, dim3(grid), dim3(kProjThreads), smem, stream, p, k, partials, phi, t_buf, n_items);
+    e = launch_chained(kPdlProject, project_kernel<MP>, dim3(grid), dim3(kProjThreads), smem, stream, p, k, partials, phi, t_buf, n_items);
     if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -452,7 +452,7 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
         const int csmem = (int)sizeof(CholSmem<MP>);
         e = cudaFuncSetAttribute(cholesky_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, csmem);
         if (e != cudaSuccess) return e;
-        e = launch_chained(cholesky_kernel<MP>, dim3(units), dim3(kCholThreads), csmem, stream, p, (const double*)t_buf, phi, w, status);
+        e = launch_chained(kPdlCholesky, cholesky_kernel<MP>, dim3(units), dim3(kCholThreads), csmem, stream, p, (const double*)t_buf, phi, w, status);
         if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();

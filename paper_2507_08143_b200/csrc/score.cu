@@ -235,7 +235,7 @@ cudaError_t launch_score_mp(const Plan& p, const CUtensorMap& kmap, const CUtens
     cudaError_t e = cudaFuncSetAttribute(score_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(p.total_schunks, p.layers * p.heads);
-    e = launch_chained(score_kernel<MP>, grid, dim3(kThreads), smem, stream, p, kmap, wmap, scores, status);
+    e = launch_chained(kPdlScore, score_kernel<MP>, grid, dim3(kThreads), smem, stream, p, kmap, wmap, scores, status);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

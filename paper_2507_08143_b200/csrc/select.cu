@@ -948,7 +948,7 @@ cudaError_t launch_select(const Plan& p, const float* scores, int* idx, cudaStre
     const int smem = (int)sizeof(SelectSmem);
     cudaError_t e = cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    e = launch_chained(select_kernel, dim3(units), dim3(kThreads), smem, stream, p, scores, idx);
+    e = launch_chained(kPdlSelect, select_kernel, dim3(units), dim3(kThreads), smem, stream, p, scores, idx);
     return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -967,11 +967,11 @@ cudaError_t launch_select_multi(const Plan& p, const float* scores, int* idx, in
     if ((e = cudaMemsetAsync(m.state, 0, sizeof(int) * (size_t)groups * kSelStateInts, stream)) != cudaSuccess) return e;
     const unsigned slices = (unsigned)units * (unsigned)m.parts;
     multi_hist_kernel<<<slices, kThreads, smem, stream>>>(p, scores, m);
-    if ((e = launch_chained(multi_candidates_kernel, dim3(slices), dim3(kThreads), smem, stream, p, scores, m)) != cudaSuccess) return e;
-    if ((e = launch_chained(multi_finalize_kernel, dim3(groups), dim3(kThreads), smem, stream, p, scores, m,
+    if ((e = launch_chained(kPdlOther, multi_candidates_kernel, dim3(slices), dim3(kThreads), smem, stream, p, scores, m)) != cudaSuccess) return e;
+    if ((e = launch_chained(kPdlOther, multi_finalize_kernel, dim3(groups), dim3(kThreads), smem, stream, p, scores, m,
                             m.across ? head_offsets : (int*)nullptr)) != cudaSuccess) return e;
     if (p.total_keep > 0) {
-        if ((e = launch_chained(multi_emit_kernel, dim3(slices), dim3(kThreads), smem, stream, p, scores, m,
+        if ((e = launch_chained(kPdlOther, multi_emit_kernel, dim3(slices), dim3(kThreads), smem, stream, p, scores, m,
                                 (const int*)head_offsets, idx)) != cudaSuccess) return e;
     }
     return cudaGetLastError();
@@ -982,14 +982,14 @@ cudaError_t launch_blend(const Plan& p, const float* attn, float lambda, float* 
     const int units = p.layers * p.heads * p.batch;
     if (units == 0 || p.total_tokens == 0) return cudaSuccess;
     if (parts > 1 && stats != nullptr) {
-        cudaError_t e = launch_chained(blend_stats_kernel, dim3(units * parts), dim3(kThreads), 0, stream, p, attn,
+        cudaError_t e = launch_chained(kPdlOther, blend_stats_kernel, dim3(units * parts), dim3(kThreads), 0, stream, p, attn,
                                        (const float*)scores, parts, stats);
         if (e != cudaSuccess) return e;
-        e = launch_chained(blend_apply_kernel, dim3(units * parts), dim3(kThreads), 0, stream, p, attn, lambda, scores, parts,
+        e = launch_chained(kPdlOther, blend_apply_kernel, dim3(units * parts), dim3(kThreads), 0, stream, p, attn, lambda, scores, parts,
                            (const double*)stats);
         if (e != cudaSuccess) return e;
     } else {
-        cudaError_t e = launch_chained(blend_kernel, dim3(units), dim3(kThreads), 0, stream, p, attn, lambda, scores);
+        cudaError_t e = launch_chained(kPdlOther, blend_kernel, dim3(units), dim3(kThreads), 0, stream, p, attn, lambda, scores);
         if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();

@@ -72,6 +72,14 @@ def test_c0_writes_nothing_outside_its_buffers(B):
     _compress_guarded(B, inputs.workload("c0"), with_attn=True)
 
 
+def test_few_long_units_write_nothing_outside_their_buffers(B):
+    # two heads with one long sequence: the blend's per-slice statistics and the sliced selection's histograms,
+    # candidate lists and counts live in the part of the workspace that the scoring stage has finished with
+    w = inputs.Workload("guard-long", 1, 2, 128, [140001, 77], [0.3, 0.5], p=0.7, seed=14)
+    _compress_guarded(B, w, with_attn=True)
+    _compress_guarded(B, w)
+
+
 def test_ragged_batch_with_tail_tiles_writes_nothing_outside_its_buffers(B):
     # lengths that end inside a tile, a piece and a Gram block; an empty sequence; total tokens not a multiple of anything
     w = inputs.Workload("guard-ragged", 2, 3, 128, [1000, 129, 0, 2501, 47, 4099, 1], [0.3, 0.5, 0.5, 0.3, 0.5, 0.11, 1.0],

@@ -31,6 +31,13 @@
  *     are unspecified), bit 1 = the sketched Gram matrix was numerically rank deficient (the
  *     singular directions contribute nothing, as a pseudo-inverse would), bit 2 = a bounded
  *     device-side wait ran out.
+ *   - On problems with at most 600 MB of keys the kernels of a call are launched as a chain of
+ *     programmatic dependent launches (each may set up while its predecessor drains); results do
+ *     not depend on it.  The library reads a few environment variables at every call, none of which
+ *     changes a result: COMPACTOR_NO_PDL=1 (no chained launches), COMPACTOR_PDL_MASK,
+ *     COMPACTOR_GRAM_BLOCK / COMPACTOR_SCORE_BLOCK (block lengths of the two sweeps, a power of two
+ *     from 256 to 65536 tokens), COMPACTOR_FUSED_SWEEP and its companions (an experimental
+ *     one-kernel sweep).  They are measuring aids; leave them unset.
  */
 #ifndef COMPACTOR_H_
 #define COMPACTOR_H_

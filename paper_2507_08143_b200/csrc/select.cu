@@ -14,6 +14,8 @@
 // score, more members than fit) take a three-pass radix select over global memory and an ordered pass
 // that counts for itself.  Where one CTA per score vector would leave most SMs idle, the vectors are cut
 // into slices over many CTAs (the multi_* kernels below).
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace compactor {
@@ -138,7 +140,8 @@ __device__ uint32_t radix_select(SelectSmem& s, int want, int* ties, Visit visit
 // Value range of a score vector from its first kSample entries: leaves in shared memory the lower end,
 // the scale that maps the sampled range onto bins 1 .. kBins-2, and `fallback` when the sample is not
 // finite or has no width.  Every CTA that is given the same sample arrives at the same numbers.
-__device__ void compute_range(SelectSmem& s, const float* __restrict__ sample, int n_sample) {
+// *lopsided (optional): nine tenths of the sample lie in a sixteenth of its range, at either end.
+__device__ void compute_range(SelectSmem& s, const float* __restrict__ sample, int n_sample, bool* lopsided = nullptr) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     float lo = INFINITY, hi = -INFINITY;
     bool finite = true;
@@ -169,8 +172,28 @@ __device__ void compute_range(SelectSmem& s, const float* __restrict__ sample, i
         s.lo = lo;
         s.scale = s.fallback ? 0.f : scale;
         s.n_cand = 0;
+        s.cnt[0][1][0] = 0; s.cnt[1][1][0] = 0;
     }
     __syncthreads();
+    if (lopsided != nullptr) {
+        *lopsided = false;
+        if (!s.fallback && n_sample >= 512) {
+            const float lo1 = s.lo, sixteenth = (float)(kBins - 2) / s.scale * 0.0625f;
+            int low = 0, high = 0;
+#pragma unroll
+            for (int u = 0; u < kSample / kThreads; ++u)
+                if (u * kThreads + tid < n_sample) { low += smp[u] < lo1 + sixteenth; high += smp[u] > lo1 + 15.f * sixteenth; }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) {
+                low += __shfl_xor_sync(0xffffffffu, low, d);
+                high += __shfl_xor_sync(0xffffffffu, high, d);
+            }
+            if (lane == 0) { atomicAdd(&s.cnt[0][1][0], low); atomicAdd(&s.cnt[1][1][0], high); }
+            __syncthreads();
+            const int n_smp = min(n_sample, kSample);
+            *lopsided = 10 * s.cnt[0][1][0] > 9 * n_smp || 10 * s.cnt[1][1][0] > 9 * n_smp;
+        }
+    }
 }
 
 // Bin of a score: monotone in v (subtraction, multiplication by a positive constant, clamping and
@@ -234,8 +257,36 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
 __device__ bool threshold_with_counts(SelectSmem& s, const float* __restrict__ sc, int n, int want_total,
                                       uint32_t* thr_out, int* ties_out) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    compute_range(s, sc, n);
+    bool lopsided = false;
+    compute_range(s, sc, n, &lopsided);
     if (s.fallback) return false;
+    // A few extreme scores among the sampled ones (the first token of a real context is one) stretch the range so
+    // that the bulk lands in a handful of bins: all atomics of the histogram pass would then hit the same words.
+    // So if nine tenths of the sample lie in a sixteenth of its range, the sample is binned, and if 99 % of it sit in
+    // less than an eighth of the bins the range is narrowed to them (values outside fall into the end bins, as before);
+    // the check is repeated once.
+    const int n_smp = min(n, kSample);
+    if (lopsided) {
+        for (int round = 0; round < 2; ++round) {
+            const float lo0 = s.lo, scale0 = s.scale;
+            for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
+            __syncthreads();
+            for (int i = tid; i < n_smp; i += kThreads) atomicAdd(&s.hist[bin_of(sc[i], lo0, scale0)], 1);
+            __syncthreads();
+            pick_bin(s, kBins, n_smp / 200 + 1);
+            const int b_hi = s.bin;
+            __syncthreads();
+            pick_bin(s, kBins, n_smp - n_smp / 200);
+            const int b_lo = s.bin;
+            __syncthreads();
+            if (b_hi - b_lo + 1 >= kBins / 8) break;
+            const float new_lo = lo0 + (float)(b_lo - 1) / scale0;
+            const float new_scale = (float)(kBins - 2) * scale0 / (float)(b_hi - b_lo + 1);
+            if (!(isfinite(new_lo) && isfinite(new_scale) && new_scale > 0.f)) break;
+            if (tid == 0) { s.lo = new_lo; s.scale = new_scale; }
+            __syncthreads();
+        }
+    }
     const float lo = s.lo, scale = s.scale;
     for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
     __syncthreads();
@@ -246,10 +297,49 @@ __device__ bool threshold_with_counts(SelectSmem& s, const float* __restrict__ s
     });
     const int any_nonfinite = __syncthreads_or(nonfinite);
     pick_bin(s, kBins, want_total);
-    const int tbin = s.bin, want = s.remaining;
-    const int members = s.hist[tbin];
+    const int tbin = s.bin;
+    int want = s.remaining;
+    int members = s.hist[tbin];
     __syncthreads();
+    // A few extreme scores among the sampled ones (the first token of a real context is one) stretch the range so that
+    // the bulk lands in a handful of bins, too crowded for the list: then a second histogram over the threshold bin
+    // alone, 2046 times finer, and the threshold bin of that.
+    bool refined = false;
+    float lo2 = 0.f, scale2 = 0.f;
+    int tbin2 = 0;
+    if (!any_nonfinite && members > kCand && tbin > 0 && tbin < kBins - 1) {
+        lo2 = lo + (float)(tbin - 1) / scale;
+        scale2 = scale * (float)(kBins - 2);
+        if (isfinite(lo2) && isfinite(scale2)) {
+            for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
+            __syncthreads();
+            for_each_score(sc, n, [&](float v) {
+                if (bin_of(v, lo, scale) == tbin) atomicAdd(&s.hist[bin_of(v, lo2, scale2)], 1);
+            });
+            __syncthreads();
+            pick_bin(s, kBins, want);
+            tbin2 = s.bin;
+            want = s.remaining;
+            members = s.hist[tbin2];
+            __syncthreads();
+            refined = true;
+        }
+    }
     if (any_nonfinite || members > kCand) return false;
+    // rank of a score: its bin, and inside the threshold bin its finer bin (both maps are monotone in the score);
+    // 2 = above the threshold's bin, 1 = in it, 0 = below
+    const bool fine = refined;
+    const float f_lo = lo2, f_scale = scale2;
+    const int f_bin = tbin2;
+    auto placed = [=](float x) -> int {
+        const int bin = bin_of(x, lo, scale);
+        int code = bin > tbin ? 2 : (bin == tbin ? 1 : 0);
+        if (fine && code == 1) {
+            const int bin2 = bin_of(x, f_lo, f_scale);
+            code = bin2 > f_bin ? 2 : (bin2 == f_bin ? 1 : 0);
+        }
+        return code;
+    };
 
     const int head = min(n, (int)((4 - ((reinterpret_cast<uintptr_t>(sc) >> 2) & 3)) & 3));
     const int n_vec = (n - head) >> 2;
@@ -263,29 +353,41 @@ __device__ bool threshold_with_counts(SelectSmem& s, const float* __restrict__ s
     };
     int above = 0;
     constexpr int kAhead = 4;
-    for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
-        float4 q[kAhead];
+    auto stretch = [&](auto fine_tag) {                    // the warp's stretch; the refined test only where it is needed
+        constexpr bool kFine = decltype(fine_tag)::value;
+        for (int v0 = vbegin; v0 < vend; v0 += 32 * kAhead) {
+            float4 q[kAhead];
 #pragma unroll
-        for (int u = 0; u < kAhead; ++u) {
-            const int vi = v0 + u * 32 + lane;
-            q[u] = vi < vend ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
+            for (int u = 0; u < kAhead; ++u) {
+                const int vi = v0 + u * 32 + lane;
+                q[u] = vi < vend ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
 #pragma unroll
-        for (int u = 0; u < kAhead; ++u) {
-            if (v0 + u * 32 + lane < vend) {
-                const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+            for (int u = 0; u < kAhead; ++u) {
+                if (v0 + u * 32 + lane < vend) {
+                    const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int bin = bin_of(x[j], lo, scale);
-                    above += bin > tbin;
-                    if (bin == tbin) candidate(x[j], warp);
+                    for (int j = 0; j < 4; ++j) {
+                        if (kFine) {
+                            const int code = placed(x[j]);
+                            above += code >> 1;
+                            if (code == 1) candidate(x[j], warp);
+                        } else {
+                            const int bin = bin_of(x[j], lo, scale);
+                            above += bin > tbin;
+                            if (bin == tbin) candidate(x[j], warp);
+                        }
+                    }
                 }
             }
         }
-    }
-    if (tid < head) { if (bin_of(sc[tid], lo, scale) == tbin) candidate(sc[tid], 255); }
-    for (int i = head + 4 * n_vec + tid; i < n; i += kThreads)
-        if (bin_of(sc[i], lo, scale) == tbin) candidate(sc[i], 255);
+    };
+    if (fine) stretch(std::true_type{}); else stretch(std::false_type{});
+    auto loose = [&](float x) {                           // the few scores outside the 16-byte aligned body
+        if (placed(x) == 1) candidate(x, 255);
+    };
+    if (tid < head) loose(sc[tid]);
+    for (int i = head + 4 * n_vec + tid; i < n; i += kThreads) loose(sc[i]);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xffffffffu, above, d);
     if (lane == 0) { s.cnt[0][0][warp] = above; s.cnt[1][0][warp] = 0; }

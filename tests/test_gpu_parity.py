@@ -235,6 +235,31 @@ def test_select_few_long_units_spread_over_several_ctas(B):
             np.testing.assert_array_equal(got, orc.top_k_indices(seg, keep[b]), err_msg=f"{h},{b}")
 
 
+@pytest.mark.parametrize("ties", [False, True])
+def test_select_with_a_few_extreme_scores_at_the_start(B, ties):
+    # leverage scores of a real context: a bulk near m/n and a first token near one.  The extreme score is among the
+    # sampled ones and stretches the histogram's range; the selection then refines the crowded bin (or, with heavy
+    # ties, falls back) and must stay exact
+    rng = np.random.default_rng(23)
+    n, keep = 131072, 39322
+    s = (48.0 / n) * (1.0 + 0.3 * rng.standard_normal((2, 2, n)))
+    s = np.abs(s).astype(np.float32)
+    if ties:
+        s = np.round(s, 5)
+    s[..., 0] = 1.0
+    s[..., 1] = 0.5
+    s[0, 1, 77777] = 0.9
+    shape = B.Shape(2, 2, 128, 48, [n])
+    sc = torch.from_numpy(s).cuda()
+    idx = torch.full((2, 2, keep), -1, dtype=torch.int32, device="cuda")
+    B.select(shape, sc, [keep], idx, B.alloc_workspace(shape))
+    torch.cuda.synchronize()
+    idx = idx.cpu().numpy()
+    for l in range(2):
+        for h in range(2):
+            np.testing.assert_array_equal(idx[l, h], orc.top_k_indices(s[l, h].astype(np.float64), keep), err_msg=f"{l},{h}")
+
+
 def test_compact_bit_exact_and_skips_bad_indices(B):
     w = inputs.Workload("compact", 2, 2, 128, [700, 300], [0.5, 0.5], seed=51)
     _, kr, v = inputs.make_tensors(w, device="cpu", want_pre=False)

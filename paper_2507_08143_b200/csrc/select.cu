@@ -246,6 +246,32 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
     });
 }
 
+// Narrows the range left by compute_range() to the bins that hold 99 % of the sample (values outside fall into
+// the end bins, as before), as long as those are less than half of all bins (three times at most).  Every CTA that
+// is given the same sample arrives at the same range.
+__device__ void narrow_range(SelectSmem& s, const float* __restrict__ sc, int n_smp) {
+    const int tid = threadIdx.x;
+    for (int round = 0; round < 3; ++round) {
+        const float lo0 = s.lo, scale0 = s.scale;
+        for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
+        __syncthreads();
+        for (int i = tid; i < n_smp; i += kThreads) atomicAdd(&s.hist[bin_of(sc[i], lo0, scale0)], 1);
+        __syncthreads();
+        pick_bin(s, kBins, n_smp / 200 + 1);
+        const int b_hi = s.bin;
+        __syncthreads();
+        pick_bin(s, kBins, n_smp - n_smp / 200);
+        const int b_lo = s.bin;
+        __syncthreads();
+        if (b_hi - b_lo + 1 >= kBins / 2) break;
+        const float new_lo = lo0 + (float)(b_lo - 1) / scale0;
+        const float new_scale = (float)(kBins - 2) * scale0 / (float)(b_hi - b_lo + 1);
+        if (!(isfinite(new_lo) && isfinite(new_scale) && new_scale > 0.f)) break;
+        if (tid == 0) { s.lo = new_lo; s.scale = new_scale; }
+        __syncthreads();
+    }
+}
+
 // The threshold of one finite score vector together with what the ordered pass needs to start: per warp
 // stretch (the same cut as emit_ordered's) the number of scores above and at the threshold.  First pass:
 // the value-linear histogram (this is the pass that brings the scores in from HBM).  Second pass: a warp
@@ -265,28 +291,7 @@ __device__ bool threshold_with_counts(SelectSmem& s, const float* __restrict__ s
     // So if nine tenths of the sample lie in a sixteenth of its range, the sample is binned, and if 99 % of it sit in
     // less than an eighth of the bins the range is narrowed to them (values outside fall into the end bins, as before);
     // the check is repeated once.
-    const int n_smp = min(n, kSample);
-    if (lopsided) {
-        for (int round = 0; round < 2; ++round) {
-            const float lo0 = s.lo, scale0 = s.scale;
-            for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
-            __syncthreads();
-            for (int i = tid; i < n_smp; i += kThreads) atomicAdd(&s.hist[bin_of(sc[i], lo0, scale0)], 1);
-            __syncthreads();
-            pick_bin(s, kBins, n_smp / 200 + 1);
-            const int b_hi = s.bin;
-            __syncthreads();
-            pick_bin(s, kBins, n_smp - n_smp / 200);
-            const int b_lo = s.bin;
-            __syncthreads();
-            if (b_hi - b_lo + 1 >= kBins / 8) break;
-            const float new_lo = lo0 + (float)(b_lo - 1) / scale0;
-            const float new_scale = (float)(kBins - 2) * scale0 / (float)(b_hi - b_lo + 1);
-            if (!(isfinite(new_lo) && isfinite(new_scale) && new_scale > 0.f)) break;
-            if (tid == 0) { s.lo = new_lo; s.scale = new_scale; }
-            __syncthreads();
-        }
-    }
+    if (lopsided) narrow_range(s, sc, min(n, kSample));
     const float lo = s.lo, scale = s.scale;
     for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;
     __syncthreads();
@@ -692,11 +697,13 @@ multi_hist_kernel(Plan p, const float* __restrict__ scores, MultiSelect m) {
     const int tid = threadIdx.x;
     int* st = m.state + (size_t)c.group * kSelStateInts;
     const float* first = scores + (size_t)(c.lh - c.hi) * p.total_tokens + p.cu_seqlens[c.b];   // the group's first head
-    compute_range(s, first, c.n);
+    bool lopsided = false;
+    compute_range(s, first, c.n, &lopsided);
     if (s.fallback) {
         if (tid == 0) atomicOr(&st[kStFlags], 1);
         return;
     }
+    if (lopsided) narrow_range(s, first, min(c.n, kSample));
     const float lo = s.lo, scale = s.scale;
     if (c.part == 0 && c.hi == 0 && tid == 0) { st[kStLo] = __float_as_int(lo); st[kStScale] = __float_as_int(scale); }
     for (int i = tid; i < kBins; i += kThreads) s.hist[i] = 0;

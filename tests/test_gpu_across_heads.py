@@ -124,3 +124,16 @@ def test_across_heads_scores_that_defeat_the_histogram(B):
     s[1] *= 1e-4
     s[1, 0, 3] = 1000.0; s[1, 0, 9] = -1000.0              # the range estimate spans 2000, the bulk 1e-3
     _select_and_check(B, shape, torch.from_numpy(s).cuda(), [30000, 700])
+
+
+def test_across_heads_with_extreme_scores_at_the_start(B):
+    # a real context's first tokens have leverage scores near one, the rest near m/n: the sampled range is lopsided and
+    # every CTA of the group narrows it in the same way
+    rng = np.random.default_rng(8)
+    n = 150000
+    shape = B.Shape(1, 4, 128, 48, [n])
+    s = np.abs((48.0 / n) * (1.0 + 0.3 * rng.standard_normal((1, 4, n)))).astype(np.float32)
+    s[..., 0] = 1.0
+    s[..., 1] = 0.6
+    s[0, 2, 99999] = 0.8
+    _select_and_check(B, shape, torch.from_numpy(s).cuda(), [45000])

@@ -441,3 +441,25 @@ def test_dependent_launches_change_nothing(B, monkeypatch):
             for x, y in zip(serial, chained):
                 assert torch.equal(x.view(torch.int16) if x.dtype == torch.bfloat16 else x,
                                    y.view(torch.int16) if y.dtype == torch.bfloat16 else y)
+
+
+def test_sequences_that_start_with_a_dominant_token(B):
+    # the first token of a real context has keys of far larger norm than the rest (an "attention sink"): its leverage
+    # score is near one, the Gram matrix is dominated by its direction, and the selection sees one extreme score first
+    w = inputs.Workload("sink", 2, 2, 128, [5000, 700, 40000], [0.3, 0.5, 0.2], p=0.7, seed=29)
+    kp, kr, v = [t.cuda() for t in inputs.make_tensors(w, device="cpu")]
+    shape = B.Shape(w.layers, w.heads, w.d, w.m, w.seqlens)
+    for b in range(w.batch):
+        start = shape.cu_seqlens[b]
+        kp[:, :, start] *= 30.0
+        kr[:, :, start] *= 30.0
+        kp[:, :, start + 1] *= 8.0
+        kr[:, :, start + 1] *= 8.0
+    phi = inputs.make_sketch_matrix(w.d, w.m, w.seed)
+    keep = _keep(B, w)
+    outs = H.run_compress(B, shape, kp, kr, v, phi, keep)
+    worst, band = H.compare_all_units(shape, keep, outs, kp, kr, v, phi, what="sink")
+    assert int(outs[4].max()) == 0
+    scores = outs[0]
+    assert float(scores[:, :, 0].min()) > 0.5            # the dominant token is most of a direction of its own
+    print(f"dominant first tokens: max rel score err {worst:.2e}, boundary band {band}")

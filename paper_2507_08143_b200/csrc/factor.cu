@@ -26,7 +26,7 @@ using namespace factor_math;
 // rounding inside the Gram partials would dominate the scores; their Gram matrix is summed in
 // fp64 straight from the keys instead (the work is tiny).
 constexpr int kExactGramTokens = 256;
-constexpr int kStageTokens = 8;
+constexpr int kStageTokens = 16;
 
 constexpr int kSlices = kFactorSlices;     // CTAs per unit in the projection
 constexpr int kRows = kD / kSlices;        // rows of C per CTA

@@ -90,6 +90,32 @@ def test_workspace_bytes():
     assert B.workspace_bytes(B.Shape(1, 2, 128, 48, [1024, 0, 77])) > 0   # empty sequences are fine
 
 
+def test_workspace_sizes_of_the_other_entry_points():
+    # selection across heads needs, per (layer, sequence), a histogram, a candidate list that grows with heads x n,
+    # and two counts per slice; the one-call entry point needs the fused call's workspace plus what its options add
+    shape = B.Shape(4, 8, 128, 48, [131072, 300, 0])
+    tables = 256 * math.ceil(16 * (shape.batch + 1) / 256)
+    across = B.across_heads_workspace_bytes(shape)
+    groups = 4 * shape.batch
+    assert across >= tables + groups * 2176 * 4 + 8 * (8 * shape.total_tokens // 256) and across % 256 == 0
+    assert across < B.workspace_bytes(shape)
+    base = B.workspace_bytes(shape)
+    per_head = B.compress_full_workspace_bytes(shape, B.options(selection=B.SELECT_PER_HEAD))
+    with_across = B.compress_full_workspace_bytes(shape, B.options(selection=B.SELECT_ACROSS_HEADS))
+    with_attn = B.compress_full_workspace_bytes(shape, B.options(selection=B.SELECT_ACROSS_HEADS, q_per_kv=4, pool=7))
+    plane = 4 * 4 * 8 * shape.total_tokens
+    assert base <= per_head < with_across < with_attn
+    assert with_attn - with_across >= 2 * plane          # the attention term and its unpooled copy
+    # a ragged batch of the same size is planned with long blocks too: its Gram partials stay a small part of the workspace
+    ragged = B.Shape(32, 8, 128, 48, [2278, 9042, 23584, 54094])
+    uniform = B.Shape(32, 8, 128, 48, [22250] * 4)
+    units, lh = 32 * 8 * 4, 32 * 8
+    fixed = 4 * lh * ragged.total_tokens + units * (2 * 48 * 128 * 2 + 128 * 48 * 8)       # scores, W, T = C Phi
+    partials = (B.workspace_bytes(ragged) - fixed) // (128 * 128 * 8 * lh)                  # Gram blocks per (layer, head)
+    assert partials == 5                                  # blocks of 32768 tokens: 1 + 1 + 1 + 2
+    assert B.workspace_bytes(ragged) < B.workspace_bytes(uniform)
+
+
 def _mat(ptr=1 << 20, sl=1 << 20, sh=1 << 17, st=128):
     return B.CompactorMat(ptr, sl, sh, st)
 

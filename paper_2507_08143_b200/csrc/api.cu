@@ -231,7 +231,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
         const double ctas = (double)count_chunks(c) * lh;
         const double waves = ceil(ctas / kFallbackSmCount);
-        const double per_cta_us = 4.0 + c * 256.0 / 44e3;
+        const double per_cta_us = 4.0 + (double)(hp->max_n < c ? hp->max_n : c) * 256.0 / 44e3;   // a block is never longer than the sequence
         const double partial_us = ctas * 2.0 * 131072.0 / 6.4e6;      // written once, read once at 6.4 TB/s
         const double cost = (ragged ? ragged_cost(c, 4.0) : waves * per_cta_us) + partial_us;
         if (cost < best * 0.999) { best = cost; chunk = c; }
@@ -250,7 +250,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     best = 1e300;
     for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
         const double ctas = (double)count_chunks(c) * lh;
-        const double per_cta_us = 2.0 + c * 256.0 / 44e3;
+        const double per_cta_us = 2.0 + (double)(hp->max_n < c ? hp->max_n : c) * 256.0 / 44e3;
         const double cost = ragged ? ragged_cost(c, 2.0)
                                    : (ctas / kFallbackSmCount < 1.0 ? 1.0 : ctas / kFallbackSmCount) * per_cta_us + 0.5 * per_cta_us;
         if (cost < best * 0.999) { best = cost; schunk = c; }

@@ -113,7 +113,8 @@ def test_workspace_sizes_of_the_other_entry_points():
     fixed = 4 * lh * ragged.total_tokens + units * (2 * 48 * 128 * 2 + 128 * 48 * 8)       # scores, W, T = C Phi
     partials = (B.workspace_bytes(ragged) - fixed) // (128 * 128 * 8 * lh)                  # Gram blocks per (layer, head)
     assert partials == 5                                  # blocks of 32768 tokens: 1 + 1 + 1 + 2
-    assert B.workspace_bytes(ragged) < B.workspace_bytes(uniform)
+    fixed_u = 4 * lh * uniform.total_tokens + units * (2 * 48 * 128 * 2 + 128 * 48 * 8)
+    assert (B.workspace_bytes(uniform) - fixed_u) // (128 * 128 * 8 * lh) == 4   # one block per sequence of 22250 tokens
 
 
 def _mat(ptr=1 << 20, sl=1 << 20, sh=1 << 17, st=128):

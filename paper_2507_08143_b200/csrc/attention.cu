@@ -181,8 +181,8 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
         };
         const int n_halves = my_items * n_iter;
         bool ok = true;
-        for (int g = 0; g < n_halves && ok; ++g) {
-            const int r = g / n_iter, it = g - r * n_iter, st = g & 1, use = g >> 1;
+        for (int g = 0, r = 0, it = 0; g < n_halves && ok; ++g, it = (it + 1 == n_iter) ? 0 : it + 1, r += (it == 0)) {
+            const int st = g & 1, use = g >> 1;
             if (it == 0) ok = mbar_wait(&s.k_full, r & 1);
             if (ok) ok = mbar_wait(&s.q_full[st], use & 1);
             if (ok && g >= 2) ok = mbar_wait(&s.drained[st], (use - 1) & 1);   // the accumulator's previous column sums are out
@@ -254,8 +254,7 @@ attention_kernel(Plan p, const __grid_constant__ CUtensorMap qmap, const __grid_
             if (*(volatile int*)&s.abort || *(volatile int*)&s.abort_mma) return;
             if (!mbar_wait(bar, parity)) s.abort = 1;
         };
-        for (int g = 0; g < n_halves; ++g) {
-            const int r = g / n_iter, it = g - r * n_iter;
+        for (int g = 0, r = 0, it = 0; g < n_halves; ++g, it = (it + 1 == n_iter) ? 0 : it + 1, r += (it == 0)) {
             if (it == 0 && r > 0) { prev = cur; cur = attn_item(p, blockIdx.x + r * gridDim.x); }
             const int n_tok = cur.n_tok;
             const bool full = n_tok == kChunk;               // only the last chunk of a sequence needs masks

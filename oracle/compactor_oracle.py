@@ -40,8 +40,9 @@ Readings taken where the paper is silent or inconsistent:
     change the scores.
   * Ties in the top-k go to the lower token index, and the kept indices are
     emitted in ascending order (the paper does not say).
-  * std in Eq. 6 is the population standard deviation; a term whose std is 0
-    contributes 0.  With no attention term the score is the outlier score o.
+  * std in Eq. 6 is the population standard deviation; a term without spread
+    (std <= 1e-3 |mean|: constant up to what the scores resolve) contributes 0.
+    With no attention term the score is the outlier score o.
   * The calibration curve is increasing in r; the paper writes the choice of
     r* as an arg max subject to f >= tau, which is read as the smallest such r
     (Section 3.5 states the goal as the least retention that keeps quality).
@@ -201,9 +202,12 @@ def approx_leverage_scores_qr(K: np.ndarray, Phi: np.ndarray) -> np.ndarray:
 # Eq. 6: blend
 # ----------------------------------------------------------------------------
 def _zscore(x: np.ndarray) -> np.ndarray:
+    """Population z-score (Eq. 6).  A vector with no spread has no z-score and contributes nothing; "no spread"
+    is read numerically: a standard deviation of at most 1e-3 of |mean| is below what the scores are asked to
+    resolve (leverage scores of a sequence no longer than the sketch are all one, up to rounding)."""
     mu = np.mean(x)
     sd = np.sqrt(np.mean((x - mu) ** 2))
-    if sd == 0.0:
+    if sd <= 1e-3 * abs(mu):
         return np.zeros_like(x)
     return (x - mu) / sd
 

@@ -942,9 +942,11 @@ blend_kernel(Plan p, const float* __restrict__ attn, float lambda, float* __rest
         va = fma(da, da, va); vo = fma(d_o, d_o, vo);
     }
     block_sum2(va, vo, 2);
+    // a term without spread contributes nothing; "without spread" is a standard deviation of at most 1e-3 of |mean|,
+    // below what the scores resolve (the leverage scores of a sequence no longer than the sketch are all one)
     const double sd_a = sqrt(stats[2] / n), sd_o = sqrt(stats[3] / n);
-    const double inv_a = sd_a > 0.0 ? 1.0 / sd_a : 0.0;
-    const double inv_o = sd_o > 0.0 ? (double)lambda / sd_o : 0.0;
+    const double inv_a = sd_a > 1e-3 * fabs(mean_a) ? 1.0 / sd_a : 0.0;
+    const double inv_o = sd_o > 1e-3 * fabs(mean_o) ? (double)lambda / sd_o : 0.0;
     for (int i = tid; i < n; i += kThreads)
         o[i] = (float)(((double)a[i] - mean_a) * inv_a + ((double)o[i] - mean_o) * inv_o);
 }
@@ -1040,8 +1042,8 @@ blend_apply_kernel(Plan p, const float* __restrict__ attn, float lambda, float* 
         cnt = tot;
     }
     const double sd_a = sqrt(m2_a / n), sd_o = sqrt(m2_o / n);
-    const double inv_a = sd_a > 0.0 ? 1.0 / sd_a : 0.0;
-    const double inv_o = sd_o > 0.0 ? (double)lambda / sd_o : 0.0;
+    const double inv_a = sd_a > 1e-3 * fabs(mean_a) ? 1.0 / sd_a : 0.0;          // as in blend_kernel
+    const double inv_o = sd_o > 1e-3 * fabs(mean_o) ? (double)lambda / sd_o : 0.0;
     const size_t off = (size_t)lh * p.total_tokens + p.cu_seqlens[b];
     const float* a = attn + off;
     float* o = scores + off;

@@ -463,3 +463,11 @@ def test_sequences_that_start_with_a_dominant_token(B):
     scores = outs[0]
     assert float(scores[:, :, 0].min()) > 0.5            # the dominant token is most of a direction of its own
     print(f"dominant first tokens: max rel score err {worst:.2e}, boundary band {band}")
+
+
+def test_blend_with_a_sequence_no_longer_than_the_sketch(B):
+    # n <= m: every leverage score is one up to rounding, the outlier term has no spread and must contribute nothing
+    # (Eq. 6's z-score does not exist for it); an exact-zero test on the standard deviation would blow the rounding up
+    w = inputs.Workload("short-blend", 1, 3, 128, [3000, 47, 30, 700], [0.5, 0.32, 0.5, 0.5], p=0.7, seed=912, m=64)
+    worst, band, outs = _run_workload(B, w, attn=True, device="cpu")
+    print(f"blend with short sequences: err {worst:.2e}")

@@ -263,6 +263,15 @@ def test_blend_properties():
     assert np.array_equal(np.argsort(orc.blend(a, o, 0.0)), np.argsort(a))
     assert np.array_equal(np.argsort(orc.blend(np.full(500, 2.0), o, 0.3)), np.argsort(o))
     np.testing.assert_array_equal(orc.blend(None, o, 0.3), o)
+    # a term that is constant up to rounding has no z-score: the leverage scores of a sequence no longer than the sketch
+    # are all one, through an SVD they come out as 1 +- 1e-15, and the blend must then be z(a) alone
+    ones = 1.0 + 1e-15 * rng.standard_normal(500)
+    np.testing.assert_allclose(orc.blend(a, ones, 0.3), za, rtol=1e-12)
+    np.testing.assert_allclose(orc.blend(ones, o, 0.3), 0.3 * zo, rtol=1e-12)
+    few = rng.standard_normal((30, 128))                 # 30 tokens, sketch of 48: every score is one
+    lev = orc.approx_leverage_scores(few, orc.make_sketch(1, 128, 48))
+    a30 = rng.random(30)
+    np.testing.assert_allclose(orc.blend(a30, lev, 0.3), (a30 - a30.mean()) / a30.std(), rtol=1e-9)
     # hand example: a = (1,3), o = (0,2): z = (-1,1) for both
     np.testing.assert_allclose(orc.blend([1.0, 3.0], [0.0, 2.0], 0.5), [-1.5, 1.5], atol=1e-15)
 

@@ -223,9 +223,16 @@ cholesky_kernel(Plan p, const double* __restrict__ t_buf, const float* __restric
     if (!finite) atomicOr(&s.flags, COMPACTOR_STATUS_NONFINITE);
     __syncthreads();
     const bool bad = (s.flags & COMPACTOR_STATUS_NONFINITE) != 0;
-    if (tid < MP) s.diag0[tid] = s.u.g[tid * MP + tid];
+    // The pivot floor (2^-20 of the original diagonal) is the noise floor of the fp32 Gram sums.  A short sequence's
+    // Gram matrix was summed in fp64 from the keys and has no such noise, while its pivots are legitimately small
+    // (few rows, nearly dependent columns): there the floor is 2^-40 (the reference diagonal is scaled down instead).
+    // What that floor lets through once the rank is used up is rounding amplified by the conditioning of the leading
+    // block; a sequence of n < m tokens has rank n at most, so no more than n pivots are kept.
+    const int n_unit = p.cu_seqlens[unit % p.batch + 1] - p.cu_seqlens[unit % p.batch];
+    const bool exact_gram = n_unit <= kExactGramTokens;
+    if (tid < MP) s.diag0[tid] = s.u.g[tid * MP + tid] * (exact_gram ? 9.5367431640625e-07 : 1.0);
     __syncthreads();
-    if (!bad) cholesky_panels<MP, kCholWarps>(s.u.g, s.diag0, s.inv_diag, m, tid, &s.flags, sync);
+    if (!bad) cholesky_panels<MP, kCholWarps>(s.u.g, s.diag0, s.inv_diag, m, tid, &s.flags, sync, exact_gram ? n_unit : (1 << 30));
     __syncthreads();
     __nv_bfloat16* w_unit = w_out + (size_t)unit * w_elems_per_unit(MP);
     if (!bad) {

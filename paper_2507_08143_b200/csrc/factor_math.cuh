@@ -49,10 +49,12 @@ __device__ __forceinline__ double fast_rsqrt(double x) {
 // solves the panel entries of its own rows (lane, lane + 32, ...) against it.  Also leaves the inverse of
 // the diagonal block's factor, X = L_JJ^-1, below the diagonal in the free triangle of `g`
 // (g[(j0 + n) * LD + j0 + k] = X[n][k], k < n; the diagonal of X is inv_diag).  Pivots not larger than
-// 2^-20 of their original diagonal entry are dropped (their column of L and of X is zero).
-// Returns true if a pivot was dropped.
+// 2^-20 of their original diagonal entry are dropped (their column of L and of X is zero), and so is every pivot
+// once `budget` of them have been kept in this panel (the caller knows an upper bound of the rank).
+// Returns (pivots kept in this panel) * 2 + (1 if a pivot was dropped).
 template <int LD>
-__device__ __noinline__ bool factor_panel(double* g, const double* diag0, double* inv_diag, int j0, int j1, int m, int lane) {
+__device__ __noinline__ int factor_panel(double* g, const double* diag0, double* inv_diag, int j0, int j1, int m, int lane,
+                                         int budget) {
     constexpr int kOwn = (LD + 31) / 32;          // rows per lane: lane, lane + 32, ...
     double dd[kPanel][kPanel];                    // lower triangle of the diagonal block
 #pragma unroll
@@ -76,10 +78,12 @@ __device__ __noinline__ bool factor_panel(double* g, const double* diag0, double
     // Columns past j1 (a short last panel) have a zero pivot: they are "dropped" (zero column) without being counted.
     double inv[kPanel];
     bool dropped = false;
+    int kept = 0;
 #pragma unroll
     for (int c = 0; c < kPanel; ++c) {
         const double piv = dd[c][c], d0 = diag0[min(j0 + c, LD - 1)];
-        const bool keep = piv > kPivotFloor * d0 && d0 > 0.0;
+        const bool keep = piv > kPivotFloor * d0 && d0 > 0.0 && kept < budget;
+        kept += keep;
         inv[c] = keep ? fast_rsqrt(keep ? piv : 1.0) : 0.0;
         dropped = dropped || (!keep && j0 + c < j1);
         dd[c][c] = piv * inv[c];
@@ -125,7 +129,7 @@ __device__ __noinline__ bool factor_panel(double* g, const double* diag0, double
                 if (j0 + n < j1) g[(j0 + n) * LD + j0 + k] = x[n];
         }
     }
-    return dropped;
+    return kept * 2 + (dropped ? 1 : 0);
 }
 
 // W = Phi L^-T for the 16 rows of Phi that one warp owns, as a blocked forward substitution on fp64
@@ -259,16 +263,20 @@ __device__ __forceinline__ bool gram_of_sketch(const double* __restrict__ t_unit
 // right-looking by panels of eight columns: warp 0 factors the panel (factor_panel), all warps update what
 // follows on fp64 mma.  `diag0` must hold the original diagonal and `inv_diag` zeros on entry; on return
 // inv_diag[j] = 1 / L[j][j] (0 for a dropped pivot) and the inverses of the diagonal blocks lie in the free
-// triangle of `g`.  COMPACTOR_STATUS_RANK is or-ed into *flags (shared memory) if a pivot was dropped.
+// triangle of `g`.  COMPACTOR_STATUS_RANK is or-ed into *flags (shared memory) if a pivot was dropped.  `rank_bound`: at
+// most this many pivots are kept (a sequence of fewer tokens than sketch columns cannot have more).
 template <int MP, int NWARPS, class Sync>
-__device__ __forceinline__ void cholesky_panels(double* g, const double* diag0, double* inv_diag, int m, int tid, int* flags, Sync sync) {
+__device__ __forceinline__ void cholesky_panels(double* g, const double* diag0, double* inv_diag, int m, int tid, int* flags, Sync sync,
+                                                int rank_bound = 1 << 30) {
     constexpr int LD = MP;
     const int warp = tid >> 5, lane = tid & 31, fr = lane >> 2, fk = lane & 3;
+    int kept = 0;                                         // pivots kept so far (only warp 0 counts)
     for (int j0 = 0; j0 < m; j0 += kPanel) {
         const int j1 = min(j0 + kPanel, m);
         if (warp == 0) {
-            const bool dropped = factor_panel<LD>(g, diag0, inv_diag, j0, j1, m, lane);
-            if (lane == 0 && dropped) atomicOr(flags, COMPACTOR_STATUS_RANK);
+            const int res = factor_panel<LD>(g, diag0, inv_diag, j0, j1, m, lane, rank_bound - kept);
+            kept += res >> 1;
+            if (lane == 0 && (res & 1)) atomicOr(flags, COMPACTOR_STATUS_RANK);
         }
         sync();
         // trailing block, rows and columns j1 .. : A_ij -= L_i L_j^T by 8 x 8 tiles (lower tiles only; rows and

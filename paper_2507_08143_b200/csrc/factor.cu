@@ -197,8 +197,89 @@ struct CholSmem {
         double g[MP * MP];                 // G, then L by columns (and the inverses of its diagonal blocks)
     } u;
     double diag0[MP], inv_diag[MP];
+    int perm[2 * MP];                      // pivot order and "already a pivot" marks of the pivoted factorisation
     int flags;
 };
+
+// Sequences about as short as the sketch is wide: G = (K Phi)^T (K Phi) has rank n or is nearly singular, and a
+// Cholesky factorisation in the given column order meets pivots that are small differences of large numbers.  Here
+// the factorisation takes the largest remaining diagonal entry as its next pivot (which is stable for positive
+// semi-definite matrices and reveals the rank: it stops at `rank_bound` pivots or when what remains is below 2^-40 of
+// the largest original entry), one CTA per unit, a step at a time: the work is tiny and such units are rare.
+// `a` holds G by columns (lower triangle valid on entry, the whole square is used); W = Phi[:, P] L^-T comes out in
+// pivot order (the order of its columns does not matter to the scores), zero beyond the rank.  Returns the rank.
+template <int MP>
+__device__ int pivoted_factor_and_solve(double* a, const float* phi, int m, int rank_bound, int tid, int* perm, double* red,
+                                        __nv_bfloat16* w_hi) {
+    constexpr int LD = MP;
+    const int lane = tid & 31, warp = tid >> 5;
+    for (int idx = tid; idx < m * m; idx += kCholThreads) {            // both triangles
+        const int i = idx % m, c = idx / m;
+        if (i < c) a[c * LD + i] = a[i * LD + c];
+    }
+    __syncthreads();
+    // block-wide maximum of the remaining diagonal with its index (ties: lower index); perm[MP + i] = 1 once i is a pivot
+    auto arg_max = [&](double& best, int& where) {
+        double v = -1.0; int at = 0x7fffffff;
+        for (int i = tid; i < m; i += kCholThreads)
+            if (perm[MP + i] == 0) { const double d = a[i * LD + i]; if (d > v || (d == v && i < at)) { v = d; at = i; } }
+#pragma unroll
+        for (int dlt = 16; dlt > 0; dlt >>= 1) {
+            const double ov = __shfl_xor_sync(0xffffffffu, v, dlt);
+            const int oa = __shfl_xor_sync(0xffffffffu, at, dlt);
+            if (ov > v || (ov == v && oa < at)) { v = ov; at = oa; }
+        }
+        __syncthreads();                                                 // earlier readers of red are done
+        if (lane == 0) { red[warp] = v; red[kCholWarps + warp] = (double)at; }
+        __syncthreads();
+        best = red[0]; where = (int)red[kCholWarps];
+        for (int w = 1; w < kCholWarps; ++w)
+            if (red[w] > best || (red[w] == best && (int)red[kCholWarps + w] < where)) { best = red[w]; where = (int)red[kCholWarps + w]; }
+    };
+    for (int i = tid; i < m; i += kCholThreads) perm[MP + i] = 0;
+    __syncthreads();
+    double d_first; int at;
+    arg_max(d_first, at);
+    const double floor_abs = d_first * 9.094947017729282e-13;           // 2^-40 of the largest diagonal entry
+    int rank = 0;
+    const int max_rank = min(m, rank_bound);
+    while (rank < max_rank) {
+        double piv; int pj;
+        arg_max(piv, pj);
+        if (!(piv > floor_abs) || !(piv > 0.0)) break;
+        const double ljj = sqrt(piv), inv = 1.0 / ljj;
+        __syncthreads();
+        for (int i = tid; i < m; i += kCholThreads)                     // column pj becomes column `rank` of L (by original row)
+            if (perm[MP + i] == 0) a[pj * LD + i] = (i == pj) ? ljj : a[pj * LD + i] * inv;
+        __syncthreads();
+        if (tid == 0) { perm[rank] = pj; perm[MP + pj] = 1; }
+        __syncthreads();
+        for (int idx = tid; idx < m * m; idx += kCholThreads) {        // what remains: A_ik -= L_i L_k
+            const int i = idx % m, k = idx / m;
+            if (perm[MP + i] == 0 && perm[MP + k] == 0) a[k * LD + i] = fma(-a[pj * LD + i], a[pj * LD + k], a[k * LD + i]);
+        }
+        __syncthreads();
+        ++rank;
+    }
+    // forward substitution, one row of Phi per thread: w_j = (phi[perm j] - sum_{t<j} w_t L[perm j][t]) / L[perm j][j]
+    __nv_bfloat16* w_lo = w_hi + (size_t)MP * kD;
+    for (int row = tid; row < kD; row += kCholThreads) {
+        double w[MP];
+        for (int j = 0; j < rank; ++j) {
+            const int pj = perm[j];
+            double acc = (double)phi[row * MP + pj];
+            for (int t = 0; t < j; ++t) acc = fma(-w[t], a[perm[t] * LD + pj], acc);
+            w[j] = acc / a[pj * LD + pj];
+        }
+        for (int j = 0; j < MP; ++j) {
+            const double v = j < rank ? w[j] : 0.0;
+            const __nv_bfloat16 hi = __double2bfloat16(v);
+            w_hi[j * kD + row] = hi;
+            w_lo[j * kD + row] = __double2bfloat16(v - (double)__bfloat162float(hi));
+        }
+    }
+    return rank;
+}
 
 template <int MP>
 __global__ void __launch_bounds__(kCholThreads, MP <= 48 ? 4 : (MP <= 64 ? 2 : 1))
@@ -230,11 +311,17 @@ cholesky_kernel(Plan p, const double* __restrict__ t_buf, const float* __restric
     // block; a sequence of n < m tokens has rank n at most, so no more than n pivots are kept.
     const int n_unit = p.cu_seqlens[unit % p.batch + 1] - p.cu_seqlens[unit % p.batch];
     const bool exact_gram = n_unit <= kExactGramTokens;
+    __nv_bfloat16* w_unit = w_out + (size_t)unit * w_elems_per_unit(MP);
+    if (!bad && n_unit <= m + 16) {
+        // about as many tokens as sketch columns: G is singular or nearly so, and only a pivoted factorisation is accurate
+        const int rank = pivoted_factor_and_solve<MP>(s.u.g, s.phi, m, n_unit, tid, s.perm, s.diag0, w_unit);
+        if (tid == 0 && status != nullptr && rank < m) atomicOr(&status[unit], COMPACTOR_STATUS_RANK);
+        return;
+    }
     if (tid < MP) s.diag0[tid] = s.u.g[tid * MP + tid] * (exact_gram ? 9.5367431640625e-07 : 1.0);
     __syncthreads();
     if (!bad) cholesky_panels<MP, kCholWarps>(s.u.g, s.diag0, s.inv_diag, m, tid, &s.flags, sync, exact_gram ? n_unit : (1 << 30));
     __syncthreads();
-    __nv_bfloat16* w_unit = w_out + (size_t)unit * w_elems_per_unit(MP);
     if (!bad) {
         for (int rb = warp * 16; rb < kD; rb += kCholWarps * 16) solve_w_tiles<MP>(s.phi, s.u.g, s.inv_diag, rb, lane, w_unit);
     } else {                                              // a unit with non-finite keys gets W = 0

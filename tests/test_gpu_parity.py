@@ -482,3 +482,28 @@ def test_short_sequences_with_a_steep_spectrum(B, p_exp):
     s = outs[0].cpu().numpy()
     np.testing.assert_allclose(s[:, :, :82], 1.0, rtol=1e-3)             # the three sequences with n < m
     print(f"short sequences, spectrum exponent {p_exp}: max rel score err {worst:.2e}")
+
+
+@pytest.mark.parametrize("m", [16, 48, 64, 96, 128])
+def test_fewer_tokens_than_sketch_columns_any_sketch_width(B, m):
+    # n < m: G = (K Phi)^T (K Phi) has rank n; the factorisation picks its pivots by size there (in the given column order
+    # the leading blocks can be arbitrarily ill conditioned) and stops at n.  Every score is one, as the oracle says.
+    for p_exp in (0.7, 1.0):
+        ns = sorted(set([max(1, m // 4), m // 2, m - 8]))
+        w = inputs.Workload("short-any", 1, 2, 128, ns, [0.5] * len(ns), p=p_exp, seed=4000 + m, m=m)
+        kp, kr, v = [t.cuda() for t in inputs.make_tensors(w, device="cpu")]
+        shape = B.Shape(1, 2, 128, m, ns)
+        phi = inputs.make_sketch_matrix(128, m, 1)
+        sc = torch.empty(1, 2, shape.total_tokens, dtype=torch.float32, device="cuda")
+        st = torch.zeros(2 * len(ns), dtype=torch.int32, device="cuda")
+        B.score(shape, kp, phi.cuda(), sc, B.alloc_workspace(shape), status=st)
+        torch.cuda.synchronize()
+        assert np.all(st.cpu().numpy() == 2)              # rank deficient by construction, nothing else
+        cu = shape.cu_seqlens
+        for h in range(2):
+            for b, n in enumerate(ns):
+                K = orc.bf16_bits_to_f64(H.bits(kp[0, h, cu[b]:cu[b + 1]]))
+                want = orc.approx_leverage_scores(K, phi.numpy())
+                got = sc[0, h, cu[b]:cu[b + 1]].cpu().numpy().astype(np.float64)
+                np.testing.assert_allclose(want, 1.0, rtol=1e-6)
+                np.testing.assert_allclose(got, want, rtol=1e-3, err_msg=f"m {m} p {p_exp} n {n}")

@@ -26,7 +26,6 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kBins = 2048;
 constexpr int kSample = 4096;          // scores used to estimate the value range
 constexpr int kCand = 8192;            // capacity of the candidate list
-constexpr int kSub = 8;                // rows of the small shared count table
 
 // Monotone map float -> uint32: larger float <=> larger key; -0 and +0 share a key (adding +0
 // turns -0 into +0) and a NaN with the sign bit clear ranks highest.
@@ -39,8 +38,8 @@ struct SelectSmem {
     int hist[kBins];
     uint32_t cand[kCand];
     unsigned char cand_warp[kCand];   // which warp's stretch a candidate lies in (255: the unaligned head or tail)
-    int cnt[2][kSub][kWarps];      // per-warp packed counts of the ordered pass, double buffered
-    int row_total[2][kSub];
+    int warp_gt[kWarps], warp_eq[kWarps];   // per warp stretch: scores above / at the threshold (ordered pass)
+    int low, high;                 // sampled scores in the lowest / highest sixteenth of the sampled range
     int stage[kWarps][512];        // kept indices of 4 x 128 scores per warp, in output order
     int warp_sums[kWarps];
     float red[2][kWarps];
@@ -172,7 +171,7 @@ __device__ void compute_range(SelectSmem& s, const float* __restrict__ sample, i
         s.lo = lo;
         s.scale = s.fallback ? 0.f : scale;
         s.n_cand = 0;
-        s.cnt[0][1][0] = 0; s.cnt[1][1][0] = 0;
+        s.low = 0; s.high = 0;
     }
     __syncthreads();
     if (lopsided != nullptr) {
@@ -188,10 +187,10 @@ __device__ void compute_range(SelectSmem& s, const float* __restrict__ sample, i
                 low += __shfl_xor_sync(0xffffffffu, low, d);
                 high += __shfl_xor_sync(0xffffffffu, high, d);
             }
-            if (lane == 0) { atomicAdd(&s.cnt[0][1][0], low); atomicAdd(&s.cnt[1][1][0], high); }
+            if (lane == 0) { atomicAdd(&s.low, low); atomicAdd(&s.high, high); }
             __syncthreads();
             const int n_smp = min(n_sample, kSample);
-            *lopsided = 10 * s.cnt[0][1][0] > 9 * n_smp || 10 * s.cnt[1][1][0] > 9 * n_smp;
+            *lopsided = 10 * s.low > 9 * n_smp || 10 * s.high > 9 * n_smp;
         }
     }
 }
@@ -395,7 +394,7 @@ __device__ bool threshold_with_counts(SelectSmem& s, const float* __restrict__ s
     for (int i = head + 4 * n_vec + tid; i < n; i += kThreads) loose(sc[i]);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xffffffffu, above, d);
-    if (lane == 0) { s.cnt[0][0][warp] = above; s.cnt[1][0][warp] = 0; }
+    if (lane == 0) { s.warp_gt[warp] = above; s.warp_eq[warp] = 0; }
     __syncthreads();
     const int nc = s.n_cand;
     uint32_t thr;
@@ -419,8 +418,8 @@ __device__ bool threshold_with_counts(SelectSmem& s, const float* __restrict__ s
     for (int i = tid; i < nc; i += kThreads) {
         const int w = s.cand_warp[i];
         if (w < kWarps) {
-            if (s.cand[i] > thr) atomicAdd(&s.cnt[0][0][w], 1);
-            else if (s.cand[i] == thr) atomicAdd(&s.cnt[1][0][w], 1);
+            if (s.cand[i] > thr) atomicAdd(&s.warp_gt[w], 1);
+            else if (s.cand[i] == thr) atomicAdd(&s.warp_eq[w], 1);
         }
     }
     *thr_out = thr;
@@ -492,12 +491,12 @@ __device__ void emit_ordered(SelectSmem& s, const float* __restrict__ sc, int n,
             cnt_eq += __shfl_xor_sync(0xffffffffu, cnt_eq, d);
         }
         __syncthreads();                                // earlier users of the shared arrays are done
-        if (lane == 0) { s.cnt[0][0][warp] = cnt_gt; s.cnt[1][0][warp] = cnt_eq; }
+        if (lane == 0) { s.warp_gt[warp] = cnt_gt; s.warp_eq[warp] = cnt_eq; }
     }
     __syncthreads();
     int base_gt, base_eq;
     {
-        const int c_gt = s.cnt[0][0][lane], c_eq = s.cnt[1][0][lane];       // kWarps == 32: one pair of counts per lane
+        const int c_gt = s.warp_gt[lane], c_eq = s.warp_eq[lane];       // kWarps == 32: one pair of counts per lane
         int incl_gt = c_gt, incl_eq = c_eq;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {

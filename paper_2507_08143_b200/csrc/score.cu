@@ -53,7 +53,7 @@ struct __align__(1024) ScoreSmem {
 template <int MP>
 __global__ void __launch_bounds__(kThreads, 1)
 score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap,
-             float* __restrict__ scores, int* __restrict__ status) {
+             float* __restrict__ scores, int* __restrict__ status, int chained) {
     extern __shared__ unsigned char smem_raw[];
     using Smem = ScoreSmem<MP>;
     constexpr int kStages = Smem::kStages;
@@ -90,9 +90,10 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
 
     if (warp == 0) {
         if (lane == 0) {
-            // the first key tiles come from the caller and are fetched at once; W is the factor stage's and must wait for it
+            // In a chained launch the first key tiles, which come from the caller, are fetched at once and W, which is the
+            // factor stage's, waits for it; otherwise W goes first (the first product needs it) and the tiles follow.
             int t = 0;
-            for (; t < n_tiles && t < kStages; ++t) {
+            for (; chained && t < n_tiles && t < kStages; ++t) {
                 mbar_arrive_expect_tx(&s.full[t], kTileBytes);
                 const int tok = tok_begin + t * kTile;
                 tma_load_4d(s.tiles[t], &kmap, &s.full[t], 0, tok, head, layer);
@@ -235,7 +236,8 @@ cudaError_t launch_score_mp(const Plan& p, const CUtensorMap& kmap, const CUtens
     cudaError_t e = cudaFuncSetAttribute(score_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(p.total_schunks, p.layers * p.heads);
-    e = launch_chained(kPdlScore, score_kernel<MP>, grid, dim3(kThreads), smem, stream, p, kmap, wmap, scores, status);
+    e = launch_chained(kPdlScore, score_kernel<MP>, grid, dim3(kThreads), smem, stream, p, kmap, wmap, scores, status,
+                       pdl_enabled(kPdlScore) ? 1 : 0);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

@@ -39,7 +39,6 @@ struct SelectSmem {
     uint32_t cand[kCand];
     unsigned char cand_warp[kCand];   // which warp's stretch a candidate lies in (255: the unaligned head or tail)
     int warp_gt[kWarps], warp_eq[kWarps];   // per warp stretch: scores above / at the threshold (ordered pass)
-    int low, high;                 // sampled scores in the lowest / highest sixteenth of the sampled range
     int stage[kWarps][512];        // kept indices of 4 x 128 scores per warp, in output order
     int warp_sums[kWarps];
     float red[2][kWarps];
@@ -102,6 +101,10 @@ __device__ __forceinline__ void for_each_score(const float* __restrict__ sc, int
             const int vi = v0 + u * kThreads + tid;
             q[u] = vi < n_vec ? __ldg(body + vi) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        {   // the next round's lines (128 bytes = 8 vectors each) are asked into L2 while this round is consumed
+            const int vi = v0 + 4 * kThreads + tid * 8;
+            if (tid < kThreads / 2 && vi < n_vec) asm volatile("prefetch.global.L2 [%0];" ::"l"(body + vi));
+        }
 #pragma unroll
         for (int u = 0; u < 4; ++u)
             if (v0 + u * kThreads + tid < n_vec) { f(q[u].x); f(q[u].y); f(q[u].z); f(q[u].w); }
@@ -163,34 +166,39 @@ __device__ void compute_range(SelectSmem& s, const float* __restrict__ sample, i
     const int all_finite = __syncthreads_and(finite ? 1 : 0);
     if (lane == 0) { s.red[0][warp] = lo; s.red[1][warp] = hi; }
     __syncthreads();
+    if (warp == 0) {                                                   // kWarps == 32: one pair per lane
+        lo = s.red[0][lane]; hi = s.red[1][lane];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+        }
+    }
     if (tid == 0) {
-        for (int w = 1; w < kWarps; ++w) { lo = fminf(lo, s.red[0][w]); hi = fmaxf(hi, s.red[1][w]); }
         const float width = hi - lo;
         const float scale = (float)(kBins - 2) / width;              // sampled range -> bins 1 .. kBins-2
         s.fallback = !(all_finite && width > 0.f && isfinite(width) && isfinite(scale));
         s.lo = lo;
         s.scale = s.fallback ? 0.f : scale;
         s.n_cand = 0;
-        s.low = 0; s.high = 0;
     }
     __syncthreads();
     if (lopsided != nullptr) {
         *lopsided = false;
         if (!s.fallback && n_sample >= 512) {
             const float lo1 = s.lo, sixteenth = (float)(kBins - 2) / s.scale * 0.0625f;
-            int low = 0, high = 0;
+            int both = 0;                                               // low in bits 0-15, high in bits 16-31
 #pragma unroll
             for (int u = 0; u < kSample / kThreads; ++u)
-                if (u * kThreads + tid < n_sample) { low += smp[u] < lo1 + sixteenth; high += smp[u] > lo1 + 15.f * sixteenth; }
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) {
-                low += __shfl_xor_sync(0xffffffffu, low, d);
-                high += __shfl_xor_sync(0xffffffffu, high, d);
-            }
-            if (lane == 0) { atomicAdd(&s.low, low); atomicAdd(&s.high, high); }
+                if (u * kThreads + tid < n_sample)
+                    both += (smp[u] < lo1 + sixteenth ? 1 : 0) + (smp[u] > lo1 + 15.f * sixteenth ? 1 << 16 : 0);
+            both = __reduce_add_sync(0xffffffffu, both);
+            if (lane == 0) s.warp_sums[warp] = both;
             __syncthreads();
+            both = __reduce_add_sync(0xffffffffu, s.warp_sums[lane]);   // kWarps == 32: one sum per lane
+            const int low = both & 0xffff, high = both >> 16;
             const int n_smp = min(n_sample, kSample);
-            *lopsided = 10 * s.low > 9 * n_smp || 10 * s.high > 9 * n_smp;
+            *lopsided = 10 * low > 9 * n_smp || 10 * high > 9 * n_smp;
         }
     }
 }
@@ -248,7 +256,7 @@ __device__ uint32_t find_threshold(SelectSmem& s, Visit visit, const float* __re
 // Narrows the range left by compute_range() to the bins that hold 99 % of the sample (values outside fall into
 // the end bins, as before), as long as those are less than half of all bins (three times at most).  Every CTA that
 // is given the same sample arrives at the same range.
-__device__ void narrow_range(SelectSmem& s, const float* __restrict__ sc, int n_smp) {
+__device__ __noinline__ void narrow_range(SelectSmem& s, const float* __restrict__ sc, int n_smp) {
     const int tid = threadIdx.x;
     for (int round = 0; round < 3; ++round) {
         const float lo0 = s.lo, scale0 = s.scale;
@@ -642,6 +650,7 @@ select_kernel(Plan p, const float* __restrict__ scores, int* __restrict__ idx_ou
 //   4. ordered emission of every slice at its offset.
 // Per-group scratch words: histogram, range, candidate counter, flags, per-head counts.
 constexpr int kStLo = kBins, kStScale = kBins + 1, kStCand = kBins + 2, kStFlags = kBins + 3, kStAbove = kBins + 4;
+static_assert(kWarps == 32, "block-wide sums take one warp, one partial per lane");
 static_assert(kStAbove + 64 <= kSelStateInts, "per-group scratch too small");
 static_assert(kCand / 2 >= 64 * 64, "per-slice counts of a group live in the candidate array");
 

@@ -232,7 +232,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
         const double ctas = (double)count_chunks(c) * lh;
         const double waves = ceil(ctas / kFallbackSmCount);
         const double per_cta_us = 4.0 + (double)(hp->max_n < c ? hp->max_n : c) * 256.0 / 44e3;   // a block is never longer than the sequence
-        const double partial_us = ctas * 2.0 * 131072.0 / 6.4e6;      // written once, read once at 6.4 TB/s
+        const double partial_us = ctas * 2.0 * 131072.0 / 6.4e6;      // written once, read once (a whole 128 x 128 fp64 matrix at 6.4 TB/s fits the measurements; ten of its sixteen blocks move)
         const double cost = (ragged ? ragged_cost(c, 4.0) : waves * per_cta_us) + partial_us;
         if (cost < best * 0.999) { best = cost; chunk = c; }
     }
@@ -276,7 +276,7 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     size_t off = 0;
     hp->off_tables = off;   off += align_up(sizeof(int) * 4 * nb1);
     hp->off_w = off;        off += align_up(sizeof(__nv_bfloat16) * w_elems_per_unit(p.mp) * hp->units);
-    hp->off_gpart = off;    off += align_up(sizeof(double) * kD * p.mp * hp->units);             // T = C Phi per unit
+    hp->off_gpart = off;    off += align_up(sizeof(double) * a_elems_per_unit(p.mp) * hp->units);   // the parts of A = Phi^T M Phi per unit
     hp->off_partials = off; off += align_up(sizeof(double) * kGramElems * (size_t)p.total_chunks * s->layers * s->heads);
     hp->off_scores = off;   off += align_up(sizeof(float) * (size_t)p.total_tokens * s->layers * s->heads);
     hp->total_bytes = off;

@@ -14,7 +14,8 @@ constexpr int kMaxChunk = 65536;   // most tokens per block (one CTA of a stream
 constexpr int kMinChunk = 256;
 constexpr int kGramFlushTokens = 512;    // most tokens whose Gram matrix is summed in fp32 (tensor-core accumulators) before going to fp64
 constexpr int kGramElems = kD * kD;
-constexpr int kFactorSlices = 4;   // CTAs per unit that share the fp64 projection of the Gram matrix
+constexpr int kFactorSlices = 4;   // 32-row slices of the Gram matrix in its fp64 projection
+constexpr int kFactorParts = 2;    // parts of A (G = A + A^T) per unit, one per pair of slices and work item
 
 // Device-side view of one call: shapes plus the four prefix-sum tables that live at the start
 // of the workspace.  Passed to kernels by value.
@@ -111,7 +112,7 @@ inline cudaError_t launch_chained(int which, void (*kernel)(KArgs...), dim3 grid
 // Kernel launchers (each defined next to its kernel).  All enqueue on `stream` and return the
 // launch status.
 cudaError_t launch_gram(const Plan& p, const Mat& k, double* partials, int* status, cudaStream_t stream);
-cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* t_buf,
+cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* a_parts,
                           __nv_bfloat16* w, int* status, int factorization, double eig_floor, int sm_count,
                           cudaStream_t stream);
 cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
@@ -185,5 +186,11 @@ cudaError_t launch_attention(const Plan& p, const Mat& q, const Mat& k, int q_pe
 
 // Bytes of W (two bf16 terms, [term][mp][128]) per unit.
 __host__ __device__ inline size_t w_elems_per_unit(int mp) { return (size_t)2 * mp * kD; }
+// doubles per unit between the projection and the factorisation: the parts of A (never less than what one T = C Phi takes,
+// which the one-kernel sweep keeps there)
+__host__ __device__ inline size_t a_elems_per_unit(int mp) {
+    const size_t parts = (size_t)kFactorParts * mp * mp, t = (size_t)kD * mp;
+    return parts > t ? parts : t;
+}
 
 }  // namespace compactor

@@ -1,10 +1,14 @@
 // Small factorisation (Algorithm 1, line 4, by the Cholesky route that Section 3.2 and
 // Appendix C allow), in two kernels, all fp64:
 //
-//   project_kernel   four CTAs per unit, each owning 32 rows of C = sum of the unit's Gram
-//                    partials: T[rows,:] = C[rows,:] Phi on fp64 mma.m8n8k4 (this is where the
-//                    fp64 work is: 0.8 M multiply-adds per unit, spread over the whole device).
-//   cholesky_kernel  one small CTA per unit, several per SM: G = Phi^T T (fp64 mma), G = L L^T by
+//   project_kernel   two work items per unit.  C = sum of the unit's Gram partials is symmetric, so
+//                    G = Phi^T C Phi = A + A^T with A = Phi^T M Phi, M the half of C below the
+//                    diagonal (plus half the diagonal).  An item takes two of the four 32-row
+//                    slices of M, forms their rows of M Phi and then their share of A on fp64
+//                    mma.m8n8k4 (this is where the fp64 work is: 0.8 M multiply-adds per unit,
+//                    spread over the whole device) and writes an m x m part of A.
+//   cholesky_kernel  one small CTA per unit, several per SM: G = sum of the parts and their
+//                    transposes, G = L L^T by
 //                    panels of eight columns (the 8 x 8 diagonal blocks are factored redundantly
 //                    by every lane of a warp, so no pivot has to travel), then W = Phi L^-T as a
 //                    blocked substitution on fp64 mma, split into two bf16 terms.  The score of a
@@ -28,162 +32,288 @@ using namespace factor_math;
 constexpr int kExactGramTokens = 256;
 constexpr int kStageTokens = 16;
 
-constexpr int kSlices = kFactorSlices;     // CTAs per unit in the projection
-constexpr int kRows = kD / kSlices;        // rows of C per CTA
+// The sketch [128][m] from global memory into shared memory as [128][MP] with row stride LD (columns from m on are
+// zero), eight loads per thread in flight at a time (a plain copy loop waits for every load in turn).
+template <int MP, int LD, int NTHREADS, class T>
+__device__ __forceinline__ void load_sketch(T* dst, const float* __restrict__ phi, int m, int tid) {
+    constexpr int kBatch = 8;
+    static_assert(kD * MP % (kBatch * NTHREADS) == 0, "whole batches");
+    for (int i0 = tid; i0 < kD * MP; i0 += kBatch * NTHREADS) {
+        float v[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int i = i0 + u * NTHREADS, row = i / MP, col = i - row * MP;
+            v[u] = __ldg(phi + row * m + min(col, m - 1));          // unconditional, masked below
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int i = i0 + u * NTHREADS, row = i / MP, col = i - row * MP;
+            dst[row * LD + col] = col < m ? (T)v[u] : (T)0;
+        }
+    }
+}
+
+constexpr int kSlices = kFactorSlices;     // 32-row slices of C per unit
+constexpr int kRows = kD / kSlices;        // rows of C per slice
+constexpr int kPairs = kFactorParts;       // work items per unit: slices s and kSlices-1-s together cost the same for every s
 constexpr int kProjThreads = 256;
+static_assert(kSlices == 2 * kPairs, "slices are paired");
 
 template <int MP>
 struct ProjectSmem {
     static constexpr int kLd = MP + 4;     // row stride (doubles): the four k-rows of a B fragment land in distinct banks
     double phi[kD * kLd];                  // Phi widened, [channel][column]
     static constexpr int kLdc = kRows + 4; // stride of a k-row of c: the four k-rows of an A fragment land in distinct banks
-    double c[kD * kLdc];                   // C[k][row0 + i] at [k * kLdc + i]  (C is symmetric)
-    double keys[kStageTokens * kD];
+    double c[kD * kLdc];                   // the slice of the triangular half of C, [k][row0 + i] at [k * kLdc + i]
+    union {
+        double keys[kStageTokens * kD];    // short sequences: staged key rows
+        double t[kRows * kLd];             // the slice's rows of the half product, until they are multiplied by Phi^T
+    } u;
 };
 
-// Persistent: each CTA loads Phi once and then walks (unit, slice) items with a grid stride.
+// C is symmetric, so G = Phi^T C Phi = A + A^T with A = Phi^T M Phi, where M is the part of C below the diagonal plus half of
+// the diagonal.  Only that half is read (the Gram pass writes only the blocks it needs) and multiplied:
+// a slice of 32 rows of M has non-zeros in its first 32 (s + 1) columns only.  Each item takes two slices of a unit
+// (s and 3 - s: five blocks of 32 x 32 whatever s is), forms their rows of M Phi, multiplies them by the matching rows of
+// Phi^T and writes the sum, an MP x MP part of A; the factor kernel adds the parts of a unit and their transposes.
+// Persistent: each CTA loads Phi once and then walks the items with a grid stride.
 template <int MP>
 __global__ void __launch_bounds__(kProjThreads, 2)
 project_kernel(Plan p, Mat kmat, const double* __restrict__ partials, const float* __restrict__ phi,
-               double* __restrict__ t_buf, int n_items) {
+               double* __restrict__ a_parts, int n_items) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using Smem = ProjectSmem<MP>;
     Smem& s = *reinterpret_cast<Smem*>(smem_raw);
     constexpr int LD = Smem::kLd;
-    constexpr int kPer = kD * kRows / kProjThreads;     // elements of the C slice per thread: e = tid + 256 q
-    constexpr int kInFlight = 1;                        // partials loaded together (more would spill at two CTAs per SM)
+    constexpr int LDC = Smem::kLdc;
     constexpr int kWarps = kProjThreads / 32;
     const int m = p.m, tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int fr = lane >> 2, fk = lane & 3;            // fragment coordinates: A[fr][fk], B[fk][fr], C[fr][2 fk, 2 fk + 1]
     constexpr int kNT = MP / 8;                         // 8-column tiles
+    constexpr int kATiles = kNT * kNT;                  // 8 x 8 tiles of a part of A
+    constexpr int kAGroup = 8;                          // tiles of A a warp holds in registers at a time
+    constexpr int kAPer = (kATiles + kWarps - 1) / kWarps;
+    constexpr bool kKeepA = kAPer <= kAGroup;           // a part of A stays in registers over both slices (else: added up in global memory)
+    constexpr int kAHeld = kKeepA ? kAPer : kAGroup;
 
     pdl_trigger();
-    for (int i = tid; i < kD * MP; i += kProjThreads) {   // Phi, widened
-        const int row = i / MP, col = i - row * MP;
-        s.phi[row * LD + col] = (col < m) ? (double)__ldg(phi + row * m + col) : 0.0;
-    }
+    load_sketch<MP, LD, kProjThreads>(s.phi, phi, m, tid);   // Phi, widened
     pdl_wait();                                           // the Gram partials are complete
 
-    // Item bookkeeping and the look-ahead loads.
-    struct Item { int unit, slice, b, lh, n_part, n_tok; const double* part; };
-    auto decode = [&](int item) {
-        Item it;
-        it.unit = item / kSlices; it.slice = item % kSlices;
-        it.b = it.unit % p.batch; it.lh = it.unit / p.batch;
-        const int chunk_begin = p.cu_chunks[it.b];
-        it.n_part = p.cu_chunks[it.b + 1] - chunk_begin;
-        it.n_tok = p.cu_seqlens[it.b + 1] - p.cu_seqlens[it.b];
-        it.part = partials + ((size_t)it.lh * p.total_chunks + chunk_begin) * kGramElems;
-        return it;
-    };
-    constexpr int LDC = Smem::kLdc;
-    // Two CTAs share an SM: while one waits for its partial sums the other multiplies.
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const Item cur = decode(item);
-        const Item done = cur;
-        const int row0 = cur.slice * kRows;
-        // ---- the item's 32 columns of C (= 32 rows, by symmetry), summed over the partials ------
-        if (cur.n_tok > kExactGramTokens) {
-            double acc[kPer];
+        const int unit = item / kPairs, pair = item % kPairs;
+        const int b = unit % p.batch, lh = unit / p.batch;
+        const int chunk_begin = p.cu_chunks[b];
+        const int n_part = p.cu_chunks[b + 1] - chunk_begin;
+        const int n_tok = p.cu_seqlens[b + 1] - p.cu_seqlens[b];
+        const double* part = partials + ((size_t)lh * p.total_chunks + chunk_begin) * kGramElems;
+        double* a_out = a_parts + (size_t)unit * a_elems_per_unit(MP) + (size_t)pair * MP * MP;
+        double a[kAHeld][2];
 #pragma unroll
-            for (int q = 0; q < kPer; ++q) acc[q] = 0.0;
-            for (int pp = 0; pp < cur.n_part; pp += kInFlight) {
-                double v[kInFlight][kPer];
-#pragma unroll
-                for (int u = 0; u < kInFlight; ++u) {
-                    // unconditional loads (a partial past the last one re-reads the last and is not added): loads under
-                    // a per-load condition are issued one after the other instead of together
-                    const int uu = pp + u < cur.n_part ? pp + u : cur.n_part - 1;
-#pragma unroll
-                    for (int q = 0; q < kPer; ++q) {
-                        const int e = tid + q * kProjThreads;
-                        v[u][q] = __ldcs(cur.part + (size_t)uu * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < kInFlight; ++u)
-                    if (pp + u < cur.n_part) {
-#pragma unroll
-                        for (int q = 0; q < kPer; ++q) acc[q] += v[u][q];
-                    }
-            }
-            __syncthreads();                              // the previous item's products are done with c
-#pragma unroll
-            for (int q = 0; q < kPer; ++q) {
-                const int e = tid + q * kProjThreads;
-                s.c[(e / kRows) * LDC + (e % kRows)] = acc[q];
-            }
-        } else {
-            // short sequence: fp64 Gram straight from the keys, C[:, rows] = K^T K[:, rows], as fp64 mma.m8n8k4
-            // over four tokens at a time
-            const int layer = cur.lh / p.heads, head = cur.lh % p.heads;
-            const __nv_bfloat16* kbase = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
-                                         (long long)p.cu_seqlens[cur.b] * kmat.stride_token;
-            constexpr int kTilesPerWarp = (kD / 8) * (kRows / 8) / kWarps;
-            double d[kTilesPerWarp][2];
-#pragma unroll
-            for (int j = 0; j < kTilesPerWarp; ++j) d[j][0] = d[j][1] = 0.0;
-            // the keys of the next stage are on their way while the current stage is multiplied
-            constexpr int kLoads = kStageTokens * kD / kProjThreads;
-            float nxt[kLoads];
-            auto fetch = [&](int t0) {                    // missing tokens of the last stage are zeros
-#pragma unroll
-                for (int u = 0; u < kLoads; ++u) {
-                    const int i = tid + u * kProjThreads, t = min(t0 + i / kD, cur.n_tok - 1);
-                    nxt[u] = __bfloat162float(kbase[(long long)t * kmat.stride_token + (i % kD)]);
-                    if (t0 + i / kD >= cur.n_tok) nxt[u] = 0.f;
-                }
-            };
-            if (cur.n_tok > 0) fetch(0);
-            for (int t0 = 0; t0 < cur.n_tok; t0 += kStageTokens) {
-                __syncthreads();
-#pragma unroll
-                for (int u = 0; u < kLoads; ++u) s.keys[tid + u * kProjThreads] = (double)nxt[u];
-                __syncthreads();
-                if (t0 + kStageTokens < cur.n_tok) fetch(t0 + kStageTokens);
-#pragma unroll
-                for (int ks = 0; ks < kStageTokens / 4; ++ks) {
-                    const double* krow = s.keys + (ks * 4 + fk) * kD;          // token ks*4 + fk of the stage
-#pragma unroll
-                    for (int j = 0; j < kTilesPerWarp; ++j) {
-                        const int tile = warp + j * kWarps;
-                        const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
-                        mma_f64(d[j], krow[mt * 8 + fr], krow[row0 + nt8 * 8 + fr]);   // A[channel][token], B[token][channel of the slice]
-                    }
-                }
-            }
-            __syncthreads();                              // the previous item's products are done with c
-#pragma unroll
-            for (int j = 0; j < kTilesPerWarp; ++j) {
-                const int tile = warp + j * kWarps;
-                const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
-                s.c[(mt * 8 + fr) * LDC + nt8 * 8 + 2 * fk] = d[j][0];
-                s.c[(mt * 8 + fr) * LDC + nt8 * 8 + 2 * fk + 1] = d[j][1];
-            }
-        }
-        __syncthreads();
+        for (int si = 0; si < kAHeld; ++si) a[si][0] = a[si][1] = 0.0;
 
-        // ---- T[rows] (32 x MP) = C[rows,:] (32 x 128) Phi (128 x MP): a warp-wide fp64 mma does 256 multiply-adds for two
-        // 8-byte shared-memory loads per lane; the contraction is cut into four independent chains --------------------
-        double* t_rows = t_buf + ((size_t)done.unit * kD + row0) * MP;
-        for (int tile = warp; tile < (kRows / 8) * kNT; tile += kWarps) {
-            const int mt = tile / kNT, nt = tile % kNT;
-            double d[4][2];
+        // One slice: kS is its number as a type, so that every loop below has constant bounds.
+        auto do_slice = [&](auto slice_tag, bool second) {
+            constexpr int kS = decltype(slice_tag)::value;
+            constexpr int kmax = kRows * (kS + 1);                   // columns of M that this slice can have non-zeros in
+            constexpr int kPer = kmax * kRows / kProjThreads;        // elements of the slice per thread: e = tid + 256 q
+            constexpr int kInFlight = kPer <= 4 ? 4 : (kPer <= 8 ? 2 : 1);   // partials loaded together
+            const int row0 = kS * kRows;
+            // element (k, i) of the slice is M[row0 + i][k] = C[k][row0 + i] below the diagonal, half of it on the diagonal
+            auto masked = [&](int k, int i, double v) {
+                const int kk = k - row0;
+                return kk < i ? v : (kk == i ? 0.5 * v : 0.0);
+            };
+            if (n_tok > kExactGramTokens) {
+                double acc[kPer];
 #pragma unroll
-            for (int g = 0; g < 4; ++g) d[g][0] = d[g][1] = 0.0;
+                for (int q = 0; q < kPer; ++q) acc[q] = 0.0;
+                for (int pp = 0; pp < n_part; pp += kInFlight) {
+                    double v[kInFlight][kPer];
 #pragma unroll
-            for (int k0 = 0; k0 < kD / 4; k0 += 4) {
+                    for (int u = 0; u < kInFlight; ++u) {
+                        // unconditional loads (a partial past the last one re-reads the last and is not added): loads under
+                        // a per-load condition are issued one after the other instead of together
+                        const int uu = pp + u < n_part ? pp + u : n_part - 1;
 #pragma unroll
-                for (int g = 0; g < 4; ++g) {
-                    const int k = g * (kD / 4) + k0 + fk;
-                    mma_f64(d[g], s.c[k * LDC + mt * 8 + fr], s.phi[k * LD + nt * 8 + fr]);   // A[row][k] = C[k][row0 + row], B[k][col]
+                        for (int q = 0; q < kPer; ++q) {
+                            const int e = tid + q * kProjThreads;
+                            v[u][q] = __ldcs(part + (size_t)uu * kGramElems + (e / kRows) * kD + row0 + (e % kRows));
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < kInFlight; ++u)
+                        if (pp + u < n_part) {
+#pragma unroll
+                            for (int q = 0; q < kPer; ++q) acc[q] += v[u][q];
+                        }
+                }
+                __syncthreads();                              // the previous slice's products are done with c
+#pragma unroll
+                for (int q = 0; q < kPer; ++q) {
+                    const int e = tid + q * kProjThreads;
+                    s.c[(e / kRows) * LDC + (e % kRows)] = masked(e / kRows, e % kRows, acc[q]);
+                }
+            } else {
+                // short sequence: fp64 Gram straight from the keys, C[:, rows] = K^T K[:, rows], as fp64 mma.m8n8k4
+                // over four tokens at a time (only the 8-row tiles that the slice needs)
+                const int layer = lh / p.heads, head = lh % p.heads;
+                const __nv_bfloat16* kbase = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
+                                             (long long)p.cu_seqlens[b] * kmat.stride_token;
+                constexpr int kTilesPerWarp = (kD / 8) * (kRows / 8) / kWarps;
+                double d[kTilesPerWarp][2];
+#pragma unroll
+                for (int j = 0; j < kTilesPerWarp; ++j) d[j][0] = d[j][1] = 0.0;
+                // the keys of the next stage are on their way while the current stage is multiplied
+                constexpr int kLoads = kStageTokens * kD / kProjThreads;
+                float nxt[kLoads];
+                auto fetch = [&](int t0) {                    // missing tokens of the last stage are zeros
+#pragma unroll
+                    for (int u = 0; u < kLoads; ++u) {
+                        const int i = tid + u * kProjThreads, t = min(t0 + i / kD, n_tok - 1);
+                        nxt[u] = __bfloat162float(kbase[(long long)t * kmat.stride_token + (i % kD)]);
+                        if (t0 + i / kD >= n_tok) nxt[u] = 0.f;
+                    }
+                };
+                if (n_tok > 0) fetch(0);
+                for (int t0 = 0; t0 < n_tok; t0 += kStageTokens) {
+                    __syncthreads();                          // the previous stage, and the previous slice's products, are done
+#pragma unroll
+                    for (int u = 0; u < kLoads; ++u) s.u.keys[tid + u * kProjThreads] = (double)nxt[u];
+                    __syncthreads();
+                    if (t0 + kStageTokens < n_tok) fetch(t0 + kStageTokens);
+#pragma unroll
+                    for (int ks = 0; ks < kStageTokens / 4; ++ks) {
+                        const double* krow = s.u.keys + (ks * 4 + fk) * kD;        // token ks*4 + fk of the stage
+#pragma unroll
+                        for (int j = 0; j < kTilesPerWarp; ++j) {
+                            const int tile = warp + j * kWarps;
+                            const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
+                            if (mt * 8 < kmax)
+                                mma_f64(d[j], krow[mt * 8 + fr], krow[row0 + nt8 * 8 + fr]);   // A[channel][token], B[token][channel of the slice]
+                        }
+                    }
+                }
+                __syncthreads();                              // the previous slice's products are done with c
+#pragma unroll
+                for (int j = 0; j < kTilesPerWarp; ++j) {
+                    const int tile = warp + j * kWarps;
+                    const int mt = tile / (kRows / 8), nt8 = tile % (kRows / 8);
+                    if (mt * 8 < kmax) {
+                        s.c[(mt * 8 + fr) * LDC + nt8 * 8 + 2 * fk] = masked(mt * 8 + fr, nt8 * 8 + 2 * fk, d[j][0]);
+                        s.c[(mt * 8 + fr) * LDC + nt8 * 8 + 2 * fk + 1] = masked(mt * 8 + fr, nt8 * 8 + 2 * fk + 1, d[j][1]);
+                    }
                 }
             }
-            __stcg(reinterpret_cast<double2*>(t_rows + (size_t)(mt * 8 + fr) * MP + nt * 8 + 2 * fk),
-                   make_double2((d[0][0] + d[1][0]) + (d[2][0] + d[3][0]), (d[0][1] + d[1][1]) + (d[2][1] + d[3][1])));
+            __syncthreads();
+
+            // ---- (M Phi)[rows] (32 x MP) = M[rows, :kmax] Phi[:kmax] : a warp-wide fp64 mma does 256 multiply-adds for two
+            // 8-byte shared-memory loads per lane; the contraction is cut into four independent chains --------------------
+            for (int tile = warp; tile < (kRows / 8) * kNT; tile += kWarps) {
+                const int mt = tile / kNT, nt = tile % kNT;
+                double d[4][2];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) d[g][0] = d[g][1] = 0.0;
+#pragma unroll
+                for (int k0 = 0; k0 < kmax / 4; k0 += 4) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const int k = g * (kmax / 4) + k0 + fk;
+                        mma_f64(d[g], s.c[k * LDC + mt * 8 + fr], s.phi[k * LD + nt * 8 + fr]);   // A[row][k] = M[row0 + row][k], B[k][col]
+                    }
+                }
+                *reinterpret_cast<double2*>(&s.u.t[(mt * 8 + fr) * LD + nt * 8 + 2 * fk]) =
+                    make_double2((d[0][0] + d[1][0]) + (d[2][0] + d[3][0]), (d[0][1] + d[1][1]) + (d[2][1] + d[3][1]));
+            }
+            __syncthreads();
+
+            // ---- the slice's share of the part of A: Phi[rows]^T (MP x 32) times those rows (32 x MP) ---------------------
+            if constexpr (kKeepA) {
+#pragma unroll
+                for (int si = 0; si < kAPer; ++si) {
+                    const int tile = warp + si * kWarps;
+                    if (tile < kATiles) {
+                        const int mt = tile / kNT, nt = tile % kNT;
+#pragma unroll
+                        for (int k0 = 0; k0 < kRows; k0 += 4)
+                            mma_f64(a[si], s.phi[(row0 + k0 + fk) * LD + mt * 8 + fr], s.u.t[(k0 + fk) * LD + nt * 8 + fr]);
+                    }
+                }
+            } else {
+                for (int g0 = 0; g0 < kAPer; g0 += kAGroup) {
+#pragma unroll
+                    for (int si = 0; si < kAGroup; ++si) {
+                        const int tile = warp + (g0 + si) * kWarps;
+                        if (tile >= kATiles) continue;
+                        const int mt = tile / kNT, nt = tile % kNT;
+                        double* out = a_out + (size_t)(mt * 8 + fr) * MP + nt * 8 + 2 * fk;
+                        double2 sum = make_double2(0.0, 0.0);
+                        if (second) sum = __ldcg(reinterpret_cast<const double2*>(out));     // what this thread wrote for the first slice
+                        a[si][0] = sum.x; a[si][1] = sum.y;
+#pragma unroll
+                        for (int k0 = 0; k0 < kRows; k0 += 4)
+                            mma_f64(a[si], s.phi[(row0 + k0 + fk) * LD + mt * 8 + fr], s.u.t[(k0 + fk) * LD + nt * 8 + fr]);
+                        __stcg(reinterpret_cast<double2*>(out), make_double2(a[si][0], a[si][1]));
+                    }
+                }
+            }
+        };
+        if (pair == 0) {
+            do_slice(std::integral_constant<int, 0>{}, false);
+            do_slice(std::integral_constant<int, kSlices - 1>{}, true);
+        } else {
+            do_slice(std::integral_constant<int, 1>{}, false);
+            do_slice(std::integral_constant<int, kSlices - 2>{}, true);
+        }
+        if constexpr (kKeepA) {
+#pragma unroll
+            for (int si = 0; si < kAPer; ++si) {
+                const int tile = warp + si * kWarps;
+                if (tile < kATiles) {
+                    const int mt = tile / kNT, nt = tile % kNT;
+                    __stcg(reinterpret_cast<double2*>(a_out + (size_t)(mt * 8 + fr) * MP + nt * 8 + 2 * fk), make_double2(a[si][0], a[si][1]));
+                }
+            }
         }
     }
+}
+
+// G = sum over the unit's parts of (A + A^T), the 8 x 8 tiles on and below the diagonal, by columns
+// (g[c * MP + i] = G[i][c]); the loads of four elements per thread are in flight together.  Returns false in a
+// thread that met an entry that is not finite.
+template <int MP, int NTHREADS>
+__device__ __forceinline__ bool gram_from_parts(const double* __restrict__ a_unit, double* g, int tid) {
+    constexpr int kNT = MP / 8, kElems = kNT * (kNT + 1) / 2 * 64, kBatch = 4;
+    bool finite = true;
+    for (int e0 = tid; e0 < kElems; e0 += kBatch * NTHREADS) {
+        double v[kBatch][2 * kPairs];
+        int at[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int e = min(e0 + u * NTHREADS, kElems - 1);       // unconditional loads; the surplus is not stored
+            int rem = e >> 6, mt = 0;
+            while (rem > mt) { rem -= mt + 1; ++mt; }                // tile number -> (mt, nt = rem), mt >= nt
+            const int i = mt * 8 + (e & 7), c = rem * 8 + ((e >> 3) & 7);
+            at[u] = c * MP + i;
+#pragma unroll
+            for (int part = 0; part < kPairs; ++part) {
+                v[u][2 * part] = __ldcg(a_unit + (size_t)part * MP * MP + i * MP + c);
+                v[u][2 * part + 1] = __ldcg(a_unit + (size_t)part * MP * MP + c * MP + i);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            double sum = 0.0;
+#pragma unroll
+            for (int j = 0; j < 2 * kPairs; ++j) sum += v[u][j];
+            if (e0 + u * NTHREADS < kElems) {
+                g[at[u]] = sum;
+                finite = finite && isfinite(sum);
+            }
+        }
+    }
+    return finite;
 }
 
 constexpr int kCholThreads = 128;
@@ -192,10 +322,7 @@ constexpr int kCholWarps = kCholThreads / 32;
 template <int MP>
 struct CholSmem {
     float phi[kD * MP];                    // the sketch, zero in the padded columns
-    union {
-        double t[kTRows * (MP + 4)];       // staged rows of T while G is formed
-        double g[MP * MP];                 // G, then L by columns (and the inverses of its diagonal blocks)
-    } u;
+    double g[MP * MP];                     // G, then L by columns (and the inverses of its diagonal blocks)
     double diag0[MP], inv_diag[MP];
     int perm[2 * MP];                      // pivot order and "already a pivot" marks of the pivoted factorisation
     int flags;
@@ -283,7 +410,7 @@ __device__ int pivoted_factor_and_solve(double* a, const float* phi, int m, int 
 
 template <int MP>
 __global__ void __launch_bounds__(kCholThreads, MP <= 48 ? 4 : (MP <= 64 ? 2 : 1))
-cholesky_kernel(Plan p, const double* __restrict__ t_buf, const float* __restrict__ phi,
+cholesky_kernel(Plan p, const double* __restrict__ a_parts, const float* __restrict__ phi,
                 __nv_bfloat16* __restrict__ w_out, int* __restrict__ status) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     CholSmem<MP>& s = *reinterpret_cast<CholSmem<MP>*>(chol_smem_raw);
@@ -292,15 +419,12 @@ cholesky_kernel(Plan p, const double* __restrict__ t_buf, const float* __restric
 
     pdl_trigger();
     if (tid == 0) s.flags = 0;
-    for (int i = tid; i < kD * MP; i += kCholThreads) {
-        const int row = i / MP, col = i - row * MP;
-        s.phi[i] = col < m ? __ldg(phi + row * m + col) : 0.f;
-    }
+    load_sketch<MP, MP, kCholThreads>(s.phi, phi, m, tid);
     if (tid < MP) s.inv_diag[tid] = 0.0;
-    pdl_wait();                                           // T = C Phi of every unit is complete
+    pdl_wait();                                           // the parts of A of every unit are complete
     __syncthreads();
     auto sync = [] { __syncthreads(); };
-    const bool finite = gram_of_sketch<MP, kCholWarps>(t_buf + (size_t)unit * kD * MP, s.phi, s.u.g, s.u.t, tid, sync);
+    const bool finite = gram_from_parts<MP, kCholThreads>(a_parts + (size_t)unit * a_elems_per_unit(MP), s.g, tid);
     if (!finite) atomicOr(&s.flags, COMPACTOR_STATUS_NONFINITE);
     __syncthreads();
     const bool bad = (s.flags & COMPACTOR_STATUS_NONFINITE) != 0;
@@ -314,16 +438,16 @@ cholesky_kernel(Plan p, const double* __restrict__ t_buf, const float* __restric
     __nv_bfloat16* w_unit = w_out + (size_t)unit * w_elems_per_unit(MP);
     if (!bad && n_unit <= m + 16) {
         // about as many tokens as sketch columns: G is singular or nearly so, and only a pivoted factorisation is accurate
-        const int rank = pivoted_factor_and_solve<MP>(s.u.g, s.phi, m, n_unit, tid, s.perm, s.diag0, w_unit);
+        const int rank = pivoted_factor_and_solve<MP>(s.g, s.phi, m, n_unit, tid, s.perm, s.diag0, w_unit);
         if (tid == 0 && status != nullptr && rank < m) atomicOr(&status[unit], COMPACTOR_STATUS_RANK);
         return;
     }
-    if (tid < MP) s.diag0[tid] = s.u.g[tid * MP + tid] * (exact_gram ? 9.5367431640625e-07 : 1.0);
+    if (tid < MP) s.diag0[tid] = s.g[tid * MP + tid] * (exact_gram ? 9.5367431640625e-07 : 1.0);
     __syncthreads();
-    if (!bad) cholesky_panels<MP, kCholWarps>(s.u.g, s.diag0, s.inv_diag, m, tid, &s.flags, sync, exact_gram ? n_unit : (1 << 30));
+    if (!bad) cholesky_panels<MP, kCholWarps>(s.g, s.diag0, s.inv_diag, m, tid, &s.flags, sync, exact_gram ? n_unit : (1 << 30));
     __syncthreads();
     if (!bad) {
-        for (int rb = warp * 16; rb < kD; rb += kCholWarps * 16) solve_w_tiles<MP>(s.phi, s.u.g, s.inv_diag, rb, lane, w_unit);
+        for (int rb = warp * 16; rb < kD; rb += kCholWarps * 16) solve_w_tiles<MP>(s.phi, s.g, s.inv_diag, rb, lane, w_unit);
     } else {                                              // a unit with non-finite keys gets W = 0
         for (int e = tid; e < (int)w_elems_per_unit(MP); e += kCholThreads) w_unit[e] = __float2bfloat16(0.f);
     }
@@ -342,7 +466,6 @@ struct EigSmem {
     static constexpr int kLd = MP + 1;
     double a[MP * kLd];          // G, driven to diagonal form
     double v[MP * kLd];          // accumulated rotations: columns are the eigenvectors (first: G by columns, as it is formed)
-    double t[kTRows * (MP + 4)]; // staged rows of T while G is formed
     float phi[kD * MP];
     double rot_c[MP / 2], rot_s[MP / 2];
     int rot_p[MP / 2], rot_q[MP / 2];
@@ -353,7 +476,7 @@ struct EigSmem {
 
 template <int MP>
 __global__ void __launch_bounds__(kEigThreads, 3)
-eig_kernel(Plan p, const double* __restrict__ t_buf, const float* __restrict__ phi, double floor,
+eig_kernel(Plan p, const double* __restrict__ a_parts, const float* __restrict__ phi, double floor,
            __nv_bfloat16* __restrict__ w_out, int* __restrict__ status) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using Smem = EigSmem<MP>;
@@ -367,14 +490,10 @@ eig_kernel(Plan p, const double* __restrict__ t_buf, const float* __restrict__ p
     if (tid == 0) s.flags = 0;
     __syncthreads();
     {
-        // G = Phi^T T on fp64 mma into `v` (by columns, lower triangle), then mirrored into `a`
-        for (int i = tid; i < kD * MP; i += kEigThreads) {
-            const int row = i / MP, col = i - row * MP;
-            s.phi[i] = col < m ? __ldg(phi + row * m + col) : 0.f;
-        }
+        // G from its parts into `v` (by columns, lower triangle), then mirrored into `a`
+        load_sketch<MP, MP, kEigThreads>(s.phi, phi, m, tid);
         __syncthreads();
-        auto sync = [] { __syncthreads(); };
-        const bool finite = gram_of_sketch<MP, kEigThreads / 32>(t_buf + (size_t)unit * kD * MP, s.phi, s.v, s.t, tid, sync);
+        const bool finite = gram_from_parts<MP, kEigThreads>(a_parts + (size_t)unit * a_elems_per_unit(MP), s.v, tid);
         if (!finite) atomicOr(&s.flags, COMPACTOR_STATUS_NONFINITE);
         __syncthreads();
         for (int e = tid; e < MP * MP; e += kEigThreads) {
@@ -520,16 +639,16 @@ eig_kernel(Plan p, const double* __restrict__ t_buf, const float* __restrict__ p
 
 template <int MP>
 cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials, const float* phi,
-                             double* t_buf, __nv_bfloat16* w, int* status, int factorization, double eig_floor,
+                             double* a_parts, __nv_bfloat16* w, int* status, int factorization, double eig_floor,
                              int sm_count, cudaStream_t stream) {
     const int units = p.layers * p.heads * p.batch;
     const int smem = (int)sizeof(ProjectSmem<MP>);
     cudaError_t e = cudaFuncSetAttribute(project_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
-    const int n_items = units * kSlices;
+    const int n_items = units * kPairs;
     const int resident = 2 * sm_count;                            // two CTAs fit on an SM
     const int grid = n_items < resident ? n_items : resident;
-    e = launch_chained(kPdlProject, project_kernel<MP>, dim3(grid), dim3(kProjThreads), smem, stream, p, k, partials, phi, t_buf, n_items);
+    e = launch_chained(kPdlProject, project_kernel<MP>, dim3(grid), dim3(kProjThreads), smem, stream, p, k, partials, phi, a_parts, n_items);
     if (e != cudaSuccess) return e;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -538,7 +657,7 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
             const int esmem = (int)sizeof(EigSmem<MP>);
             e = cudaFuncSetAttribute(eig_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, esmem);
             if (e != cudaSuccess) return e;
-            eig_kernel<MP><<<units, kEigThreads, esmem, stream>>>(p, t_buf, phi, eig_floor, w, status);
+            eig_kernel<MP><<<units, kEigThreads, esmem, stream>>>(p, a_parts, phi, eig_floor, w, status);
         } else {
             return cudaErrorInvalidValue;        // two m x m fp64 matrices no longer fit in shared memory
         }
@@ -546,7 +665,7 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
         const int csmem = (int)sizeof(CholSmem<MP>);
         e = cudaFuncSetAttribute(cholesky_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, csmem);
         if (e != cudaSuccess) return e;
-        e = launch_chained(kPdlCholesky, cholesky_kernel<MP>, dim3(units), dim3(kCholThreads), csmem, stream, p, (const double*)t_buf, phi, w, status);
+        e = launch_chained(kPdlCholesky, cholesky_kernel<MP>, dim3(units), dim3(kCholThreads), csmem, stream, p, (const double*)a_parts, phi, w, status);
         if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();
@@ -554,16 +673,16 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
 
 }  // namespace
 
-cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* t_buf,
+cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* a_parts,
                           __nv_bfloat16* w, int* status, int factorization, double eig_floor, int sm_count,
                           cudaStream_t stream) {
     if (p.layers * p.heads * p.batch == 0) return cudaSuccess;
     switch (p.mp) {
-        case 16: return launch_factor_mp<16>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
-        case 32: return launch_factor_mp<32>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
-        case 48: return launch_factor_mp<48>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
-        case 64: return launch_factor_mp<64>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
-        case 128: return launch_factor_mp<128>(p, k, partials, phi, t_buf, w, status, factorization, eig_floor, sm_count, stream);
+        case 16: return launch_factor_mp<16>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
+        case 32: return launch_factor_mp<32>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
+        case 48: return launch_factor_mp<48>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
+        case 64: return launch_factor_mp<64>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
+        case 128: return launch_factor_mp<128>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
         default: return cudaErrorInvalidValue;
     }
 }

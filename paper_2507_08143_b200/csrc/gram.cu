@@ -10,7 +10,8 @@
 // into fp64 registers (64 columns of one row per thread) while the other accumulator fills; the
 // fp64 sums go to global memory once, at the end of the block.  So no fp32 sum is longer than
 // 512 tokens, whatever the block length: the tensor-core accumulator loses accuracy in proportion
-// to the length of the run.
+// to the length of the run.  C_p is symmetric: of its sixteen 32 x 32 blocks only the ten on and
+// above the diagonal are summed and written (the projection reads no others).
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -135,6 +136,7 @@ gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, double* __restrict
             tc_fence_after_sync();
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
+                if (half * 2 + c0 / 32 < q) continue;         // a block below the diagonal: its mirror image is kept
                 uint32_t r[32];
                 tmem_ld_32x32b_x32(tmem + ((uint32_t)(q * 32) << 16) + buf * 128 + half * 64 + c0, r);
                 tmem_ld_wait();
@@ -149,7 +151,8 @@ gram_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, double* __restrict
         if (ok) {
             double* out = partials + ((size_t)lh * p.total_chunks + chunk_id) * kGramElems + (size_t)row * kD + half * 64;
 #pragma unroll
-            for (int i = 0; i < 64; i += 2) *reinterpret_cast<double2*>(out + i) = make_double2(acc[i], acc[i + 1]);
+            for (int i = 0; i < 64; i += 2)
+                if (half * 2 + i / 32 >= q) *reinterpret_cast<double2*>(out + i) = make_double2(acc[i], acc[i + 1]);
         }
     }
     tc_fence_before_sync();

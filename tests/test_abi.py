@@ -110,7 +110,7 @@ def test_workspace_sizes_of_the_other_entry_points():
     ragged = B.Shape(32, 8, 128, 48, [2278, 9042, 23584, 54094])
     uniform = B.Shape(32, 8, 128, 48, [22250] * 4)
     units, lh = 32 * 8 * 4, 32 * 8
-    fixed = 4 * lh * ragged.total_tokens + units * (2 * 48 * 128 * 2 + 128 * 48 * 8)       # scores, W, T = C Phi
+    fixed = 4 * lh * ragged.total_tokens + units * (2 * 48 * 128 * 2 + 128 * 48 * 8)       # scores, W, the parts of A = Phi^T M Phi (G = A + A^T)
     partials = (B.workspace_bytes(ragged) - fixed) // (128 * 128 * 8 * lh)                  # Gram blocks per (layer, head)
     assert partials == 5                                  # blocks of 32768 tokens: 1 + 1 + 1 + 2
     fixed_u = 4 * lh * uniform.total_tokens + units * (2 * 48 * 128 * 2 + 128 * 48 * 8)

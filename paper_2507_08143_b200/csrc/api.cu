@@ -250,9 +250,20 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     best = 1e300;
     for (int c = kMinChunk; c <= kMaxChunk; c *= 2) {
         const double ctas = (double)count_chunks(c) * lh;
-        const double per_cta_us = 2.0 + (double)(hp->max_n < c ? hp->max_n : c) * 256.0 / 44e3;
-        const double cost = ragged ? ragged_cost(c, 2.0)
-                                   : (ctas / kFallbackSmCount < 1.0 ? 1.0 : ctas / kFallbackSmCount) * per_cta_us + 0.5 * per_cta_us;
+        const double block_bytes = (double)(hp->max_n < c ? hp->max_n : c) * 256.0;
+        const double per_cta_us = 2.0 + block_bytes / 44e3;
+        double cost = ragged ? ragged_cost(c, 2.0)
+                             : (ctas / kFallbackSmCount < 1.0 ? 1.0 : ctas / kFallbackSmCount) * per_cta_us + 0.5 * per_cta_us;
+        if (!ragged && ctas <= 2.0 * kFallbackSmCount) {
+            // Two CTAs of this sweep fit on an SM, so these are all resident at once and nothing runs in waves: every
+            // SM streams its q or q + 1 blocks at its share of the bandwidth, one SM alone at 60 GB/s at most (measured:
+            // 112 CTAs of 8 MB reach 6.3 TB/s; 224 take as long as this says).
+            const double sms = kFallbackSmCount, cap = 60e3, all = 6.4e6;
+            const double q = floor(ctas / sms), more = ctas - q * sms;            // `more` SMs have q + 1 blocks
+            const double t1 = q * block_bytes / (all / sms < cap ? all / sms : cap);       // until the SMs with q blocks are done
+            const double t2 = more > 0 ? block_bytes / (all / more < cap ? all / more : cap) : 0.0;
+            cost = 2.0 + t1 + t2;
+        }
         if (cost < best * 0.999) { best = cost; schunk = c; }
     }
     if (const char* e = getenv("COMPACTOR_SCORE_BLOCK")) {              // tuning aid

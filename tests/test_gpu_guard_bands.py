@@ -87,6 +87,13 @@ def test_ragged_batch_with_tail_tiles_writes_nothing_outside_its_buffers(B):
     _compress_guarded(B, w)
 
 
+def test_wide_sketches_write_nothing_outside_their_buffers(B):
+    # sketches of more than 64 columns keep two 128 x 128 parts of the projected Gram matrix per unit, more than the
+    # narrow ones need; m = 80 is padded to 128 columns, m = 128 is the exact-score route
+    for m in (80, 128):
+        _compress_guarded(B, inputs.Workload(f"guard-wide-{m}", 1, 3, 128, [1500, 200, 333], [0.3, 0.5, 0.4], p=0.7, seed=16, m=m))
+
+
 def test_across_heads_selection_writes_nothing_outside_its_buffers(B):
     w = inputs.Workload("guard-across", 2, 3, 128, [700, 1301], [0.3, 0.4], p=0.7, seed=14)
     _, kr, v = [None if t is None else t.cuda() for t in inputs.make_tensors(w, device="cpu", want_pre=False)]

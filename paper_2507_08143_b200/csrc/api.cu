@@ -417,10 +417,10 @@ int run_scoring(HostPlan& hp, const Mat& k, const float* phi, const float* attn,
         CK(mk.mark(0, stream));
         CK(launch_gram(hp.plan, k, partials, status, stream));
         CK(mk.mark(1, stream));
-        CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, status,
+        CK(launch_factor(hp.plan, k, partials, phi, reinterpret_cast<double*>(ws + hp.off_gpart), w, scores, status,
                          factorization, eig_floor, sm_count(), stream));
         CK(mk.mark(2, stream));
-        CK(launch_score(hp.plan, k, w, scores, status, stream));
+        CK(launch_score(hp.plan, k, w, scores, status, factorization == COMPACTOR_FACTOR_CHOLESKY, stream));
         CK(mk.mark(3, stream));
     }
     if (attn != nullptr) {

@@ -15,6 +15,7 @@ constexpr int kMinChunk = 256;
 constexpr int kGramFlushTokens = 512;    // most tokens whose Gram matrix is summed in fp32 (tensor-core accumulators) before going to fp64
 constexpr int kGramElems = kD * kD;
 constexpr int kFactorSlices = 4;   // 32-row slices of the Gram matrix in its fp64 projection
+constexpr int kTinyExtra = 16;     // a unit of at most m + kTinyExtra tokens is factored with pivoting and scored in fp64 by the factor kernel
 constexpr int kFactorParts = 2;    // parts of A (G = A + A^T) per unit, one per pair of slices and work item
 
 // Device-side view of one call: shapes plus the four prefix-sum tables that live at the start
@@ -112,10 +113,12 @@ inline cudaError_t launch_chained(int which, void (*kernel)(KArgs...), dim3 grid
 // Kernel launchers (each defined next to its kernel).  All enqueue on `stream` and return the
 // launch status.
 cudaError_t launch_gram(const Plan& p, const Mat& k, double* partials, int* status, cudaStream_t stream);
+// `scores`: where the Cholesky route writes the scores of its tiny units (see kTinyExtra); the scoring sweep is then
+// told to leave those units alone (`tiny_done`).
 cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* a_parts,
-                          __nv_bfloat16* w, int* status, int factorization, double eig_floor, int sm_count,
+                          __nv_bfloat16* w, float* scores, int* status, int factorization, double eig_floor, int sm_count,
                           cudaStream_t stream);
-cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
+cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status, bool tiny_done,
                          cudaStream_t stream);
 cudaError_t launch_sweep(const SweepArgs& a, int sm_count, cudaStream_t stream);
 // parts > 1 (with `stats`, 4 doubles per unit and part): every unit's vectors are cut into that many slices.

@@ -335,9 +335,13 @@ struct CholSmem {
 // the largest original entry), one CTA per unit, a step at a time: the work is tiny and such units are rare.
 // `a` holds G by columns (lower triangle valid on entry, the whole square is used); W = Phi[:, P] L^-T comes out in
 // pivot order (the order of its columns does not matter to the scores), zero beyond the rank.  Returns the rank.
+// With `scores_unit` the unit's scores are written too, in fp64 arithmetic: o_i = || y_i ||^2, y_i the same
+// substitution applied to k^_i = Phi^T k_i (W in two bf16 terms resolves 2^-17 of its largest entries, and
+// with a G this close to singular the products k_i W cancel far below that).  `keys`: the unit's first key row.
 template <int MP>
 __device__ int pivoted_factor_and_solve(double* a, const float* phi, int m, int rank_bound, int tid, int* perm, double* red,
-                                        __nv_bfloat16* w_hi) {
+                                        __nv_bfloat16* w_hi, const __nv_bfloat16* keys, long long stride_token, int n_tok,
+                                        float* scores_unit) {
     constexpr int LD = MP;
     const int lane = tid & 31, warp = tid >> 5;
     for (int idx = tid; idx < m * m; idx += kCholThreads) {            // both triangles
@@ -405,13 +409,33 @@ __device__ int pivoted_factor_and_solve(double* a, const float* phi, int m, int 
             w_lo[j * kD + row] = __double2bfloat16(v - (double)__bfloat162float(hi));
         }
     }
+    if (scores_unit != nullptr) {
+        for (int tok = tid; tok < n_tok; tok += kCholThreads) {
+            double kh[MP], y[MP];
+            for (int j = 0; j < m; ++j) kh[j] = 0.0;
+            const __nv_bfloat16* krow = keys + (long long)tok * stride_token;
+            for (int c = 0; c < kD; ++c) {
+                const double kv = (double)__bfloat162float(krow[c]);
+                for (int j = 0; j < m; ++j) kh[j] = fma(kv, (double)phi[c * MP + j], kh[j]);
+            }
+            double o = 0.0;
+            for (int j = 0; j < rank; ++j) {
+                const int pj = perm[j];
+                double acc = kh[pj];
+                for (int t = 0; t < j; ++t) acc = fma(-y[t], a[perm[t] * LD + pj], acc);
+                y[j] = acc / a[pj * LD + pj];
+                o = fma(y[j], y[j], o);
+            }
+            scores_unit[tok] = (float)o;
+        }
+    }
     return rank;
 }
 
 template <int MP>
 __global__ void __launch_bounds__(kCholThreads, MP <= 48 ? 4 : (MP <= 64 ? 2 : 1))
-cholesky_kernel(Plan p, const double* __restrict__ a_parts, const float* __restrict__ phi,
-                __nv_bfloat16* __restrict__ w_out, int* __restrict__ status) {
+cholesky_kernel(Plan p, Mat kmat, const double* __restrict__ a_parts, const float* __restrict__ phi,
+                __nv_bfloat16* __restrict__ w_out, float* __restrict__ scores, int* __restrict__ status) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     CholSmem<MP>& s = *reinterpret_cast<CholSmem<MP>*>(chol_smem_raw);
     const int unit = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -436,12 +460,22 @@ cholesky_kernel(Plan p, const double* __restrict__ a_parts, const float* __restr
     const int n_unit = p.cu_seqlens[unit % p.batch + 1] - p.cu_seqlens[unit % p.batch];
     const bool exact_gram = n_unit <= kExactGramTokens;
     __nv_bfloat16* w_unit = w_out + (size_t)unit * w_elems_per_unit(MP);
-    if (!bad && n_unit <= m + 16) {
-        // about as many tokens as sketch columns: G is singular or nearly so, and only a pivoted factorisation is accurate
-        const int rank = pivoted_factor_and_solve<MP>(s.g, s.phi, m, n_unit, tid, s.perm, s.diag0, w_unit);
+    // about as many tokens as sketch columns: G is singular or nearly so; only a pivoted factorisation is accurate, and the
+    // scores are worked out here as well (the scoring sweep leaves such units alone)
+    const bool tiny = n_unit <= m + kTinyExtra;
+    const int b_unit = unit % p.batch, lh_unit = unit / p.batch;
+    float* scores_unit = scores == nullptr ? nullptr : scores + (size_t)lh_unit * p.total_tokens + p.cu_seqlens[b_unit];
+    if (!bad && tiny) {
+        const int layer = lh_unit / p.heads, head = lh_unit % p.heads;
+        const __nv_bfloat16* keys = kmat.ptr + layer * kmat.stride_layer + head * kmat.stride_head +
+                                    (long long)p.cu_seqlens[b_unit] * kmat.stride_token;
+        const int rank = pivoted_factor_and_solve<MP>(s.g, s.phi, m, n_unit, tid, s.perm, s.diag0, w_unit, keys,
+                                                      kmat.stride_token, n_unit, scores_unit);
         if (tid == 0 && status != nullptr && rank < m) atomicOr(&status[unit], COMPACTOR_STATUS_RANK);
         return;
     }
+    if (bad && tiny && scores_unit != nullptr)              // non-finite keys: W = 0 below, and so are the scores
+        for (int tok = tid; tok < n_unit; tok += kCholThreads) scores_unit[tok] = 0.f;
     if (tid < MP) s.diag0[tid] = s.g[tid * MP + tid] * (exact_gram ? 9.5367431640625e-07 : 1.0);
     __syncthreads();
     if (!bad) cholesky_panels<MP, kCholWarps>(s.g, s.diag0, s.inv_diag, m, tid, &s.flags, sync, exact_gram ? n_unit : (1 << 30));
@@ -639,7 +673,7 @@ eig_kernel(Plan p, const double* __restrict__ a_parts, const float* __restrict__
 
 template <int MP>
 cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials, const float* phi,
-                             double* a_parts, __nv_bfloat16* w, int* status, int factorization, double eig_floor,
+                             double* a_parts, __nv_bfloat16* w, float* scores, int* status, int factorization, double eig_floor,
                              int sm_count, cudaStream_t stream) {
     const int units = p.layers * p.heads * p.batch;
     const int smem = (int)sizeof(ProjectSmem<MP>);
@@ -665,7 +699,7 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
         const int csmem = (int)sizeof(CholSmem<MP>);
         e = cudaFuncSetAttribute(cholesky_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, csmem);
         if (e != cudaSuccess) return e;
-        e = launch_chained(kPdlCholesky, cholesky_kernel<MP>, dim3(units), dim3(kCholThreads), csmem, stream, p, (const double*)a_parts, phi, w, status);
+        e = launch_chained(kPdlCholesky, cholesky_kernel<MP>, dim3(units), dim3(kCholThreads), csmem, stream, p, k, (const double*)a_parts, phi, w, scores, status);
         if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();
@@ -674,15 +708,15 @@ cudaError_t launch_factor_mp(const Plan& p, const Mat& k, const double* partials
 }  // namespace
 
 cudaError_t launch_factor(const Plan& p, const Mat& k, const double* partials, const float* phi, double* a_parts,
-                          __nv_bfloat16* w, int* status, int factorization, double eig_floor, int sm_count,
+                          __nv_bfloat16* w, float* scores, int* status, int factorization, double eig_floor, int sm_count,
                           cudaStream_t stream) {
     if (p.layers * p.heads * p.batch == 0) return cudaSuccess;
     switch (p.mp) {
-        case 16: return launch_factor_mp<16>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
-        case 32: return launch_factor_mp<32>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
-        case 48: return launch_factor_mp<48>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
-        case 64: return launch_factor_mp<64>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
-        case 128: return launch_factor_mp<128>(p, k, partials, phi, a_parts, w, status, factorization, eig_floor, sm_count, stream);
+        case 16: return launch_factor_mp<16>(p, k, partials, phi, a_parts, w, scores, status, factorization, eig_floor, sm_count, stream);
+        case 32: return launch_factor_mp<32>(p, k, partials, phi, a_parts, w, scores, status, factorization, eig_floor, sm_count, stream);
+        case 48: return launch_factor_mp<48>(p, k, partials, phi, a_parts, w, scores, status, factorization, eig_floor, sm_count, stream);
+        case 64: return launch_factor_mp<64>(p, k, partials, phi, a_parts, w, scores, status, factorization, eig_floor, sm_count, stream);
+        case 128: return launch_factor_mp<128>(p, k, partials, phi, a_parts, w, scores, status, factorization, eig_floor, sm_count, stream);
         default: return cudaErrorInvalidValue;
     }
 }

@@ -53,7 +53,7 @@ struct __align__(1024) ScoreSmem {
 template <int MP>
 __global__ void __launch_bounds__(kThreads, 1)
 score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap wmap,
-             float* __restrict__ scores, int* __restrict__ status, int chained) {
+             float* __restrict__ scores, int* __restrict__ status, int chained, int tiny_done) {
     extern __shared__ unsigned char smem_raw[];
     using Smem = ScoreSmem<MP>;
     constexpr int kStages = Smem::kStages;
@@ -71,6 +71,13 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
     const int n_tiles = (n_tok + kTile - 1) / kTile;
     const int unit = lh * p.batch + b;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // a unit about as short as the sketch is wide has been scored in fp64 by the factor kernel (W in two bf16 terms
+    // is too coarse for its nearly singular G).  In a chained launch this grid must not be complete before the factor
+    // kernel is: what follows waits for this grid alone.
+    if (tiny_done && p.cu_seqlens[b + 1] - p.cu_seqlens[b] <= p.m + kTinyExtra) {
+        pdl_wait();
+        return;
+    }
 
     if (threadIdx.x == 0) {
         prefetch_tensormap(&kmap);
@@ -231,20 +238,20 @@ score_kernel(Plan p, const __grid_constant__ CUtensorMap kmap, const __grid_cons
 
 template <int MP>
 cudaError_t launch_score_mp(const Plan& p, const CUtensorMap& kmap, const CUtensorMap& wmap, float* scores,
-                            int* status, cudaStream_t stream) {
+                            int* status, bool tiny_done, cudaStream_t stream) {
     const int smem = (int)sizeof(ScoreSmem<MP>) + 1024;
     cudaError_t e = cudaFuncSetAttribute(score_kernel<MP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     dim3 grid(p.total_schunks, p.layers * p.heads);
     e = launch_chained(kPdlScore, score_kernel<MP>, grid, dim3(kThreads), smem, stream, p, kmap, wmap, scores, status,
-                       pdl_enabled(kPdlScore) ? 1 : 0);
+                       pdl_enabled(kPdlScore) ? 1 : 0, tiny_done ? 1 : 0);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status,
+cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, float* scores, int* status, bool tiny_done,
                          cudaStream_t stream) {
     if (p.total_schunks == 0) return cudaSuccess;
     CUtensorMap kmap, wmap;
@@ -254,11 +261,11 @@ cudaError_t launch_score(const Plan& p, const Mat& k, const __nv_bfloat16* w, fl
         !make_rows_tensor_map(&wmap, w, units * 2 * p.mp, p.mp))
         return cudaErrorInvalidValue;
     switch (p.mp) {
-        case 16: return launch_score_mp<16>(p, kmap, wmap, scores, status, stream);
-        case 32: return launch_score_mp<32>(p, kmap, wmap, scores, status, stream);
-        case 48: return launch_score_mp<48>(p, kmap, wmap, scores, status, stream);
-        case 64: return launch_score_mp<64>(p, kmap, wmap, scores, status, stream);
-        case 128: return launch_score_mp<128>(p, kmap, wmap, scores, status, stream);
+        case 16: return launch_score_mp<16>(p, kmap, wmap, scores, status, tiny_done, stream);
+        case 32: return launch_score_mp<32>(p, kmap, wmap, scores, status, tiny_done, stream);
+        case 48: return launch_score_mp<48>(p, kmap, wmap, scores, status, tiny_done, stream);
+        case 64: return launch_score_mp<64>(p, kmap, wmap, scores, status, tiny_done, stream);
+        case 128: return launch_score_mp<128>(p, kmap, wmap, scores, status, tiny_done, stream);
         default: return cudaErrorInvalidValue;
     }
 }

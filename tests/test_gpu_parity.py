@@ -507,3 +507,35 @@ def test_fewer_tokens_than_sketch_columns_any_sketch_width(B, m):
                 got = sc[0, h, cu[b]:cu[b + 1]].cpu().numpy().astype(np.float64)
                 np.testing.assert_allclose(want, 1.0, rtol=1e-6)
                 np.testing.assert_allclose(got, want, rtol=1e-3, err_msg=f"m {m} p {p_exp} n {n}")
+
+
+@pytest.mark.parametrize("m", [16, 48, 64, 96])
+def test_sequences_about_as_long_as_the_sketch_is_wide(B, m):
+    # n in m - 1 .. m + 16: G is singular or nearly so (cond(G) up to 1e9 with these keys), and W in two bf16 terms is too
+    # coarse for it (errors of 1e-3 and more); such units are scored in fp64 by the factor kernel, and the scoring
+    # sweep leaves them alone.  The longer sequence beside them goes the ordinary way.
+    for p_exp in (0.7, 1.0):
+        ns = [m - 1, m, m + 1, m + 8, m + 16, m + 17, 900]
+        w = inputs.Workload("near-m", 1, 2, 128, ns, [0.5] * len(ns), p=p_exp, seed=4100 + m, m=m)
+        kp, kr, v = [t.cuda() for t in inputs.make_tensors(w, device="cpu")]
+        shape = B.Shape(1, 2, 128, m, ns)
+        phi = inputs.make_sketch_matrix(128, m, 2)
+        sc = torch.full((1, 2, shape.total_tokens), float("nan"), dtype=torch.float32, device="cuda")
+        B.score(shape, kp, phi.cuda(), sc, B.alloc_workspace(shape))
+        torch.cuda.synchronize()
+        cu = shape.cu_seqlens
+        for h in range(2):
+            for b, n in enumerate(ns):
+                K = orc.bf16_bits_to_f64(H.bits(kp[0, h, cu[b]:cu[b + 1]]))
+                want = orc.approx_leverage_scores(K, phi.numpy())
+                got = sc[0, h, cu[b]:cu[b + 1]].cpu().numpy().astype(np.float64)
+                tol = 1e-4 if n <= m + 16 else 1e-3          # measured: 3e-5 at n = m with the steep spectrum, 1e-7 elsewhere
+                np.testing.assert_allclose(got, want, rtol=tol, err_msg=f"m {m} p {p_exp} n {n}")
+
+
+def test_blend_with_a_sequence_one_longer_than_the_sketch(B):
+    # n = m + 1: the leverage scores are all close to one, so Eq. 6's z-score magnifies their errors by mean / spread
+    # (a random batch had 1.2e-3 here while W in two bf16 terms was used for such units)
+    w = inputs.Workload("near-m-blend", 1, 1, 128, [65628, 49], [1.0, 1.0], p=0.7, seed=2913)
+    worst, band, outs = _run_workload(B, w, attn=True, device="cpu")
+    assert worst < 2e-4, worst

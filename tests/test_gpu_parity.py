@@ -506,7 +506,7 @@ def test_fewer_tokens_than_sketch_columns_any_sketch_width(B, m):
                 want = orc.approx_leverage_scores(K, phi.numpy())
                 got = sc[0, h, cu[b]:cu[b + 1]].cpu().numpy().astype(np.float64)
                 np.testing.assert_allclose(want, 1.0, rtol=1e-6)
-                np.testing.assert_allclose(got, want, rtol=1e-3, err_msg=f"m {m} p {p_exp} n {n}")
+                np.testing.assert_allclose(got, want, rtol=1e-5, err_msg=f"m {m} p {p_exp} n {n}")   # scored in fp64: 1e-7 measured
 
 
 @pytest.mark.parametrize("m", [16, 48, 64, 96])

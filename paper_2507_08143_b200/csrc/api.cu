@@ -142,6 +142,12 @@ bool make_plan(const compactor_shape* s, HostPlan* hp, int* err, bool allow_fuse
     compactor::set_chain_for((long long)s->layers * s->heads * p.total_tokens * kD * 2);
     hp->units = s->layers * s->heads * s->batch;
     hp->fused = allow_fused && p.mp <= kFusedMaxMp && fused_sweep_enabled();
+    // the one-kernel sweep has no pivoted factorisation and no fp64 scores for sequences about as short as the sketch is
+    // wide: a batch with one of those takes the separate kernels
+    for (int b = 0; b < s->batch && hp->fused; ++b) {
+        const int n = s->cu_seqlens[b + 1] - s->cu_seqlens[b];
+        if (n > 0 && n <= s->m + kTinyExtra) hp->fused = false;
+    }
     hp->slices = 0; hp->window = 0; hp->n_slots = 0; hp->max_pieces = 0; hp->total_pieces = 0;
     hp->off_sched = 0; hp->sched_bytes = 0; hp->off_tbuf = 0;
 

@@ -362,6 +362,27 @@ def test_nonfinite_input_sets_status_and_returns(B):
     assert len(np.unique(i)) == 300 and i.min() >= 0 and i.max() < 600
 
 
+def test_nonfinite_key_in_a_sequence_about_as_short_as_the_sketch(B):
+    # such a unit is scored by the factor kernel, not by the scoring sweep: its scores must still be written (zeros, as
+    # W = 0 gives elsewhere), its status set, and its neighbours untouched
+    w = inputs.Workload("nan-tiny", 1, 2, 128, [50, 700, 20], [0.5, 0.5, 0.5], seed=72)
+    _, kr, v = inputs.make_tensors(w, device="cpu", want_pre=False)
+    kr[0, 1, 17, 3] = float("inf")                      # head 1, first sequence (50 tokens)
+    kr, v = kr.cuda(), v.cuda()
+    shape = B.Shape(1, 2, 128, 48, w.seqlens)
+    keep = [25, 350, 10]
+    phi = inputs.make_sketch_matrix(128, 48, 1)
+    scores, idx, ko, vo, status = H.run_compress(B, shape, kr, kr, v, phi, keep)
+    st = status.cpu().numpy()
+    assert (st[3] & 1) and st[0] in (0, 2) and st[4] == 0 and (st[5] & 2) and (st[2] & 2)   # units: head * 3 + sequence
+    s = scores.cpu().numpy()
+    assert np.all(s[0, 1, :50] == 0.0) and np.all(np.isfinite(s))
+    i = idx[0, 1, :25].cpu().numpy()
+    np.testing.assert_array_equal(i, np.arange(25))     # all scores equal: ties go to the lower index
+    H.compare_all_units(shape, keep, (scores, idx, ko, vo, status), kr, kr, v, phi, units=[(0, 0, 0), (0, 0, 1), (0, 1, 1), (0, 1, 2)],
+                        what="nan-tiny")
+
+
 @pytest.mark.parametrize("name,layers,heads", [("c1", 2, None), ("c2", 1, None), ("c4", 1, 2)])
 def test_benchmark_shapes_reduced_layers(B, name, layers, heads):
     w = inputs.workload(name, layers=layers)

@@ -8,11 +8,13 @@
 //                    mma.m8n8k4 (this is where the fp64 work is: 0.8 M multiply-adds per unit,
 //                    spread over the whole device) and writes an m x m part of A.
 //   cholesky_kernel  one small CTA per unit, several per SM: G = sum of the parts and their
-//                    transposes, G = L L^T by
-//                    panels of eight columns (the 8 x 8 diagonal blocks are factored redundantly
-//                    by every lane of a warp, so no pivot has to travel), then W = Phi L^-T as a
-//                    blocked substitution on fp64 mma, split into two bf16 terms.  The score of a
-//                    key row k_i is then || k_i W ||^2 (Algorithm 1, lines 5-6).
+//                    transposes, G = L L^T by panels of eight columns (the 8 x 8 diagonal blocks
+//                    are factored redundantly by every lane of a warp, so no pivot has to travel),
+//                    then W = Phi L^-T as a blocked substitution on fp64 mma, split into two bf16
+//                    terms.  The score of a key row k_i is then || k_i W ||^2 (Algorithm 1, lines
+//                    5-6), which the scoring sweep computes.  A unit about as short as the sketch
+//                    is wide (n <= m + 16) has a G too close to singular for that: it is factored
+//                    with diagonal pivoting and its scores are written here, in fp64.
 //
 // Rank handling: a pivot not larger than 2^-20 of its original diagonal entry (the fp32 noise
 // floor of the fp32 Gram runs) is treated as a direction of the null space and dropped;
